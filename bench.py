@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the batch-1 dual-sparse decode product y = W.x on RLC-CSC weights.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl celty|reference] [--workload NAME]
+
+A step is one celty_spmspv call (activation compaction, column fetch, run-length decode,
+shared-memory accumulation, reduction to y) on the Llama-2-7B attention shape (4096 x 4096, W
+magnitude-pruned 50% per column, x ~ Laplace thresholded to 50% density).  Calls rotate over
+device copies of the layer whose total size exceeds twice the L2, so every call reads HBM.
+Prints ONE JSON line (see the design doc for the keys).  `--impl reference` times the CPU oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_01536_b200 import synth  # noqa: E402
+
+METRIC = "SpMSpV achieved HBM GB/s on fetched bytes (batch 1)"
+
+WORKLOADS = {
+    # name: (M, K, weight sparsity, mask family, activation dist, activation density, config id)
+    "llama7b_attn_4096x4096_s50_a50": (4096, 4096, 0.5, "magnitude", "laplace", 0.5, 2),
+    "llama7b_gateup_11008x4096_s50_a50": (11008, 4096, 0.5, "magnitude", "laplace", 0.5, 3),
+    "llama7b_down_4096x11008_s50_a50": (4096, 11008, 0.5, "magnitude", "swiglu", 0.5, 3),
+    "llama13b_attn_5120x5120_s50_a40": (5120, 5120, 0.5, "bernoulli", "laplace", 0.4, 4),
+    "llama70b_mlp_28672x8192_s50_a50": (28672, 8192, 0.5, "bernoulli", "laplace", 0.5, 5),
+    "small_1024x1024_s50_a50": (1024, 1024, 0.5, "bernoulli", "normal", 0.5, 1),
+}
+DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"
+
+
+def make_layer(name: str, variant: int):
+    M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
+    seed = synth.point_seed(cfg, variant)
+    W = synth.weights(seed, M, K)
+    if family == "magnitude":
+        mask = synth.mask_magnitude(W, s)
+    elif family == "bernoulli":
+        mask = synth.mask_bernoulli(seed, M, K, 1.0 - s)
+    else:
+        mask = synth.mask_powerlaw(seed, M, K, 1.0 - s)
+    return W, mask
+
+
+def make_x(name: str, variant: int):
+    M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
+    x = synth.activations(synth.point_seed(cfg, 50 + variant), K, dist)
+    return x, synth.threshold_for_density(x, d_a)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def oracle_seconds_per_call(name: str, budget_s: float, threads: int):
+    """The oracle's plain definition on the bench workload, repeated for about budget_s seconds."""
+    from oracle import celty_oracle as orc
+    W, mask = make_layer(name, 0)
+    x, tau = make_x(name, 0)
+    orc.masked_gemv(W[:64], mask[:64], x, tau, threads=threads)          # load the library
+    t0 = time.perf_counter()
+    calls = 0
+    while True:
+        orc.masked_gemv(W, mask, x, tau, threads=threads)
+        calls += 1
+        if time.perf_counter() - t0 >= budget_s:
+            break
+    return (time.perf_counter() - t0) / calls, calls
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import celty_oracle as orc
+    from paper_2608_01536_b200 import build as lib_build, celty
+    name = args.workload
+    M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
+    W, mask = make_layer(name, 0)
+    x, tau = make_x(name, 0)
+    threads = orc.max_threads()
+    t0 = time.perf_counter()
+    orc.masked_gemv(W, mask, x, tau, threads=threads)
+    t_full = time.perf_counter() - t0
+    # rows sampled per step so that warmup + steps stay within about two minutes
+    frac = min(1.0, 100.0 / max(1e-9, (args.steps + args.warmup) * t_full))
+    rows = max(1, int(M * frac))
+    Ws, ms = np.ascontiguousarray(W[:rows]), np.ascontiguousarray(mask[:rows])
+    for _ in range(args.warmup):
+        orc.masked_gemv(Ws, ms, x, tau, threads=threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.masked_gemv(Ws, ms, x, tau, threads=threads)
+    dt = (time.perf_counter() - t0) / args.steps
+    sec_per_call = dt * (M / rows)
+    # bytes the GPU path would fetch for this call: host-side table arithmetic of the library
+    lib_build.build()
+    idx = orc.compact(x, tau)[0]
+    total_bytes = celty.Matrix(W, mask).fetched_bytes(idx)[1]
+    gbs = total_bytes / sec_per_call / 1e9
+    sample = f"rows 0..{rows - 1} of {M} per step, scaled to a full call"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_per_call * 1e3,
+        "us_per_call": sec_per_call * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": name, "M": M, "K": K, "weight_sparsity": s, "activation_density": d_a},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_celty(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_01536_b200 import build as lib_build, celty
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lib_build.build()
+    celty.load()
+    dev = torch.device("cuda", local)
+    name = args.workload
+    M, K, s, family, dist_name, d_a, cfg = WORKLOADS[name]
+    layout = celty.LAYOUT_COLUMN if args.layout == "column" else celty.LAYOUT_LANE_TILE
+
+    # ---- workload: a few distinct matrices, replicated on the device until the copies exceed 2x L2
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    distinct = [make_layer(name, v) for v in range(args.distinct)]
+    probe = celty.Matrix(*distinct[0], layout=layout)
+    image_bytes = probe.device_bytes()[0]
+    copies = max(args.distinct, int(np.ceil(2.5 * l2 / image_bytes)) + 1)
+    if args.copies:
+        copies = args.copies
+    mats, xs, taus, fetched = [], [], [], []
+    for c in range(copies):
+        W, mask = distinct[c % args.distinct]
+        m = celty.Matrix(W, mask, layout=layout, device=dev)
+        if args.grid or args.variant:
+            m.set_launch(args.grid, args.variant)
+        x, tau = make_x(name, c)
+        mats.append(m)
+        xs.append(torch.from_numpy(x).to(dev))
+        taus.append(tau)
+    ys = [torch.empty(M, dtype=torch.float32, device=dev) for _ in range(copies)]
+    torch.cuda.synchronize()
+
+    def call(c):
+        mats[c].spmspv(xs[c], taus[c], ys[c])
+
+    # bytes per call (host arithmetic on the library's tables, from the oracle-free compacted list)
+    for c in range(copies):
+        call(c)
+        idx, _ = mats[c].last_compaction()
+        fetched.append(mats[c].fetched_bytes(idx.cpu().numpy()))
+        assert mats[c].last_status() == 0
+    stream_bytes = float(np.mean([f[0] for f in fetched]))
+    total_bytes = float(np.mean([f[1] for f in fetched]))
+    info = mats[0].info()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up, then one CUDA graph holding one rotation over all copies
+    for i in range(max(3, args.warmup)):
+        call(i % copies)
+    torch.cuda.synchronize()
+    graph = None
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for c in range(copies):
+                call(c)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+    reps, rem = (args.steps // copies, args.steps % copies) if graph is not None else (0, args.steps)
+
+    def timed_region():
+        for _ in range(reps):
+            graph.replay()
+        for i in range(rem):
+            call(i % copies)
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        barrier()
+        e0.record()
+        timed_region()
+        e1.record()
+        barrier()
+    ms = e0.elapsed_time(e1)
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    sec_per_call = ms / 1e3 / args.steps
+    gbs = world * total_bytes / sec_per_call / 1e9
+
+    # ---- stream-enqueued (no graph) and L2-warm numbers, for context
+    def time_calls(fn, n):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(n):
+            fn(i)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n * 1e3
+    n_ctx = min(args.steps, 2000)
+    us_enqueued = time_calls(lambda i: call(i % copies), n_ctx)
+    us_warm = None
+    if graph is not None:
+        gw = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gw):
+            for _ in range(copies):
+                call(0)
+        gw.replay()
+        us_warm = time_calls(lambda i: gw.replay(), max(1, n_ctx // copies)) / copies
+
+    # ---- end to end through the host-buffer entry point: pinned x in, y out, every step
+    xh = [torch.from_numpy(make_x(name, c)[0]).pin_memory() for c in range(copies)]
+    yh = torch.empty(M, dtype=torch.float32).pin_memory()
+    xstage = torch.empty(K, dtype=torch.float16, device=dev)
+    n_e2e = min(args.steps, 2000)
+    for i in range(5):
+        mats[i % copies].spmspv_host(xh[i % copies], taus[i % copies], yh, xstage, ys[0])
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(n_e2e):
+        c = i % copies
+        mats[c].spmspv_host(xh[c], taus[c], yh, xstage, ys[0])
+    barrier()
+    e2e_sec = (time.perf_counter() - t0) / n_e2e
+    t = torch.tensor([e2e_sec], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_sec = float(t.item())
+
+    # ---- dense cuBLAS GEMV on the same GPU, same rotation (context, not the target)
+    dense_us = None
+    if not args.no_dense:
+        Wd = [torch.from_numpy(distinct[c % args.distinct][0]).to(dev) for c in range(min(copies, 12))]
+        if len(Wd) * Wd[0].numel() * 2 < 2 * l2:
+            Wd = Wd + [w.clone() for w in Wd]
+        yd = torch.empty(M, dtype=torch.float16, device=dev)
+        gd = torch.cuda.CUDAGraph()
+        torch.mv(Wd[0], xs[0], out=yd)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(gd):
+            for c in range(len(Wd)):
+                torch.mv(Wd[c], xs[c % copies], out=yd)
+        gd.replay()
+        dense_us = time_calls(lambda i: gd.replay(), max(3, n_ctx // len(Wd))) / len(Wd)
+        del Wd
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_src = measured_peaks()
+    out = {
+        "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": sec_per_call * 1e3, "us_per_call": sec_per_call * 1e6,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": name, "M": M, "K": K, "weight_sparsity": s, "mask": family, "activations": dist_name,
+            "activation_density": d_a, "layout": "column" if layout == celty.LAYOUT_COLUMN else "lane_tile",
+            "tile_rows": info.tile_rows, "l2": f"rotation over {copies} device copies ({args.distinct} distinct "
+            f"matrices, {copies} distinct x), {copies * image_bytes / 1e6:.0f} MB > 2x L2 ({l2 / 1e6:.0f} MB)",
+            "launch": "cuda graph of one rotation" if graph is not None else "stream enqueue",
+            "multi_gpu": "replicas only" if world > 1 else "single",
+        },
+        "bytes_per_call": {"entry_stream": stream_bytes, "total": total_bytes, "dense_fp16": 2.0 * M * K,
+                           "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad},
+        "roofline": {"bound": "hbm", "achieved": total_bytes / sec_per_call / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": total_bytes / sec_per_call / 1e9 / peak, "traffic": None, "peak_source": peak_src,
+                     "note": "time per call covers every kernel of the call"},
+        "e2e": {"value": world * total_bytes / e2e_sec / 1e9, "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
+                "h2d_bytes_per_step": 2 * K, "d2h_bytes_per_step": 4 * M},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks.summary(),
+        "context": {"us_per_call_stream_enqueued": us_enqueued, "us_per_call_l2_warm": us_warm,
+                    "cublas_gemv_fp16_us": dense_us,
+                    "speedup_vs_cublas_gemv": (dense_us / (sec_per_call * 1e6)) if dense_us else None},
+    }
+    if world == 1 and not args.no_cpu:
+        from oracle import celty_oracle as orc
+        threads = orc.max_threads()
+        sec, calls = oracle_seconds_per_call(name, args.cpu_seconds, threads)
+        out["cpu_baseline"] = {"value": total_bytes / sec / 1e9, "unit": "GB/s", "us_per_call": sec * 1e6,
+                               "cores": threads, "kind": "oracle",
+                               "sample": f"{calls} full calls of the fp64 masked product on this workload"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="celty", choices=["celty", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--layout", default="lane_tile", choices=["lane_tile", "column"])
+    ap.add_argument("--distinct", type=int, default=2, help="distinct synthetic matrices behind the copies")
+    ap.add_argument("--copies", type=int, default=0, help="device copies in the rotation (0 = enough for 2.5x L2)")
+    ap.add_argument("--grid", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_celty(args)
+
+
+if __name__ == "__main__":
+    main()

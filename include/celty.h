@@ -1,0 +1,215 @@
+/*
+ * celty.h -- C ABI of the B200 (sm_100a) library for the batch-1 dual-sparse decode product
+ *
+ *     y = W . x      W: M x K, unstructured-pruned FP16, stored in 4-bit run-length coded CSC
+ *                    x: K FP16 activations, made sparse at run time by magnitude thresholding
+ *                    y: M FP32
+ *
+ * (Celty: sparse format Section 3.2, kernel formulation Section 3.1, index reconstruction
+ * Algorithm 1, shared-memory scatter-accumulation Section 3.3.)
+ *
+ * Conventions
+ *   - Every function returns 0 (CELTY_OK) or a negative celty_status; nothing throws or aborts.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA device memory of the
+ *     current device.  The library never allocates device memory: the caller provides it
+ *     (celty_device_bytes says how much) and keeps it alive while the handle uses it.
+ *   - celty_stream_t is a cudaStream_t passed as void* (NULL = the default stream).  Calls that
+ *     take a stream only enqueue work on it and return without synchronising unless stated.
+ *   - M = rows = outputs, K = columns = inputs.  W and mask are row-major on the host.
+ *   - One handle must not be used from two streams or two threads at the same time: the
+ *     compacted activation list and the status word live in the handle's workspace.
+ */
+#ifndef CELTY_H
+#define CELTY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct celty_matrix celty_matrix;   /* opaque: host copy of the encoded matrix + device binding */
+typedef void *celty_stream_t;               /* cudaStream_t */
+
+typedef enum {
+    CELTY_OK = 0,
+    CELTY_EINVAL = -1,     /* null pointer, size out of range, misaligned vector, bad option, tau < 0 or not finite */
+    CELTY_ENOMEM = -2,     /* host allocation failed, or a caller-provided device buffer is too small */
+    CELTY_ECUDA = -3,      /* a CUDA runtime call failed; celty_last_cuda_error() returns its code */
+    CELTY_ESTATE = -4,     /* handle not bound to device memory yet */
+    CELTY_ETIMEOUT = -5,   /* device status word: a bounded wait inside a kernel ran out */
+    CELTY_EBOUNDS = -6     /* device status word: a decoded row or list index was out of range */
+} celty_status;
+
+/* Device-image layouts.  Both hold exactly the (value, 4-bit run) entries that Section 3.2
+ * defines, one run per value; they differ in how entries are grouped for the kernel.
+ *   CELTY_LAYOUT_COLUMN     tile_rows must be 0: runs are counted along the whole column.
+ *                           A warp decodes 256 consecutive entries at a time with the intra-warp
+ *                           prefix sum of Algorithm 1 and scatters with shared-memory atomics.
+ *   CELTY_LAYOUT_LANE_TILE  tile_rows = R > 0: the rule of Section 3.2 is applied separately to
+ *                           consecutive tiles of R rows (the row partition of Section 3.1 taken
+ *                           down to one tile per lane).  Lane L of a warp owns tile 32*s + L, so
+ *                           every lane writes its own shared-memory bank: no conflicts, no atomics.
+ */
+enum { CELTY_LAYOUT_COLUMN = 0, CELTY_LAYOUT_LANE_TILE = 1 };
+
+typedef struct {
+    int32_t run_bits;    /* must be 4 (Section 3.2: "Celty uses 4-bit RLC-CSC")                      */
+    int32_t layout;      /* CELTY_LAYOUT_COLUMN or CELTY_LAYOUT_LANE_TILE                             */
+    int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: rows per tile, 1..2040, or 0 = choose      */
+    int32_t reserved;    /* must be 0                                                                 */
+} celty_encode_opts;
+
+/*
+ * celty_encode -- offline packing of a pruned weight matrix into RLC-CSC (Section 3.2, Fig. 2(a)).
+ *   W_host     M x K FP16 bit patterns, row-major, leading dimension ldw (elements, >= K).
+ *   mask_host  M x K bytes, row-major, leading dimension K; non-zero = the weight is kept.
+ *              NULL keeps every weight whose value is not +-0.
+ *   opts       NULL = { 4, CELTY_LAYOUT_LANE_TILE, 0, 0 }.
+ *   out        receives a new handle (free it with celty_destroy).
+ * Per column (per row tile), rows ascending: every kept weight becomes one entry (value, run) with
+ * run = number of dropped rows since the previous entry; a gap larger than 15 first emits
+ * zero-valued padding entries (run 15, each standing for 15 dropped rows plus its own row).
+ * Nothing is emitted after the last kept row.  The caller keeps ownership of W_host and mask_host;
+ * the handle copies what it needs.  Limits: 1 <= M <= 49152 (one thread block's FP32 accumulators
+ * must fit shared memory), 1 <= K < 2^31, at most 2^32 - 1 stored entries, at most 1024 tiles.
+ * Errors: CELTY_EINVAL, CELTY_ENOMEM.
+ */
+int celty_encode(const uint16_t *W_host, int64_t ldw, const uint8_t *mask_host, int64_t M, int64_t K,
+                 const celty_encode_opts *opts, celty_matrix **out);
+
+/* Frees the handle and its host memory.  Device buffers stay with the caller.  NULL is allowed. */
+void celty_destroy(celty_matrix *m);
+
+/*
+ * celty_info -- sizes of the encoded matrix.  Any output pointer may be NULL.
+ *   nnz               kept weights;  n_pad: padding entries;  stored entries = nnz + n_pad
+ *   compressed_bytes  2.5 bytes per stored entry + 4 bytes per column pointer: the figure the
+ *                     "compression efficiency" of Section 3.2 is the ratio of, over 2*M*K
+ *   tile_rows, layout the values in effect (after "0 = choose")
+ */
+int celty_info(const celty_matrix *m, int64_t *M, int64_t *K, int64_t *nnz, int64_t *n_pad,
+               int64_t *compressed_bytes, int32_t *layout, int32_t *tile_rows);
+
+/*
+ * celty_decode_host -- the stored entries of column `col`, decoded on the host from the handle's
+ * own packed image (round-trip tests): absolute row (Algorithm 1: prefix sum of runs + ordinal),
+ * FP16 bit pattern, run and pad flag of each entry, row tiles concatenated in ascending order.
+ * cap = capacity of the output arrays (entries); *n receives the entry count even when it exceeds
+ * cap (then nothing is written and CELTY_ENOMEM is returned).  Output pointers may be NULL.
+ */
+int celty_decode_host(const celty_matrix *m, int64_t col, int32_t *rows, uint16_t *vals, uint8_t *runs,
+                      uint8_t *is_pad, int64_t cap, int64_t *n);
+
+/*
+ * celty_host_image -- read-only view of the packed image held by the handle (what
+ * celty_bind_device copies to the device): pointer, size, and the offset at which the entry
+ * stream starts (column metadata comes first).  Valid until celty_destroy.  The runs of 8
+ * consecutive entries of a lane share one little-endian 32-bit word, entry e in bits 4e..4e+3.
+ */
+int celty_host_image(const celty_matrix *m, const void **image, size_t *image_bytes, size_t *stream_offset);
+
+/*
+ * celty_device_bytes -- how much device memory the caller must provide:
+ *   image_bytes      the packed matrix as the kernels read it (column metadata + entry stream)
+ *   workspace_bytes  per-handle scratch: compacted activation list (indices, values, count) and
+ *                    the status word
+ * Both are multiples of 256; the buffers must be 256-byte aligned.
+ */
+int celty_device_bytes(const celty_matrix *m, size_t *image_bytes, size_t *workspace_bytes);
+
+/*
+ * celty_bind_device -- attach caller-owned device memory and enqueue the host-to-device copy of
+ * the image (and the clearing of the workspace) on `stream`.  The host image is ordinary pageable
+ * memory, so the copy may block the calling thread; the handle is usable on `stream` on return
+ * and on other streams after the caller has synchronised.
+ * Errors: CELTY_EINVAL, CELTY_ENOMEM (buffer too small or misaligned), CELTY_ECUDA.
+ */
+int celty_bind_device(celty_matrix *m, void *image_dev, size_t image_bytes, void *workspace_dev,
+                      size_t workspace_bytes, celty_stream_t stream);
+
+/*
+ * celty_compact -- activation compaction alone (magnitude thresholding, Sections 1 and 2.1; the
+ * column skip of Section 3.1 made explicit):  S = { j : not(|x_j| <= tau) } in ascending j,
+ * compared in FP32 after exact widening (tau = 0 drops exactly +-0; NaN survives).
+ *   x_dev      K FP16 values (device, 16-byte aligned), not modified
+ *   idx_dev    int32[K]   receives the surviving column indices   (device)
+ *   val_dev    uint16[K]  receives their FP16 bit patterns        (device)
+ *   count_dev  int32[1]   receives |S|                            (device)
+ * Errors: CELTY_EINVAL (null, K <= 0, tau < 0 or not finite), CELTY_ECUDA.
+ */
+int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *idx_dev, uint16_t *val_dev,
+                  int32_t *count_dev, celty_stream_t stream);
+
+/*
+ * celty_spmspv -- the hot path: y = W . threshold(x, tau), batch 1 (Sections 3.1-3.3).
+ * Enqueues on `stream`: activation compaction (+ clearing y), then the SpMSpV kernel that visits
+ * only the surviving columns, decodes their runs to rows, accumulates value * x_j in shared memory
+ * in FP32 (fmaf) and reduces the partial sums into y.
+ *   x_dev  K FP16 (device, 16-byte aligned), not modified
+ *   y_dev  M FP32 (device, 16-byte aligned), overwritten
+ * The order of FP32 additions is not fixed (Section 4.2: scatter-accumulation is order-
+ * independent), so results may differ in the last bits between calls.  Inputs must be finite for
+ * the result to equal the definition in every row (a pad times an infinite x_j is NaN).
+ * Errors: CELTY_EINVAL, CELTY_ESTATE, CELTY_ECUDA.  Device-side problems (a bounded wait that ran
+ * out, an out-of-range index) do not fault: they set the status word, see celty_last_status.
+ */
+int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, celty_stream_t stream);
+
+/*
+ * celty_spmspv_host -- the same call for HOST vectors: copies x_host (K FP16) to x_stage_dev,
+ * runs celty_spmspv into y_stage_dev, copies it to y_host (M FP32) and synchronises `stream`
+ * before returning.  Use page-locked host memory for the copies to be asynchronous.
+ * x_stage_dev (2K bytes) and y_stage_dev (4M bytes) are caller-provided device buffers.
+ */
+int celty_spmspv_host(celty_matrix *m, const void *x_host, float tau, void *y_host, void *x_stage_dev,
+                      void *y_stage_dev, celty_stream_t stream);
+
+/*
+ * celty_last_compaction -- device pointers into the handle's workspace holding the list the last
+ * celty_spmspv produced (valid after that call's work on its stream has finished): |S|, indices,
+ * FP16 values.  For parity tests and for byte accounting.
+ */
+int celty_last_compaction(const celty_matrix *m, const int32_t **count_dev, const int32_t **idx_dev,
+                          const uint16_t **val_dev);
+
+/*
+ * celty_decode_device -- run the kernels' own run-length decoder (the device function the SpMSpV
+ * kernel uses) on column `col` of the bound image and write, for each stored entry, in
+ * the order of celty_decode_host, its absolute row and FP16 bit pattern (slots that exist only to
+ * fill a 16-byte group are skipped).  rows_dev / vals_dev have room for cap entries;
+ * count_dev[0] receives the number written.  For bit-exact decode parity tests.
+ */
+int celty_decode_device(celty_matrix *m, int64_t col, int32_t *rows_dev, uint16_t *vals_dev, int64_t cap,
+                        int32_t *count_dev, celty_stream_t stream);
+
+/*
+ * celty_fetched_bytes -- algorithmic HBM bytes of one celty_spmspv call for a given surviving
+ * column list (host array of n ascending indices): entry stream of those columns as laid out
+ * (including alignment padding and per-block headers), their metadata words, x, the list written
+ * and read back, and y written (cleared + reduced).  Host-only arithmetic on the handle's tables.
+ */
+int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx_host, int64_t n, int64_t *stream_bytes,
+                        int64_t *total_bytes);
+
+/*
+ * celty_last_status -- synchronises `stream`, reads the workspace status word and clears it.
+ * Returns CELTY_OK, CELTY_ETIMEOUT or CELTY_EBOUNDS (or CELTY_ECUDA / CELTY_ESTATE).
+ */
+int celty_last_status(celty_matrix *m, celty_stream_t stream);
+
+/* Tuning knob for experiments: thread blocks per launch (0 = default, one per SM times the
+ * kernel's residency) and the kernel variant (0 = default for the layout). */
+int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant);
+
+/* The cudaError_t of the last failing CUDA call made through this library (0 if none). */
+int celty_last_cuda_error(void);
+
+/* Static string for a celty_status. */
+const char *celty_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CELTY_H */

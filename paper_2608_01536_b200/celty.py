@@ -1,0 +1,237 @@
+"""Thin ctypes binding over the C-ABI library declared in include/celty.h.
+
+Argument marshalling only: every step of the path (packing, thresholding/compaction, run-length
+decode, accumulation, reduction) runs inside the library.  PyTorch provides device memory and
+streams.  There is no fallback: if the library is missing or a call fails, this raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from types import SimpleNamespace
+
+import numpy as np
+
+LAYOUT_COLUMN = 0
+LAYOUT_LANE_TILE = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcelty.so")
+_lib = None
+
+_vp, _i64, _i32, _f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float
+_sz = ctypes.c_size_t
+
+# name -> (restype, argtypes); mirrors include/celty.h one to one
+SIGNATURES = {
+    "celty_encode": (ctypes.c_int, [_vp, _i64, _vp, _i64, _i64, _vp, ctypes.POINTER(_vp)]),
+    "celty_destroy": (None, [_vp]),
+    "celty_info": (ctypes.c_int, [_vp] + [ctypes.POINTER(_i64)] * 5 + [ctypes.POINTER(_i32)] * 2),
+    "celty_decode_host": (ctypes.c_int, [_vp, _i64, _vp, _vp, _vp, _vp, _i64, ctypes.POINTER(_i64)]),
+    "celty_host_image": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
+    "celty_device_bytes": (ctypes.c_int, [_vp, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
+    "celty_bind_device": (ctypes.c_int, [_vp, _vp, _sz, _vp, _sz, _vp]),
+    "celty_compact": (ctypes.c_int, [_vp, _i64, _f32, _vp, _vp, _vp, _vp]),
+    "celty_spmspv": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp]),
+    "celty_spmspv_host": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp, _vp]),
+    "celty_last_compaction": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
+    "celty_decode_device": (ctypes.c_int, [_vp, _i64, _vp, _vp, _i64, _vp, _vp]),
+    "celty_fetched_bytes": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "celty_last_status": (ctypes.c_int, [_vp, _vp]),
+    "celty_set_launch": (ctypes.c_int, [_vp, _i32, _i32]),
+    "celty_last_cuda_error": (ctypes.c_int, []),
+    "celty_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+}
+
+
+class CeltyError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        lib = load()
+        msg = lib.celty_strerror(status).decode()
+        if status == -3:
+            msg += f" (cudaError {lib.celty_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{status}]")
+        self.status = status
+
+
+def load():
+    """Load libcelty.so (built by paper_2608_01536_b200.build).  Raises if it is not there."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: run `python -m paper_2608_01536_b200.build` (needs nvcc). "
+                "There is no CPU or PyTorch fallback for this path.")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise CeltyError(status, where)
+
+
+def _np_ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _stream_ptr(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class _Opts(ctypes.Structure):
+    _fields_ = [("run_bits", _i32), ("layout", _i32), ("tile_rows", _i32), ("reserved", _i32)]
+
+
+class Matrix:
+    """An RLC-CSC encoded weight matrix (host handle), optionally bound to device memory."""
+
+    def __init__(self, W, mask=None, layout: int = LAYOUT_LANE_TILE, tile_rows: int = 0, device=None):
+        lib = load()
+        W = np.asarray(W)
+        if W.dtype == np.float16:
+            W = W.view(np.uint16)
+        if W.dtype != np.uint16 or W.ndim != 2:
+            raise TypeError("W must be a 2-D float16 array (or its uint16 bit patterns)")
+        W = np.ascontiguousarray(W)
+        M, K = W.shape
+        mptr = None
+        if mask is not None:
+            mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+            if mask.shape != (M, K):
+                raise ValueError("mask shape")
+            mptr = _np_ptr(mask)
+        opts = _Opts(4, layout, tile_rows, 0)
+        h = _vp()
+        _check(lib.celty_encode(_np_ptr(W), K, mptr, M, K, ctypes.byref(opts), ctypes.byref(h)), "celty_encode")
+        self._h = h
+        self.M, self.K = M, K
+        self._image = self._ws = None
+        if device is not None:
+            self.to(device)
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h and _lib is not None:
+            _lib.celty_destroy(h)
+
+    # ---------------------------------------------------------------- host side
+    def info(self):
+        v = [_i64() for _ in range(5)]
+        w = [_i32() for _ in range(2)]
+        _check(load().celty_info(self._h, *[ctypes.byref(a) for a in v + w]), "celty_info")
+        return SimpleNamespace(M=v[0].value, K=v[1].value, nnz=v[2].value, n_pad=v[3].value,
+                               compressed_bytes=v[4].value, layout=w[0].value, tile_rows=w[1].value)
+
+    def host_image(self):
+        """(uint8 copy of the packed image, offset of the entry stream in it)."""
+        p, n, o = _vp(), _sz(), _sz()
+        _check(load().celty_host_image(self._h, ctypes.byref(p), ctypes.byref(n), ctypes.byref(o)), "celty_host_image")
+        buf = (ctypes.c_uint8 * n.value).from_address(p.value)
+        return np.frombuffer(buf, dtype=np.uint8).copy(), o.value
+
+    def device_bytes(self):
+        a, b = _sz(), _sz()
+        _check(load().celty_device_bytes(self._h, ctypes.byref(a), ctypes.byref(b)), "celty_device_bytes")
+        return a.value, b.value
+
+    def decode_host(self, col: int):
+        lib = load()
+        n = _i64()
+        rc = lib.celty_decode_host(self._h, col, None, None, None, None, 0, ctypes.byref(n))
+        if rc not in (0, -2):
+            _check(rc, "celty_decode_host")
+        rows = np.zeros(n.value, np.int32)
+        vals = np.zeros(n.value, np.uint16)
+        runs = np.zeros(n.value, np.uint8)
+        pad = np.zeros(n.value, np.uint8)
+        _check(lib.celty_decode_host(self._h, col, _np_ptr(rows), _np_ptr(vals), _np_ptr(runs), _np_ptr(pad),
+                                     n.value, ctypes.byref(n)), "celty_decode_host")
+        return rows, vals, runs, pad
+
+    def fetched_bytes(self, idx):
+        idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
+        s, t = _i64(), _i64()
+        _check(load().celty_fetched_bytes(self._h, _np_ptr(idx), idx.size, ctypes.byref(s), ctypes.byref(t)),
+               "celty_fetched_bytes")
+        return s.value, t.value
+
+    def set_launch(self, grid: int = 0, variant: int = 0):
+        _check(load().celty_set_launch(self._h, grid, variant), "celty_set_launch")
+
+    # ---------------------------------------------------------------- device side
+    def to(self, device="cuda", stream=None):
+        import torch
+        ib, wb = self.device_bytes()
+        dev = torch.device(device)
+        with torch.cuda.device(dev):
+            self._image = torch.empty(ib, dtype=torch.uint8, device=dev)
+            self._ws = torch.empty(wb, dtype=torch.uint8, device=dev)
+            _check(load().celty_bind_device(self._h, self._image.data_ptr(), ib, self._ws.data_ptr(), wb,
+                                            _stream_ptr(stream)), "celty_bind_device")
+        self.device = dev
+        return self
+
+    def spmspv(self, x, tau: float, y=None, stream=None):
+        """y = W . threshold(x, tau); x: K float16 CUDA tensor, y: M float32 CUDA tensor (overwritten)."""
+        import torch
+        if y is None:
+            y = torch.empty(self.M, dtype=torch.float32, device=x.device)
+        assert x.dtype == torch.float16 and x.numel() == self.K and x.is_contiguous()
+        assert y.dtype == torch.float32 and y.numel() == self.M and y.is_contiguous()
+        _check(load().celty_spmspv(self._h, x.data_ptr(), tau, y.data_ptr(), _stream_ptr(stream)), "celty_spmspv")
+        return y
+
+    def spmspv_host(self, x_host, tau: float, y_host, x_stage, y_stage, stream=None):
+        """Same product for host tensors (pinned for speed); copies run inside the library call."""
+        _check(load().celty_spmspv_host(self._h, x_host.data_ptr(), tau, y_host.data_ptr(), x_stage.data_ptr(),
+                                        y_stage.data_ptr(), _stream_ptr(stream)), "celty_spmspv_host")
+        return y_host
+
+    def last_compaction(self):
+        """(idx int32 tensor, val int16-bit-pattern tensor) of the last spmspv call; synchronises."""
+        import torch
+        c, i, v = _vp(), _vp(), _vp()
+        _check(load().celty_last_compaction(self._h, ctypes.byref(c), ctypes.byref(i), ctypes.byref(v)),
+               "celty_last_compaction")
+        torch.cuda.synchronize()
+        ws0 = self._ws.data_ptr()
+        n = int(self._ws[c.value - ws0:c.value - ws0 + 4].view(torch.int32).item())
+        idx = self._ws[i.value - ws0:i.value - ws0 + 4 * n].view(torch.int32).clone()
+        val = self._ws[v.value - ws0:v.value - ws0 + 2 * n].view(torch.int16).clone()
+        return idx, val
+
+    def decode_device(self, col: int, stream=None):
+        import torch
+        n = self.decode_host(col)[0].size
+        rows = torch.full((max(n, 1),), -1, dtype=torch.int32, device=self.device)
+        vals = torch.zeros(max(n, 1), dtype=torch.int16, device=self.device)
+        cnt = torch.zeros(1, dtype=torch.int32, device=self.device)
+        _check(load().celty_decode_device(self._h, col, rows.data_ptr(), vals.data_ptr(), n, cnt.data_ptr(),
+                                          _stream_ptr(stream)), "celty_decode_device")
+        torch.cuda.synchronize()
+        k = int(cnt.item())
+        return rows[:k].cpu().numpy(), vals[:k].cpu().numpy().view(np.uint16)
+
+    def last_status(self, stream=None) -> int:
+        return load().celty_last_status(self._h, _stream_ptr(stream))
+
+
+def compact(x, tau: float, stream=None):
+    """Activation compaction alone: returns (idx int32[n], val uint16-pattern int16[n]) CUDA tensors."""
+    import torch
+    assert x.dtype == torch.float16 and x.is_contiguous()
+    K = x.numel()
+    idx = torch.empty(K, dtype=torch.int32, device=x.device)
+    val = torch.empty(K, dtype=torch.int16, device=x.device)
+    cnt = torch.zeros(1, dtype=torch.int32, device=x.device)
+    _check(load().celty_compact(x.data_ptr(), K, tau, idx.data_ptr(), val.data_ptr(), cnt.data_ptr(),
+                                _stream_ptr(stream)), "celty_compact")
+    n = int(cnt.item())
+    return idx[:n], val[:n]

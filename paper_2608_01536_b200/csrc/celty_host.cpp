@@ -1,0 +1,359 @@
+// Host half of the library: offline packing into RLC-CSC (Section 3.2, Fig. 2(a)), the handle,
+// host-side decoding for round-trip tests and byte accounting.  No CUDA calls in this file.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "celty_internal.h"
+
+using namespace celty;
+
+namespace {
+
+inline bool kept(const uint16_t *W, int64_t ldw, const uint8_t *mask, int64_t K, int64_t r, int64_t j)
+{
+    return mask ? mask[r * K + j] != 0 : (W[r * ldw + j] & 0x7FFFu) != 0;
+}
+
+// Pack the 4-bit runs of 8 consecutive entries, entry e in bits 4e .. 4e+3.
+inline uint32_t pack_runs(const uint8_t *r, int n)
+{
+    uint32_t w = 0;
+    for (int e = 0; e < n; ++e) w |= (uint32_t)(r[e] & 15u) << (4 * e);
+    return w;
+}
+
+struct Logical {                 // one run per byte, block-major (column, tile), rows ascending
+    std::vector<uint16_t> vals;
+    std::vector<uint8_t> runs;
+};
+
+int choose_tile_rows(int64_t M)
+{
+    // about 128 rows per lane keeps a lane's run stream at ~8 groups per column at 50% density;
+    // slabs of 32 lanes then cover M with at most one partly filled slab.
+    int64_t S = std::max<int64_t>(1, (M + 2048) / 4096);
+    int64_t R = (M + 32 * S - 1) / (32 * S);
+    R = (R + 3) / 4 * 4;                       // keeps 16-byte vector stores of y aligned
+    return (int)std::max<int64_t>(4, R);
+}
+
+// Build the COLUMN image: meta uint2[K] {off16, entries}, then per column its chunks of up to 32
+// groups; chunk = [groups x 16 B values][groups x 4 B runs]; column block padded to 16 bytes.
+void pack_column(celty_matrix *m, const Logical &lg)
+{
+    const int64_t K = m->K;
+    m->meta_bytes = round_up((size_t)K * 8, kAlign);
+    std::vector<uint64_t> off(K + 1, 0);
+    for (int64_t j = 0; j < K; ++j) {
+        uint64_t n = m->block_ptr[j + 1] - m->block_ptr[j];
+        uint64_t groups = (n + kGroup - 1) / kGroup;
+        off[j + 1] = off[j] + round_up((size_t)groups * 20, 16);
+        m->max_unit16 = std::max<uint32_t>(m->max_unit16, (uint32_t)((off[j + 1] - off[j]) / 16));
+    }
+    m->stream_bytes = round_up((size_t)off[K], kAlign);
+    m->image.assign(m->meta_bytes + m->stream_bytes, 0);
+    uint32_t *meta = reinterpret_cast<uint32_t *>(m->image.data());
+    uint8_t *stream = m->image.data() + m->meta_bytes;
+    for (int64_t j = 0; j < K; ++j) {
+        const uint64_t e0 = m->block_ptr[j], n = m->block_ptr[j + 1] - e0;
+        meta[2 * j] = (uint32_t)(off[j] / 16);
+        meta[2 * j + 1] = (uint32_t)n;
+        const uint64_t groups = (n + kGroup - 1) / kGroup;
+        uint8_t *col = stream + off[j];
+        for (uint64_t g = 0; g < groups; ++g) {
+            const uint64_t c = g / kChunkGroups, gl = g % kChunkGroups;
+            const uint64_t gc = std::min<uint64_t>(kChunkGroups, groups - c * kChunkGroups);
+            uint8_t *chunk = col + c * (kChunkGroups * 20);
+            const int cnt = (int)std::min<uint64_t>(kGroup, n - g * kGroup);
+            std::memcpy(chunk + 16 * gl, &lg.vals[e0 + g * kGroup], (size_t)cnt * 2);
+            uint32_t w = pack_runs(&lg.runs[e0 + g * kGroup], cnt);
+            std::memcpy(chunk + 16 * gc + 4 * gl, &w, 4);
+        }
+    }
+}
+
+// Build the LANE_TILE image: meta uint32[K*S + 1] (offset/16 of each sub-block), then per
+// (column j, slab s) a sub-block
+//   [32 x u8: groups of lane L's tile 32s+L][G x 16 B values][G x 4 B runs], padded to 16 bytes,
+// G = sum of the lanes' group counts.  Vectors are stored step-major: for step q = 0, 1, ... the
+// lanes that still have a q-th group, in lane order, so that a warp reads one contiguous span per step.
+void pack_lane_tile(celty_matrix *m, const Logical &lg)
+{
+    const int64_t K = m->K, S = m->S, T = m->T;
+    m->meta_bytes = round_up((size_t)(K * S + 1) * 4, kAlign);
+    std::vector<uint64_t> off((size_t)(K * S + 1), 0);
+    for (int64_t j = 0; j < K; ++j)
+        for (int64_t s = 0; s < S; ++s) {
+            uint64_t G = 0;
+            for (int L = 0; L < 32; ++L) {
+                int64_t t = 32 * s + L;
+                if (t >= T) break;
+                uint64_t n = m->block_ptr[j * T + t + 1] - m->block_ptr[j * T + t];
+                G += (n + kGroup - 1) / kGroup;
+            }
+            size_t b = j * S + s;
+            off[b + 1] = off[b] + round_up(32 + (size_t)G * 20, 16);
+            m->max_unit16 = std::max<uint32_t>(m->max_unit16, (uint32_t)((off[b + 1] - off[b]) / 16));
+        }
+    m->stream_bytes = round_up((size_t)off[K * S], kAlign);
+    m->image.assign(m->meta_bytes + m->stream_bytes, 0);
+    uint32_t *meta = reinterpret_cast<uint32_t *>(m->image.data());
+    uint8_t *stream = m->image.data() + m->meta_bytes;
+    for (size_t b = 0; b <= (size_t)(K * S); ++b) meta[b] = (uint32_t)(off[b] / 16);
+    for (int64_t j = 0; j < K; ++j)
+        for (int64_t s = 0; s < S; ++s) {
+            uint8_t *sub = stream + off[j * S + s];
+            uint64_t e0[32], n[32], g[32], G = 0, steps = 0;
+            for (int L = 0; L < 32; ++L) {
+                int64_t t = 32 * s + L;
+                if (t < T) {
+                    e0[L] = m->block_ptr[j * T + t];
+                    n[L] = m->block_ptr[j * T + t + 1] - e0[L];
+                } else {
+                    e0[L] = 0; n[L] = 0;
+                }
+                g[L] = (n[L] + kGroup - 1) / kGroup;
+                sub[L] = (uint8_t)g[L];
+                G += g[L];
+                steps = std::max(steps, g[L]);
+            }
+            uint8_t *vbase = sub + 32, *rbase = vbase + 16 * G;
+            uint64_t slot = 0;
+            for (uint64_t q = 0; q < steps; ++q)
+                for (int L = 0; L < 32; ++L) {
+                    if (g[L] <= q) continue;
+                    const int cnt = (int)std::min<uint64_t>(kGroup, n[L] - q * kGroup);
+                    std::memcpy(vbase + 16 * slot, &lg.vals[e0[L] + q * kGroup], (size_t)cnt * 2);
+                    uint32_t w = pack_runs(&lg.runs[e0[L] + q * kGroup], cnt);
+                    std::memcpy(rbase + 4 * slot, &w, 4);
+                    ++slot;
+                }
+        }
+}
+
+}  // namespace
+
+extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask, int64_t M, int64_t K,
+                            const celty_encode_opts *opts, celty_matrix **out)
+{
+    if (!W || !out || M <= 0 || K <= 0 || ldw < K || M > kMaxM || K >= ((int64_t)1 << 31)) return CELTY_EINVAL;
+    celty_encode_opts o = {4, CELTY_LAYOUT_LANE_TILE, 0, 0};
+    if (opts) o = *opts;
+    if (o.run_bits != 4 || o.reserved != 0) return CELTY_EINVAL;
+    if (o.layout != CELTY_LAYOUT_COLUMN && o.layout != CELTY_LAYOUT_LANE_TILE) return CELTY_EINVAL;
+    if (o.layout == CELTY_LAYOUT_COLUMN && o.tile_rows != 0) return CELTY_EINVAL;
+    if (o.layout == CELTY_LAYOUT_LANE_TILE && (o.tile_rows < 0 || o.tile_rows > 2040)) return CELTY_EINVAL;
+    *out = nullptr;
+    try {
+        celty_matrix *m = new celty_matrix();
+        m->M = M; m->K = K; m->layout = o.layout;
+        if (o.layout == CELTY_LAYOUT_COLUMN) {
+            m->R = (int32_t)M; m->T = 1; m->S = 1;
+        } else {
+            m->R = o.tile_rows > 0 ? o.tile_rows : choose_tile_rows(M);
+            m->T = (M + m->R - 1) / m->R;
+            m->S = (m->T + 31) / 32;
+            if (m->S > 32) { delete m; return CELTY_EINVAL; }   // one warp per slab, 32 warps per block
+        }
+        const int64_t R = m->R, T = m->T;
+        // Pass 1: one sweep over the rows of W keeps, per column, the last kept row; the gap before a
+        // kept weight is split into floor(gap/16) pads and a run of gap mod 16 (Section 3.2).
+        std::vector<uint32_t> cnt((size_t)(K * T), 0);
+        std::vector<int32_t> last((size_t)K);
+        uint64_t total = 0;
+        for (int64_t t = 0; t < T; ++t) {
+            const int64_t r0 = t * R, r1 = std::min<int64_t>(M, r0 + R);
+            std::fill(last.begin(), last.end(), (int32_t)r0 - 1);
+            for (int64_t r = r0; r < r1; ++r)
+                for (int64_t j = 0; j < K; ++j) {
+                    if (!kept(W, ldw, mask, K, r, j)) continue;
+                    const uint32_t gap = (uint32_t)(r - last[j] - 1);
+                    cnt[j * T + t] += (gap >> 4) + 1;
+                    total += (gap >> 4) + 1;
+                    m->n_pad += gap >> 4;
+                    m->nnz += 1;
+                    last[j] = (int32_t)r;
+                }
+        }
+        if (total > 0xFFFFFFFFull) { delete m; return CELTY_EINVAL; }
+        m->block_ptr.resize((size_t)(K * T + 1));
+        uint32_t acc = 0;
+        for (int64_t b = 0; b < K * T; ++b) { m->block_ptr[b] = acc; acc += cnt[b]; }
+        m->block_ptr[K * T] = acc;
+        // Pass 2: same sweep, now writing (value, run) pairs at each block's cursor.
+        Logical lg;
+        lg.vals.assign((size_t)total + kGroup, 0);
+        lg.runs.assign((size_t)total + kGroup, 0);
+        m->pad_bits.assign((size_t)(total + 7) / 8, 0);
+        std::vector<uint32_t> cur(m->block_ptr.begin(), m->block_ptr.end() - 1);
+        for (int64_t t = 0; t < T; ++t) {
+            const int64_t r0 = t * R, r1 = std::min<int64_t>(M, r0 + R);
+            std::fill(last.begin(), last.end(), (int32_t)r0 - 1);
+            for (int64_t r = r0; r < r1; ++r)
+                for (int64_t j = 0; j < K; ++j) {
+                    if (!kept(W, ldw, mask, K, r, j)) continue;
+                    uint32_t gap = (uint32_t)(r - last[j] - 1);
+                    uint32_t &c = cur[j * T + t];
+                    for (; gap > 15; gap -= 16) {
+                        lg.vals[c] = 0; lg.runs[c] = 15;
+                        m->pad_bits[c >> 3] |= (uint8_t)(1u << (c & 7));
+                        ++c;
+                    }
+                    lg.vals[c] = W[r * ldw + j]; lg.runs[c] = (uint8_t)gap; ++c;
+                    last[j] = (int32_t)r;
+                }
+        }
+        if (m->layout == CELTY_LAYOUT_COLUMN) pack_column(m, lg); else pack_lane_tile(m, lg);
+        m->ws = workspace_layout(K, T);
+        *out = m;
+        return CELTY_OK;
+    } catch (const std::bad_alloc &) {
+        return CELTY_ENOMEM;
+    }
+}
+
+extern "C" void celty_destroy(celty_matrix *m) { delete m; }
+
+extern "C" int celty_info(const celty_matrix *m, int64_t *M, int64_t *K, int64_t *nnz, int64_t *n_pad,
+                          int64_t *compressed_bytes, int32_t *layout, int32_t *tile_rows)
+{
+    if (!m) return CELTY_EINVAL;
+    if (M) *M = m->M;
+    if (K) *K = m->K;
+    if (nnz) *nnz = m->nnz;
+    if (n_pad) *n_pad = m->n_pad;
+    if (compressed_bytes) *compressed_bytes = (m->nnz + m->n_pad) * 5 / 2 + 4 * (m->K + 1);
+    if (layout) *layout = m->layout;
+    if (tile_rows) *tile_rows = m->layout == CELTY_LAYOUT_COLUMN ? 0 : m->R;
+    return CELTY_OK;
+}
+
+// Decode column `col` from the packed image (not from the encoder's temporaries).
+extern "C" int celty_decode_host(const celty_matrix *m, int64_t col, int32_t *rows, uint16_t *vals,
+                                 uint8_t *runs, uint8_t *is_pad, int64_t cap, int64_t *n_out)
+{
+    if (!m || col < 0 || col >= m->K) return CELTY_EINVAL;
+    const int64_t T = m->T;
+    const int64_t n = (int64_t)m->block_ptr[(col + 1) * T] - (int64_t)m->block_ptr[col * T];
+    if (n_out) *n_out = n;
+    if (n > cap) return CELTY_ENOMEM;
+    const uint8_t *stream = m->image.data() + m->meta_bytes;
+    const uint32_t *meta = reinterpret_cast<const uint32_t *>(m->image.data());
+    int64_t o = 0;
+    // A pad cannot be told from a kept +0 that follows 15 dropped rows by looking at the image, so
+    // the flag comes from the bit the encoder recorded for the entry's logical position.
+    auto emit = [&](uint64_t logical, int64_t row, uint16_t v, uint8_t run) {
+        if (rows) rows[o] = (int32_t)row;
+        if (vals) vals[o] = v;
+        if (runs) runs[o] = run;
+        if (is_pad) is_pad[o] = (m->pad_bits[logical >> 3] >> (logical & 7)) & 1u;
+        ++o;
+    };
+    if (m->layout == CELTY_LAYOUT_COLUMN) {
+        const uint8_t *colp = stream + (size_t)meta[2 * col] * 16;
+        const int64_t groups = (n + kGroup - 1) / kGroup;
+        int64_t s = 0;
+        for (int64_t e = 0; e < n; ++e) {
+            const int64_t g = e / kGroup, c = g / kChunkGroups, gl = g % kChunkGroups;
+            const int64_t gc = std::min<int64_t>(kChunkGroups, groups - c * kChunkGroups);
+            const uint8_t *chunk = colp + c * (kChunkGroups * 20);
+            uint16_t v; uint32_t w;
+            std::memcpy(&v, chunk + 16 * gl + 2 * (e % kGroup), 2);
+            std::memcpy(&w, chunk + 16 * gc + 4 * gl, 4);
+            const uint8_t run = (w >> (4 * (e % kGroup))) & 15u;
+            s += run;
+            emit((uint64_t)m->block_ptr[col] + e, s + e, v, run);
+        }
+    } else {
+        for (int64_t sl = 0; sl < m->S; ++sl) {
+            const uint8_t *sub = stream + (size_t)meta[col * m->S + sl] * 16;
+            int64_t G = 0;
+            for (int L = 0; L < 32; ++L) G += sub[L];
+            const uint8_t *vbase = sub + 32, *rbase = vbase + 16 * G;
+            for (int L = 0; L < 32; ++L) {
+                const int64_t t = 32 * sl + L;
+                if (t >= T) break;
+                const int64_t nt = (int64_t)m->block_ptr[col * T + t + 1] - (int64_t)m->block_ptr[col * T + t];
+                int64_t s = 0;
+                for (int64_t e = 0; e < nt; ++e) {
+                    const int64_t q = e / kGroup;
+                    // slot of (step q, lane L): all lanes' groups of earlier steps + lower lanes of this step
+                    int64_t slot = 0;
+                    for (int L2 = 0; L2 < 32; ++L2) slot += std::min<int64_t>(sub[L2], q) + (L2 < L && sub[L2] > q ? 1 : 0);
+                    uint16_t v; uint32_t w;
+                    std::memcpy(&v, vbase + 16 * slot + 2 * (e % kGroup), 2);
+                    std::memcpy(&w, rbase + 4 * slot, 4);
+                    const uint8_t run = (w >> (4 * (e % kGroup))) & 15u;
+                    s += run;
+                    emit((uint64_t)m->block_ptr[col * T + t] + e, t * m->R + s + e, v, run);
+                }
+            }
+        }
+    }
+    return CELTY_OK;
+}
+
+extern "C" int celty_host_image(const celty_matrix *m, const void **image, size_t *image_bytes, size_t *stream_offset)
+{
+    if (!m) return CELTY_EINVAL;
+    if (image) *image = m->image.data();
+    if (image_bytes) *image_bytes = m->image.size();
+    if (stream_offset) *stream_offset = m->meta_bytes;
+    return CELTY_OK;
+}
+
+extern "C" int celty_device_bytes(const celty_matrix *m, size_t *image_bytes, size_t *workspace_bytes)
+{
+    if (!m) return CELTY_EINVAL;
+    if (image_bytes) *image_bytes = m->image.size();
+    if (workspace_bytes) *workspace_bytes = m->ws.total;
+    return CELTY_OK;
+}
+
+extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, int64_t n, int64_t *stream_bytes,
+                                   int64_t *total_bytes)
+{
+    if (!m || (!idx && n > 0) || n < 0) return CELTY_EINVAL;
+    const uint32_t *meta = reinterpret_cast<const uint32_t *>(m->image.data());
+    int64_t sb = 0, mb = 0;
+    for (int64_t p = 0; p < n; ++p) {
+        const int64_t j = idx[p];
+        if (j < 0 || j >= m->K) return CELTY_EINVAL;
+        if (m->layout == CELTY_LAYOUT_COLUMN) {
+            const int64_t groups = ((int64_t)meta[2 * j + 1] + kGroup - 1) / kGroup;
+            sb += (int64_t)round_up((size_t)groups * 20, 16);
+            mb += 8;
+        } else {
+            sb += ((int64_t)meta[(j + 1) * m->S] - (int64_t)meta[j * m->S]) * 16;
+            mb += 4 * (m->S + 1);
+        }
+    }
+    if (stream_bytes) *stream_bytes = sb;
+    // x read, list written then read (4-byte index + 2-byte value each way), y cleared and reduced
+    if (total_bytes) *total_bytes = sb + mb + 2 * m->K + 12 * n + 8 * m->M;
+    return CELTY_OK;
+}
+
+extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant)
+{
+    if (!m || grid < 0 || variant < 0) return CELTY_EINVAL;
+    m->grid = grid;
+    m->variant = variant;
+    return CELTY_OK;
+}
+
+extern "C" const char *celty_strerror(int status)
+{
+    switch (status) {
+        case CELTY_OK: return "ok";
+        case CELTY_EINVAL: return "invalid argument";
+        case CELTY_ENOMEM: return "out of memory or buffer too small";
+        case CELTY_ECUDA: return "CUDA runtime error";
+        case CELTY_ESTATE: return "handle is not bound to device memory";
+        case CELTY_ETIMEOUT: return "a bounded wait inside a kernel ran out";
+        case CELTY_EBOUNDS: return "a decoded index was out of range";
+        default: return "unknown status";
+    }
+}

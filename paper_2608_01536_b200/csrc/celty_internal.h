@@ -1,0 +1,65 @@
+// Internal definitions shared by the host encoder and the CUDA translation unit.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "celty.h"
+
+namespace celty {
+
+constexpr int kGroup = 8;            // entries per 16-byte value vector / 32-bit run word
+constexpr int kChunkGroups = 32;     // COLUMN layout: groups per warp-wide chunk (256 entries)
+constexpr int kTileSlack = 8;        // LANE_TILE: spare accumulator rows per slab for group-tail slots
+constexpr int64_t kMaxM = 49152;     // accumulators of one thread block must fit shared memory
+constexpr size_t kAlign = 256;
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Workspace layout (device): all offsets multiples of 256.
+struct WorkspaceLayout {
+    size_t status_off;   // uint32 status, int32 count (and spare words)
+    size_t idx_off;      // int32[K]
+    size_t val_off;      // uint16[K]
+    size_t scratch_off;  // uint32[T + 2] for celty_decode_device
+    size_t total;
+};
+
+inline WorkspaceLayout workspace_layout(int64_t K, int64_t T)
+{
+    WorkspaceLayout w{};
+    w.status_off = 0;
+    w.idx_off = kAlign;
+    w.val_off = w.idx_off + round_up((size_t)K * 4, kAlign);
+    w.scratch_off = w.val_off + round_up((size_t)K * 2, kAlign);
+    w.total = w.scratch_off + round_up((size_t)(T + 2) * 4, kAlign);
+    return w;
+}
+
+}  // namespace celty
+
+// The handle.  Host side: logical block pointers and the packed image exactly as it is copied to
+// the device.  Device side: caller-owned buffers recorded by celty_bind_device.
+struct celty_matrix {
+    int64_t M = 0, K = 0;
+    int32_t layout = 0;
+    int32_t R = 0;          // rows per tile (LANE_TILE) or M (COLUMN)
+    int64_t T = 1;          // tiles per column
+    int64_t S = 1;          // slabs of 32 tiles per column (LANE_TILE), 1 for COLUMN
+    int64_t nnz = 0, n_pad = 0;
+    std::vector<uint32_t> block_ptr;   // K*T + 1, stored entries before block (j, t)
+    std::vector<uint8_t> pad_bits;     // one bit per stored entry (logical order): 1 = padding entry
+    // image = [meta | stream]
+    //   COLUMN:    meta = uint2[K]  {offset/16 of the column block in the stream, entries}
+    //   LANE_TILE: meta = uint32[K*S + 1]  offset/16 of sub-block (j, s); sub-blocks are contiguous
+    std::vector<uint8_t> image;
+    size_t meta_bytes = 0;             // stream starts at image[meta_bytes]
+    size_t stream_bytes = 0;
+    uint32_t max_unit16 = 0;           // largest column block / sub-block in 16-byte units
+
+    // device binding
+    uint8_t *d_image = nullptr;
+    uint8_t *d_ws = nullptr;
+    celty::WorkspaceLayout ws{};
+    int32_t grid = 0, variant = 0;
+};

@@ -1,0 +1,518 @@
+// CUDA half of the library (sm_100a): activation compaction, the two SpMSpV kernels, the decode
+// kernels used by parity tests, and the C-ABI entry points that launch them.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <mutex>
+
+#include "celty_internal.h"
+
+using namespace celty;
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+
+#define CELTY_CUDA(expr)                                   \
+    do {                                                   \
+        cudaError_t err_ = (expr);                         \
+        if (err_ != cudaSuccess) {                         \
+            g_last_cuda = (int)err_;                       \
+            return CELTY_ECUDA;                            \
+        }                                                  \
+    } while (0)
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+enum : uint32_t { kStatusTimeout = 1u, kStatusBounds = 2u };
+
+struct DeviceInfo { int sms = 0; int max_smem_optin = 0; };
+
+int device_info(DeviceInfo *out)
+{
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    CELTY_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CELTY_EINVAL;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache[dev].sms == 0) {
+        CELTY_CUDA(cudaDeviceGetAttribute(&cache[dev].sms, cudaDevAttrMultiProcessorCount, dev));
+        CELTY_CUDA(cudaDeviceGetAttribute(&cache[dev].max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    }
+    *out = cache[dev];
+    return CELTY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Run-length decode of one group of 8 entries (Algorithm 1, the per-lane part, done on packed bytes).
+// w holds the eight 4-bit runs, entry e in bits 4e..4e+3.  On return byte m of `even` is the
+// inclusive sum of runs 0..2m plus the ordinal 2m, byte m of `odd` the same for entry 2m+1, and
+// `total` the sum of the 8 runs.  The row of entry e is base + that byte; the largest is 15*8+7 = 127.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void decode_group(uint32_t w, uint32_t &even, uint32_t &odd, uint32_t &total)
+{
+    const uint32_t lo = w & 0x0F0F0F0Fu;          // runs of entries 0,2,4,6
+    const uint32_t hi = (w >> 4) & 0x0F0F0F0Fu;   // runs of entries 1,3,5,7
+    const uint32_t p = (lo + hi) * 0x01010101u;   // byte m = runs 0..2m+1 summed
+    total = p >> 24;
+    odd = p + 0x07050301u;
+    even = p - hi + 0x06040200u;
+}
+
+__device__ __forceinline__ uint32_t entry_offset(uint32_t even, uint32_t odd, int e)
+{
+    const uint32_t src = (e & 1) ? odd : even;
+    return (src >> (8 * (e >> 1))) & 0xFFu;
+}
+
+__device__ __forceinline__ float entry_value(const uint4 &v, int e)
+{
+    const uint32_t word = e < 2 ? v.x : e < 4 ? v.y : e < 6 ? v.z : v.w;
+    const __half2 h2 = *reinterpret_cast<const __half2 *>(&word);
+    return (e & 1) ? __high2float(h2) : __low2float(h2);
+}
+
+__device__ __forceinline__ uint16_t entry_bits(const uint4 &v, int e)
+{
+    const uint32_t word = e < 2 ? v.x : e < 4 ? v.y : e < 6 ? v.z : v.w;
+    return (uint16_t)((e & 1) ? (word >> 16) : (word & 0xFFFFu));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Activation compaction (magnitude thresholding, Sections 1 and 2.1): one thread block walks x in
+// tiles of 8 values per thread, keeps j iff not(|x_j| <= tau) in FP32, and writes the surviving
+// indices and FP16 bit patterns in ascending order.  The same launch clears y when y != nullptr.
+// ------------------------------------------------------------------------------------------------
+constexpr int kCompactThreads = 1024;
+
+__global__ void __launch_bounds__(kCompactThreads)
+k_compact(const uint16_t *__restrict__ x, int K, float tau, int32_t *__restrict__ idx,
+          uint16_t *__restrict__ val, int32_t *__restrict__ count, float *__restrict__ y, int M)
+{
+    __shared__ int warp_tot[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (y) {
+        for (int i = tid * 4; i < M; i += kCompactThreads * 4) {
+            if (i + 3 < M) {
+                *reinterpret_cast<float4 *>(y + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                for (int k = i; k < M; ++k) y[k] = 0.f;
+            }
+        }
+    }
+    int base = 0;
+    for (int tile = 0; tile < K; tile += kCompactThreads * 8) {
+        const int e0 = tile + tid * 8;
+        uint16_t h[8];
+        if (e0 + 8 <= K) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(x + e0);
+            h[0] = v.x & 0xFFFF; h[1] = v.x >> 16; h[2] = v.y & 0xFFFF; h[3] = v.y >> 16;
+            h[4] = v.z & 0xFFFF; h[5] = v.z >> 16; h[6] = v.w & 0xFFFF; h[7] = v.w >> 16;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) h[k] = (e0 + k < K) ? x[e0 + k] : (uint16_t)0;
+        }
+        unsigned keep = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float f = __half2float(__ushort_as_half(h[k]));
+            if (e0 + k < K && !(fabsf(f) <= tau)) keep |= 1u << k;
+        }
+        const int cnt = __popc(keep);
+        int incl = cnt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(kFull, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            const int t = warp_tot[lane];
+            int s = t;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(kFull, s, d);
+                if (lane >= d) s += up;
+            }
+            warp_tot[lane] = s;                     // inclusive totals over warps
+        }
+        __syncthreads();
+        int o = base + (warp ? warp_tot[warp - 1] : 0) + incl - cnt;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (keep & (1u << k)) {
+                idx[o] = e0 + k;
+                val[o] = h[k];
+                ++o;
+            }
+        base += warp_tot[31];
+        __syncthreads();
+    }
+    if (tid == 0) *count = base;
+}
+
+// ------------------------------------------------------------------------------------------------
+// COLUMN layout kernel: the formulation of Sections 3.1-3.3 as published.  A thread block owns a
+// slice of the surviving-column list and an M-float accumulator in shared memory.  Each warp takes
+// whole columns; per chunk of 256 entries every lane loads 8 values (one 128-bit load) and their 8
+// runs, the warp reconstructs rows with the intra-warp prefix sum of Algorithm 1 (per-lane sum,
+// five shfl_up steps, back-fill), and scatters value * x_j with shared-memory atomic adds.  The
+// accumulator is flushed to y once, with global atomic adds (split-K merge, Section 3.1).
+// ------------------------------------------------------------------------------------------------
+struct ColumnChunk {
+    uint4 v;
+    uint32_t even, odd;
+    uint32_t row0;        // row of this lane's first entry minus its own offset byte
+};
+
+__device__ __forceinline__ ColumnChunk load_column_chunk(const uint8_t *col, uint32_t groups, uint32_t c,
+                                                          int lane, uint32_t &carry)
+{
+    ColumnChunk ch;
+    const uint32_t gc = min((uint32_t)kChunkGroups, groups - c * kChunkGroups);
+    const uint8_t *chunk = col + (size_t)c * (kChunkGroups * 20);
+    uint32_t w = 0;
+    ch.v = make_uint4(0, 0, 0, 0);
+    if ((uint32_t)lane < gc) {
+        ch.v = *reinterpret_cast<const uint4 *>(chunk + 16 * lane);
+        w = *reinterpret_cast<const uint32_t *>(chunk + 16 * gc + 4 * lane);
+    }
+    uint32_t total;
+    decode_group(w, ch.even, ch.odd, total);
+    // Algorithm 1: inclusive scan over lanes of the rows each lane spans (its runs + its 8 entries)
+    const uint32_t span = ((uint32_t)lane < gc) ? total + kGroup : 0u;
+    uint32_t sum = span;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t prev = __shfl_up_sync(kFull, sum, d);
+        if (lane >= d) sum += prev;
+    }
+    ch.row0 = carry + sum - span;
+    carry += __shfl_sync(kFull, sum, 31);
+    return ch;
+}
+
+__global__ void __launch_bounds__(256)
+k_spmspv_column(const uint2 *__restrict__ meta, const uint8_t *__restrict__ stream,
+                const int32_t *__restrict__ idx, const uint16_t *__restrict__ val,
+                const int32_t *__restrict__ count, float *__restrict__ y, int M, uint32_t *status)
+{
+    extern __shared__ float acc[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    for (int i = tid; i < M; i += blockDim.x) acc[i] = 0.f;
+    __syncthreads();
+    const int n = *count;
+    const int p0 = (int)((int64_t)blockIdx.x * n / gridDim.x);
+    const int p1 = (int)((int64_t)(blockIdx.x + 1) * n / gridDim.x);
+    for (int p = p0 + warp; p < p1; p += nwarps) {
+        const int j = idx[p];
+        const float xj = __half2float(__ushort_as_half(val[p]));
+        const uint2 mj = meta[j];
+        const uint8_t *col = stream + (size_t)mj.x * 16;
+        const uint32_t nent = mj.y, groups = (nent + kGroup - 1) / kGroup;
+        uint32_t carry = 0;
+        for (uint32_t c = 0; c * kChunkGroups < groups; ++c) {
+            const ColumnChunk ch = load_column_chunk(col, groups, c, lane, carry);
+            const uint32_t e0 = (c * kChunkGroups + lane) * kGroup;
+#pragma unroll
+            for (int e = 0; e < kGroup; ++e) {
+                if (e0 + e < nent) {
+                    const uint32_t row = ch.row0 + entry_offset(ch.even, ch.odd, e);
+                    if (row < (uint32_t)M) atomicAdd(&acc[row], entry_value(ch.v, e) * xj);
+                    else atomicOr(status, kStatusBounds);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < M; i += blockDim.x) {
+        const float v = acc[i];
+        if (v != 0.f) atomicAdd(&y[i], v);
+    }
+}
+
+__global__ void k_decode_column(const uint2 *__restrict__ meta, const uint8_t *__restrict__ stream, int j,
+                                int32_t *rows, uint16_t *vals, int cap, int32_t *count)
+{
+    const int lane = threadIdx.x;
+    const uint2 mj = meta[j];
+    const uint8_t *col = stream + (size_t)mj.x * 16;
+    const uint32_t nent = mj.y, groups = (nent + kGroup - 1) / kGroup;
+    uint32_t carry = 0;
+    for (uint32_t c = 0; c * kChunkGroups < groups; ++c) {
+        const ColumnChunk ch = load_column_chunk(col, groups, c, lane, carry);
+        const uint32_t e0 = (c * kChunkGroups + lane) * kGroup;
+        for (int e = 0; e < kGroup; ++e)
+            if (e0 + e < nent && e0 + e < (uint32_t)cap) {
+                rows[e0 + e] = (int32_t)(ch.row0 + entry_offset(ch.even, ch.odd, e));
+                vals[e0 + e] = entry_bits(ch.v, e);
+            }
+    }
+    if (lane == 0) *count = (int32_t)min(nent, (uint32_t)cap);
+}
+
+// ------------------------------------------------------------------------------------------------
+// LANE_TILE layout kernel.  Rows are partitioned into tiles of R rows and the rule of Section 3.2
+// restarts in every tile.  Warp s of a warp group owns slab s (tiles 32s .. 32s+31), lane L owns tile
+// 32s+L: each lane walks its own run stream with a running row sum (no cross-lane scan is needed),
+// and local row i of lane L lives at accumulator word (s*(R+8) + i)*32 + L, i.e. in bank L -- every
+// scatter instruction touches 32 distinct banks, and no two threads ever touch the same word, so the
+// accumulation is a plain load / fmaf / store.  The 8 spare rows per slab absorb the zero-valued slots
+// that fill a lane's last 16-byte group.  G warp groups per block work on different columns with an
+// accumulator each; the flush adds them and merges into y with global atomic adds.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+k_spmspv_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ stream,
+              const int32_t *__restrict__ idx, const uint16_t *__restrict__ val,
+              const int32_t *__restrict__ count, float *__restrict__ y, int M, int R, int S, int T, int G)
+{
+    extern __shared__ float acc[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int slab_words = (R + kTileSlack) * 32, group_words = S * slab_words;
+    for (int i = tid; i < G * group_words; i += blockDim.x) acc[i] = 0.f;
+    __syncthreads();
+    const int g = warp / S, s = warp - g * S;
+    const int n = *count;
+    const int64_t units = (int64_t)gridDim.x * G, u = (int64_t)blockIdx.x * G + g;
+    const int p0 = (int)(u * n / units), p1 = (int)((u + 1) * n / units);
+    float *a = acc + g * group_words + s * slab_words + lane;
+    for (int p = p0; p < p1; ++p) {
+        const int j = idx[p];
+        const float xj = __half2float(__ushort_as_half(val[p]));
+        const uint8_t *sub = stream + (size_t)meta[(size_t)j * S + s] * 16;
+        const uint32_t gl = sub[lane];
+        const uint32_t steps = __reduce_max_sync(kFull, gl);
+        const uint32_t Gs = __reduce_add_sync(kFull, gl);
+        const uint8_t *vbase = sub + 32, *rbase = vbase + 16 * (size_t)Gs;
+        uint32_t slot0 = 0, row = 0;
+        for (uint32_t q = 0; q < steps; ++q) {
+            const bool active = gl > q;
+            const uint32_t ballot = __ballot_sync(kFull, active);
+            if (active) {
+                const uint32_t slot = slot0 + __popc(ballot & ((1u << lane) - 1u));
+                const uint4 v = *reinterpret_cast<const uint4 *>(vbase + 16 * (size_t)slot);
+                const uint32_t w = *reinterpret_cast<const uint32_t *>(rbase + 4 * (size_t)slot);
+                uint32_t even, odd, total;
+                decode_group(w, even, odd, total);
+#pragma unroll
+                for (int e = 0; e < kGroup; ++e) {
+                    float *cell = a + (row + entry_offset(even, odd, e)) * 32;
+                    *cell = fmaf(entry_value(v, e), xj, *cell);
+                }
+                row += total + kGroup;
+            }
+            slot0 += __popc(ballot);
+        }
+    }
+    __syncthreads();
+    for (int w = warp; w < S * R; w += nwarps) {
+        const int sl = w / R, i = w - sl * R;
+        const int t = 32 * sl + lane, r = t * R + i;
+        if (t < T && r < M) {
+            float v = 0.f;
+            for (int gg = 0; gg < G; ++gg) v += acc[gg * group_words + sl * slab_words + i * 32 + lane];
+            if (v != 0.f) atomicAdd(&y[r], v);
+        }
+    }
+}
+
+// scratch[0 .. T] = the column's logical block pointers (entries before each tile), relative to scratch[0]
+__global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ stream, int j,
+                              int R, int S, int T, const uint32_t *__restrict__ scratch, int32_t *rows,
+                              uint16_t *vals, int cap, int32_t *count)
+{
+    const int lane = threadIdx.x & 31, s = threadIdx.x >> 5;
+    const uint8_t *sub = stream + (size_t)meta[(size_t)j * S + s] * 16;
+    const uint32_t gl = sub[lane];
+    const uint32_t steps = __reduce_max_sync(kFull, gl);
+    const uint32_t Gs = __reduce_add_sync(kFull, gl);
+    const uint8_t *vbase = sub + 32, *rbase = vbase + 16 * (size_t)Gs;
+    const int t = 32 * s + lane;
+    const uint32_t out0 = t < T ? scratch[t] - scratch[0] : 0u;
+    const uint32_t nt = t < T ? scratch[t + 1] - scratch[t] : 0u;
+    uint32_t slot0 = 0, row = 0;
+    for (uint32_t q = 0; q < steps; ++q) {
+        const bool active = gl > q;
+        const uint32_t ballot = __ballot_sync(kFull, active);
+        if (active) {
+            const uint32_t slot = slot0 + __popc(ballot & ((1u << lane) - 1u));
+            const uint4 v = *reinterpret_cast<const uint4 *>(vbase + 16 * (size_t)slot);
+            const uint32_t w = *reinterpret_cast<const uint32_t *>(rbase + 4 * (size_t)slot);
+            uint32_t even, odd, total;
+            decode_group(w, even, odd, total);
+            for (int e = 0; e < kGroup; ++e) {
+                const uint32_t k = q * kGroup + e;
+                if (k < nt && out0 + k < (uint32_t)cap) {
+                    rows[out0 + k] = (int32_t)(t * R + row + entry_offset(even, odd, e));
+                    vals[out0 + k] = entry_bits(v, e);
+                }
+            }
+            row += total + kGroup;
+        }
+        slot0 += __popc(ballot);
+    }
+    if (threadIdx.x == 0) *count = (int32_t)min(scratch[T] - scratch[0], (uint32_t)cap);
+}
+
+// Raise a kernel's dynamic shared-memory limit once per device (and again only if a larger size is
+// asked for), so that steady-state calls make no attribute calls.
+template <typename Kernel>
+int ensure_smem(Kernel kernel, size_t bytes, int *granted /* [64], per device */)
+{
+    int dev = 0;
+    CELTY_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CELTY_EINVAL;
+    if ((size_t)granted[dev] >= bytes && granted[dev] > 0) return CELTY_OK;
+    CELTY_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    granted[dev] = (int)bytes;
+    return CELTY_OK;
+}
+
+int launch_compact(const void *x, int64_t K, float tau, int32_t *idx, uint16_t *val, int32_t *count, float *y,
+                   int64_t M, cudaStream_t st)
+{
+    k_compact<<<1, kCompactThreads, 0, st>>>(static_cast<const uint16_t *>(x), (int)K, tau, idx, val, count, y, (int)M);
+    CELTY_CUDA(cudaGetLastError());
+    return CELTY_OK;
+}
+
+}  // namespace
+
+extern "C" int celty_last_cuda_error(void) { return g_last_cuda; }
+
+extern "C" int celty_bind_device(celty_matrix *m, void *image_dev, size_t image_bytes, void *workspace_dev,
+                                 size_t workspace_bytes, celty_stream_t stream)
+{
+    if (!m || !image_dev || !workspace_dev) return CELTY_EINVAL;
+    if (image_bytes < m->image.size() || workspace_bytes < m->ws.total) return CELTY_ENOMEM;
+    if (((uintptr_t)image_dev | (uintptr_t)workspace_dev) & (kAlign - 1)) return CELTY_ENOMEM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CELTY_CUDA(cudaMemcpyAsync(image_dev, m->image.data(), m->image.size(), cudaMemcpyHostToDevice, st));
+    CELTY_CUDA(cudaMemsetAsync(workspace_dev, 0, m->ws.total, st));
+    m->d_image = static_cast<uint8_t *>(image_dev);
+    m->d_ws = static_cast<uint8_t *>(workspace_dev);
+    return CELTY_OK;
+}
+
+extern "C" int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *idx_dev, uint16_t *val_dev,
+                             int32_t *count_dev, celty_stream_t stream)
+{
+    if (!x_dev || !idx_dev || !val_dev || !count_dev || K <= 0 || K >= ((int64_t)1 << 31)) return CELTY_EINVAL;
+    if (!(tau >= 0.f) || !std::isfinite(tau)) return CELTY_EINVAL;
+    if ((uintptr_t)x_dev & 15) return CELTY_EINVAL;
+    return launch_compact(x_dev, K, tau, idx_dev, val_dev, count_dev, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, celty_stream_t stream)
+{
+    if (!m || !x_dev || !y_dev) return CELTY_EINVAL;
+    if (!(tau >= 0.f) || !std::isfinite(tau)) return CELTY_EINVAL;
+    if (((uintptr_t)x_dev | (uintptr_t)y_dev) & 15) return CELTY_EINVAL;
+    if (!m->d_image || !m->d_ws) return CELTY_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    uint32_t *status = reinterpret_cast<uint32_t *>(m->d_ws + m->ws.status_off);
+    int32_t *count = reinterpret_cast<int32_t *>(status + 1);
+    int32_t *idx = reinterpret_cast<int32_t *>(m->d_ws + m->ws.idx_off);
+    uint16_t *val = reinterpret_cast<uint16_t *>(m->d_ws + m->ws.val_off);
+    float *y = static_cast<float *>(y_dev);
+    rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);
+    if (rc) return rc;
+    const uint8_t *stream_base = m->d_image + m->meta_bytes;
+    if (m->layout == CELTY_LAYOUT_COLUMN) {
+        const size_t smem = (size_t)m->M * 4;
+        if (smem > (size_t)di.max_smem_optin) return CELTY_EINVAL;
+        static int granted[64];
+        rc = ensure_smem(k_spmspv_column, smem, granted);
+        if (rc) return rc;
+        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (size_t)(di.max_smem_optin) / (smem + 1024)));
+        const int grid = m->grid > 0 ? m->grid : di.sms * per_sm;
+        k_spmspv_column<<<grid, 256, smem, st>>>(reinterpret_cast<const uint2 *>(m->d_image), stream_base, idx, val,
+                                                  count, y, (int)m->M, status);
+    } else {
+        const size_t group_bytes = (size_t)m->S * (m->R + kTileSlack) * 32 * 4;
+        if (group_bytes > (size_t)di.max_smem_optin || m->S > 32) return CELTY_EINVAL;
+        int G = (int)std::min<size_t>((size_t)di.max_smem_optin / group_bytes, (size_t)(32 / m->S));
+        G = std::max(1, std::min(G, m->variant > 0 ? m->variant : (int)std::max<int64_t>(1, 8 / m->S)));
+        const size_t smem = group_bytes * G;
+        static int granted[64];
+        rc = ensure_smem(k_spmspv_lane, smem, granted);
+        if (rc) return rc;
+        const int grid = m->grid > 0 ? m->grid : di.sms;
+        k_spmspv_lane<<<grid, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(m->d_image),
+                                                              stream_base, idx, val, count, y, (int)m->M, m->R,
+                                                              (int)m->S, (int)m->T, G);
+    }
+    CELTY_CUDA(cudaGetLastError());
+    return CELTY_OK;
+}
+
+extern "C" int celty_spmspv_host(celty_matrix *m, const void *x_host, float tau, void *y_host, void *x_stage_dev,
+                                 void *y_stage_dev, celty_stream_t stream)
+{
+    if (!m || !x_host || !y_host || !x_stage_dev || !y_stage_dev) return CELTY_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CELTY_CUDA(cudaMemcpyAsync(x_stage_dev, x_host, (size_t)m->K * 2, cudaMemcpyHostToDevice, st));
+    const int rc = celty_spmspv(m, x_stage_dev, tau, y_stage_dev, stream);
+    if (rc) return rc;
+    CELTY_CUDA(cudaMemcpyAsync(y_host, y_stage_dev, (size_t)m->M * 4, cudaMemcpyDeviceToHost, st));
+    CELTY_CUDA(cudaStreamSynchronize(st));
+    return CELTY_OK;
+}
+
+extern "C" int celty_last_compaction(const celty_matrix *m, const int32_t **count_dev, const int32_t **idx_dev,
+                                     const uint16_t **val_dev)
+{
+    if (!m) return CELTY_EINVAL;
+    if (!m->d_ws) return CELTY_ESTATE;
+    if (count_dev) *count_dev = reinterpret_cast<const int32_t *>(m->d_ws + m->ws.status_off) + 1;
+    if (idx_dev) *idx_dev = reinterpret_cast<const int32_t *>(m->d_ws + m->ws.idx_off);
+    if (val_dev) *val_dev = reinterpret_cast<const uint16_t *>(m->d_ws + m->ws.val_off);
+    return CELTY_OK;
+}
+
+extern "C" int celty_decode_device(celty_matrix *m, int64_t col, int32_t *rows_dev, uint16_t *vals_dev, int64_t cap,
+                                   int32_t *count_dev, celty_stream_t stream)
+{
+    if (!m || !rows_dev || !vals_dev || !count_dev || col < 0 || col >= m->K || cap < 0 || cap > 0x7FFFFFFF)
+        return CELTY_EINVAL;
+    if (!m->d_image || !m->d_ws) return CELTY_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint8_t *stream_base = m->d_image + m->meta_bytes;
+    if (m->layout == CELTY_LAYOUT_COLUMN) {
+        k_decode_column<<<1, 32, 0, st>>>(reinterpret_cast<const uint2 *>(m->d_image), stream_base, (int)col, rows_dev,
+                                          vals_dev, (int)cap, count_dev);
+    } else {
+        uint32_t *scratch = reinterpret_cast<uint32_t *>(m->d_ws + m->ws.scratch_off);
+        CELTY_CUDA(cudaMemcpyAsync(scratch, &m->block_ptr[(size_t)col * m->T], (size_t)(m->T + 1) * 4,
+                                   cudaMemcpyHostToDevice, st));
+        k_decode_lane<<<1, 32 * (int)m->S, 0, st>>>(reinterpret_cast<const uint32_t *>(m->d_image), stream_base,
+                                                    (int)col, m->R, (int)m->S, (int)m->T, scratch, rows_dev, vals_dev,
+                                                    (int)cap, count_dev);
+    }
+    CELTY_CUDA(cudaGetLastError());
+    return CELTY_OK;
+}
+
+extern "C" int celty_last_status(celty_matrix *m, celty_stream_t stream)
+{
+    if (!m) return CELTY_EINVAL;
+    if (!m->d_ws) return CELTY_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    CELTY_CUDA(cudaMemcpyAsync(&word, m->d_ws + m->ws.status_off, 4, cudaMemcpyDeviceToHost, st));
+    CELTY_CUDA(cudaStreamSynchronize(st));
+    if (word) {
+        CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off, 0, 4, st));
+        CELTY_CUDA(cudaStreamSynchronize(st));
+    }
+    if (word & kStatusTimeout) return CELTY_ETIMEOUT;
+    if (word & kStatusBounds) return CELTY_EBOUNDS;
+    return CELTY_OK;
+}

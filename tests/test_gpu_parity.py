@@ -1,0 +1,238 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bit-exact for the compacted list and the decoded indices; |y_gpu - y_ref| <= 2e-3 * sum_j |W_ij x_j|
++ 1e-6 per element for FP16-in / FP32-accumulate values; bit-exact too where the data make the FP32
+sum order-independent (small integers).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import celty_oracle as orc
+from paper_2608_01536_b200 import build, celty, synth
+
+pytestmark = pytest.mark.gpu
+
+LAYOUTS = [celty.LAYOUT_COLUMN, celty.LAYOUT_LANE_TILE]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    celty.load()
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _run(m, x, tau):
+    y = m.spmspv(_dev(x), tau)
+    torch.cuda.synchronize()
+    assert m.last_status() == 0
+    return y.cpu().numpy()
+
+
+def _check_y(y, W, mask, x, tau, exact=False):
+    y_ref, a_ref = orc.masked_gemv(W, mask, x, tau, threads=8)
+    if exact:
+        assert np.array_equal(y.astype(np.float64), y_ref)
+    else:
+        err = np.abs(y.astype(np.float64) - y_ref)
+        bound = 2e-3 * a_ref + 1e-6
+        worst = int(np.argmax(err - bound))
+        assert np.all(err <= bound), (worst, y[worst], y_ref[worst], a_ref[worst])
+
+
+# ----------------------------------------------------------------------------- compaction
+@pytest.mark.parametrize("K", [1, 7, 8, 9, 31, 33, 1000, 1024, 4096, 8191, 8193, 28672, 40000])
+def test_compaction_bit_exact(K):
+    x = synth.activations(K, K, "laplace")
+    if K > 40:
+        x[5] = np.float16(0.0)
+        x[6] = np.float16(-0.0)
+        x[17] = np.float16(np.nan)
+    xd = _dev(x)
+    amax = float(np.nanmax(np.abs(x.astype(np.float32))))
+    for tau in (0.0, synth.threshold_for_density(x, 0.5), synth.threshold_for_density(x, 0.1), amax, 1e4):
+        if not np.isfinite(tau):
+            continue
+        idx, val = celty.compact(xd, tau)
+        oi, ov, n = orc.compact(x, tau)
+        assert idx.numel() == n
+        assert np.array_equal(idx.cpu().numpy(), oi)
+        assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+
+
+def test_compaction_ties_are_dropped():
+    x = np.array([0.5, -0.5] * 20, np.float16)
+    assert celty.compact(_dev(x), 0.5)[0].numel() == 0
+    assert celty.compact(_dev(x), 0.499)[0].numel() == 40
+
+
+# ----------------------------------------------------------------------------- decode
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("M,K,d_w,tile_rows", [(257, 9, 0.5, 0), (4097, 6, 0.03, 0), (1000, 5, 1.0, 0),
+                                               (3000, 7, 0.3, 40), (28672, 3, 0.5, 0), (2100, 4, 0.9, 7)])
+def test_device_decode_bit_exact(layout, M, K, d_w, tile_rows):
+    if layout == celty.LAYOUT_COLUMN:
+        tile_rows = 0
+    W = synth.weights(M, M, K)
+    mask = synth.mask_bernoulli(M, M, K, d_w)
+    mask[:, 0] = 0                      # empty column
+    mask[:, 1] = 0
+    mask[-1, 1] = 1                     # only the last row: maximum number of pads
+    mask[:, 2] = 1                      # dense column
+    m = celty.Matrix(W, mask, layout=layout, tile_rows=tile_rows, device="cuda")
+    enc = orc.rlc_encode(W, mask, 4, tile_rows=m.info().tile_rows)
+    for j in range(K):
+        rows, vals = m.decode_device(j)
+        orows, ovals, _, _ = orc.column_entries(enc, j)
+        assert np.array_equal(rows, orows), j
+        assert np.array_equal(vals, ovals), j
+
+
+# ----------------------------------------------------------------------------- product
+SHAPES = [
+    # M, K, d_w, d_a
+    (1, 1, 1.0, 1.0),
+    (8, 8, 1.0, 1.0),
+    (64, 64, 0.5, 0.5),
+    (1000, 1003, 0.5, 0.5),
+    (4097, 33, 0.3, 0.7),
+    (257, 2050, 0.7, 0.3),
+    (1024, 1024, 0.5, 0.5),
+    (5120, 640, 0.5, 0.4),
+    (11008, 300, 0.5, 0.5),
+]
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("M,K,d_w,d_a", SHAPES)
+def test_spmspv_random_within_bound(layout, M, K, d_w, d_a):
+    seed = M * 7 + K
+    W = synth.weights(seed, M, K)
+    mask = synth.mask_bernoulli(seed, M, K, d_w)
+    x = synth.activations(seed, K, "laplace")
+    tau = synth.threshold_for_density(x, d_a)
+    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    y = _run(m, x, tau)
+    _check_y(y, W, mask, x, tau)
+    idx, val = m.last_compaction()
+    oi, ov, _ = orc.compact(x, tau)
+    assert np.array_equal(idx.cpu().numpy(), oi)
+    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("M,K,d_w,d_a,tile_rows", [(1000, 1003, 0.5, 0.5, 0), (4096, 512, 0.5, 0.5, 0),
+                                                    (777, 129, 0.2, 0.9, 5), (3000, 200, 0.6, 0.5, 24)])
+def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows):
+    """Small-integer W and x keep every partial sum below 2^24: FP32 addition is then exact in any
+    order, so the result must equal the fp64 definition bit for bit."""
+    if layout == celty.LAYOUT_COLUMN:
+        tile_rows = 0
+    W = synth.integer_weights(M + K, M, K)
+    mask = synth.mask_bernoulli(M + K, M, K, d_w)
+    x = synth.integer_activations(M + K, K)
+    tau = synth.threshold_for_density(x, d_a)
+    m = celty.Matrix(W, mask, layout=layout, tile_rows=tile_rows, device="cuda")
+    for grid in (0, 1, 3, 37):
+        m.set_launch(grid=grid)
+        y = _run(m, x, tau)
+        _check_y(y, W, mask, x, tau, exact=True)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_degenerate_cases(layout):
+    M, K = 600, 96
+    W = synth.weights(11, M, K)
+    mask = synth.mask_bernoulli(11, M, K, 0.5)
+    mask[:, :8] = 0                                   # empty columns
+    mask[:, 8] = 0
+    mask[-1, 8] = 1                                   # only the last row
+    mask[:, 9] = 1                                    # dense column
+    x = synth.activations(11, K, "laplace")
+    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    amax = float(np.abs(x.astype(np.float32)).max())
+    # no survivor: y must be overwritten with zeros
+    y = m.spmspv(_dev(x), amax, y=torch.full((M,), 7.0, device="cuda"))
+    assert torch.count_nonzero(y).item() == 0
+    # every activation survives
+    xs = x.copy()
+    xs[xs == 0] = np.float16(1.0)
+    _check_y(_run(m, xs, 0.0), W, mask, xs, 0.0)
+    # only empty columns survive
+    xe = np.zeros(K, np.float16)
+    xe[:8] = 1.0
+    assert np.count_nonzero(_run(m, xe, 0.0)) == 0
+    # unit vector selects a column exactly
+    for j in (8, 9, 50):
+        xu = np.zeros(K, np.float16)
+        xu[j] = 1.0
+        y = _run(m, xu, 0.0)
+        assert np.array_equal(y, np.where(mask[:, j] != 0, W[:, j].astype(np.float32), np.float32(0)))
+    # repeated calls on the same handle give the same answer
+    tau = synth.threshold_for_density(x, 0.5)
+    y1 = _run(m, x, tau)
+    y2 = _run(m, x, tau)
+    _check_y(y1, W, mask, x, tau)
+    assert np.allclose(y1, y2, rtol=0, atol=1e-5)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_identity_returns_thresholded_x(layout):
+    K = 300
+    W = np.eye(K, dtype=np.float16)
+    x = synth.activations(2, K, "laplace")
+    m = celty.Matrix(W, None, layout=layout, device="cuda")
+    y = _run(m, x, 0.6)
+    xf = x.astype(np.float32)
+    assert np.array_equal(y, np.where(np.abs(xf) > np.float32(0.6), xf, np.float32(0)))
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_longest_column_and_power_law_rows(layout):
+    """M = 28672 (the tallest configured layer): a fully dense column (112 chunks of 256 entries),
+    a column with only its last row, and row-clustered power-law masks."""
+    M, K = 28672, 96
+    W = synth.weights(5, M, K)
+    mask = synth.mask_powerlaw(5, M, K, 0.3)
+    mask[:, 0] = 1
+    mask[:, 1] = 0
+    mask[-1, 1] = 1
+    x = synth.activations(5, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.7)
+    x[0] = np.float16(2.0)
+    x[1] = np.float16(-3.0)
+    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    _check_y(_run(m, x, tau), W, mask, x, tau)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_llama7b_attention_shape_in_bench_configuration(layout):
+    """4096 x 4096, magnitude-pruned 50% per column, Laplace activations kept at 50%: the workload
+    and launch configuration bench.py times, compared in full."""
+    M = K = 4096
+    W = synth.weights(synth.point_seed(2, 4), M, K)
+    mask = synth.mask_magnitude(W, 0.5)
+    x = synth.activations(synth.point_seed(2, 4), K, "laplace")
+    tau = synth.threshold_for_density(x, 0.5)
+    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    _check_y(_run(m, x, tau), W, mask, x, tau)
+
+
+def test_host_buffer_entry_point():
+    M, K = 1024, 1024
+    W = synth.weights(1, M, K)
+    mask = synth.mask_bernoulli(1, M, K, 0.5)
+    x = synth.activations(1, K, "normal")
+    tau = synth.threshold_for_density(x, 0.5)
+    m = celty.Matrix(W, mask, device="cuda")
+    xh = torch.from_numpy(x.copy()).pin_memory()
+    yh = torch.empty(M, dtype=torch.float32).pin_memory()
+    xs = torch.empty(K, dtype=torch.float16, device="cuda")
+    ys = torch.empty(M, dtype=torch.float32, device="cuda")
+    m.spmspv_host(xh, tau, yh, xs, ys)
+    _check_y(yh.numpy(), W, mask, x, tau)

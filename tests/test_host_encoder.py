@@ -1,0 +1,103 @@
+"""The library's host encoder against the oracle's, on the logical arrays (two independent programs)."""
+import numpy as np
+import pytest
+
+from conftest import read_golden
+from oracle import celty_oracle as orc
+from paper_2608_01536_b200 import build, celty, synth
+
+build.build()
+
+CASES = [
+    # M, K, d_w, layout, tile_rows
+    (257, 19, 0.5, celty.LAYOUT_COLUMN, 0),
+    (1000, 37, 0.3, celty.LAYOUT_COLUMN, 0),
+    (4097, 5, 0.02, celty.LAYOUT_COLUMN, 0),
+    (64, 7, 1.0, celty.LAYOUT_COLUMN, 0),
+    (300, 9, 0.0, celty.LAYOUT_COLUMN, 0),
+    (257, 19, 0.5, celty.LAYOUT_LANE_TILE, 0),
+    (1000, 37, 0.3, celty.LAYOUT_LANE_TILE, 16),
+    (4097, 5, 0.02, celty.LAYOUT_LANE_TILE, 100),
+    (4097, 5, 0.6, celty.LAYOUT_LANE_TILE, 0),
+    (64, 7, 1.0, celty.LAYOUT_LANE_TILE, 8),
+    (300, 9, 0.0, celty.LAYOUT_LANE_TILE, 0),
+    (33, 3, 0.5, celty.LAYOUT_LANE_TILE, 1),
+]
+
+
+@pytest.mark.parametrize("M,K,d_w,layout,tile_rows", CASES)
+def test_encoder_matches_oracle(M, K, d_w, layout, tile_rows):
+    W = synth.weights(M + K, M, K)
+    mask = synth.mask_bernoulli(M + K, M, K, d_w)
+    m = celty.Matrix(W, mask, layout=layout, tile_rows=tile_rows)
+    info = m.info()
+    R = info.tile_rows
+    assert (R == 0) == (layout == celty.LAYOUT_COLUMN)
+    enc = orc.rlc_encode(W, mask, 4, tile_rows=R)
+    assert info.nnz == int(mask.sum())
+    assert info.n_pad == int(enc.is_pad.sum())
+    assert info.compressed_bytes == enc.vals.size * 5 // 2 + 4 * (K + 1)
+    for j in range(K):
+        rows, vals, runs, pad = m.decode_host(j)
+        orows, ovals, opad, oruns = orc.column_entries(enc, j)
+        assert np.array_equal(rows, orows)
+        assert np.array_equal(vals, ovals)
+        assert np.array_equal(runs, oruns)
+        assert np.array_equal(pad, opad)
+
+
+def test_null_mask_keeps_nonzero_weights():
+    W = synth.weights(3, 100, 11)
+    W[::3] = 0
+    W[1, 1] = np.float16(-0.0)
+    m = celty.Matrix(W, None, layout=celty.LAYOUT_COLUMN)
+    enc = orc.rlc_encode(W, (W.view(np.uint16) & 0x7FFF) != 0, 4)
+    assert m.info().nnz == int(((W.view(np.uint16) & 0x7FFF) != 0).sum())
+    for j in range(11):
+        assert np.array_equal(m.decode_host(j)[0], orc.column_entries(enc, j)[0])
+
+
+@pytest.mark.parametrize("name", sorted(read_golden("rlc_hand_vectors_4bit.txt")))
+@pytest.mark.parametrize("layout", [celty.LAYOUT_COLUMN, celty.LAYOUT_LANE_TILE])
+def test_library_encoder_on_hand_vectors(name, layout):
+    c = read_golden("rlc_hand_vectors_4bit.txt")[name]
+    M = c["M"][0]
+    W = np.zeros((M, 1), np.float16)
+    mask = np.zeros((M, 1), np.uint8)
+    for r in c["kept_rows"]:
+        W[r, 0] = r + 1
+        mask[r, 0] = 1
+    # one tile covering the whole column reproduces the whole-column encoding
+    m = celty.Matrix(W, mask, layout=layout, tile_rows=0 if layout == celty.LAYOUT_COLUMN else max(4, M))
+    rows, vals, runs, pad = m.decode_host(0)
+    assert rows.tolist() == c["rows"] and runs.tolist() == c["runs"] and pad.tolist() == c["is_pad"]
+
+
+def test_packed_run_nibbles_are_little_endian():
+    # 8 runs [0,15,0,15,5,1,2,3] must pack to the word 0x3215F0F0 (entry e in bits 4e..4e+3)
+    rows = np.cumsum([0, 16, 1, 16, 6, 2, 3, 4])
+    M = int(rows[-1]) + 1
+    W = np.zeros((M, 1), np.float16)
+    W[rows, 0] = np.arange(1, 9)
+    m = celty.Matrix(W, None, layout=celty.LAYOUT_COLUMN)
+    assert m.decode_host(0)[2].tolist() == [0, 15, 0, 15, 5, 1, 2, 3]
+    image, off = m.host_image()
+    # the column's single group: 16 bytes of values, then its run word
+    assert image[off:off + 16].view(np.float16).tolist() == [1, 2, 3, 4, 5, 6, 7, 8]
+    assert int(image[off + 16:off + 20].view(np.uint32)[0]) == 0x3215F0F0
+
+
+def test_fetched_bytes_accounting():
+    M, K = 512, 40
+    W = synth.weights(1, M, K)
+    mask = synth.mask_bernoulli(1, M, K, 0.5)
+    enc = orc.rlc_encode(W, mask, 4)
+    m = celty.Matrix(W, mask, layout=celty.LAYOUT_COLUMN)
+    idx = np.array([0, 3, 17, 39], np.int32)
+    sb, tb = m.fetched_bytes(idx)
+    n_j = np.diff(enc.block_ptr)[idx]
+    expect = sum(((int(n) + 7) // 8 * 20 + 15) // 16 * 16 for n in n_j)
+    assert sb == expect
+    assert abs(sb - 2.5 * n_j.sum()) <= 2.5 * 8 * idx.size + 16 * idx.size
+    assert tb == sb + 8 * idx.size + 2 * K + 12 * idx.size + 8 * M
+    assert m.fetched_bytes(np.zeros(0, np.int32)) == (0, 2 * K + 8 * M)
