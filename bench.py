@@ -199,7 +199,7 @@ def run_celty(args):
     # ---- workload: a few distinct matrices, replicated on the device until the copies exceed 2x L2
     l2 = torch.cuda.get_device_properties(dev).L2_cache_size
     distinct = [make_layer(name, v) for v in range(args.distinct)]
-    probe = celty.Matrix(*distinct[0], layout=layout)
+    probe = celty.Matrix(*distinct[0], layout=layout, tile_rows=args.tile_rows)
     image_bytes = probe.device_bytes()[0]
     copies = max(args.distinct, int(np.ceil(2.5 * l2 / image_bytes)) + 1)
     if args.copies:
@@ -207,9 +207,9 @@ def run_celty(args):
     mats, xs, taus, fetched = [], [], [], []
     for c in range(copies):
         W, mask = distinct[c % args.distinct]
-        m = celty.Matrix(W, mask, layout=layout, device=dev)
-        if args.grid or args.variant:
-            m.set_launch(args.grid, args.variant)
+        m = celty.Matrix(W, mask, layout=layout, tile_rows=args.tile_rows, device=dev)
+        if args.grid or args.variant or args.groups or args.depth:
+            m.set_launch(args.grid, args.variant, args.groups, args.depth)
         x, tau = make_x(name, c)
         mats.append(m)
         xs.append(torch.from_numpy(x).to(dev))
@@ -352,7 +352,7 @@ def run_celty(args):
                      "note": "time per call covers every kernel of the call"},
         "e2e": {"value": world * total_bytes / e2e_sec / 1e9, "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
                 "h2d_bytes_per_step": 2 * K, "d2h_bytes_per_step": 4 * M},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": (1 if (layout == celty.LAYOUT_LANE_TILE and args.variant == 0) else 2) * args.steps,
         "clocks": clocks.summary(),
         "context": {"us_per_call_stream_enqueued": us_enqueued, "us_per_call_l2_warm": us_warm,
                     "cublas_gemv_fp16_us": dense_us,
@@ -382,6 +382,9 @@ def main():
     ap.add_argument("--copies", type=int, default=0, help="device copies in the rotation (0 = enough for 2.5x L2)")
     ap.add_argument("--grid", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--groups", type=int, default=0)
+    ap.add_argument("--depth", type=int, default=0)
+    ap.add_argument("--tile-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -199,9 +199,16 @@ int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx_host, int64_t 
  */
 int celty_last_status(celty_matrix *m, celty_stream_t stream);
 
-/* Tuning knob for experiments: thread blocks per launch (0 = default, one per SM times the
- * kernel's residency) and the kernel variant (0 = default for the layout). */
-int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant);
+/*
+ * celty_set_launch -- tuning knobs for experiments and tests; 0 = the library's choice.
+ *   grid     thread blocks per launch (rounded down to what fits the device at once)
+ *   variant  LANE_TILE only: 0 = single fused launch (compaction + bulk-copy pipeline + reduction),
+ *            1 = two launches (compaction kernel, then a kernel that loads straight from global memory)
+ *   groups   fused kernel: warp groups per block working on different columns
+ *   depth    fused kernel: bulk copies each warp keeps in flight (ring slots)
+ * Errors: CELTY_EINVAL.
+ */
+int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth);
 
 /* The cudaError_t of the last failing CUDA call made through this library (0 if none). */
 int celty_last_cuda_error(void);

@@ -336,11 +336,14 @@ extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, in
     return CELTY_OK;
 }
 
-extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant)
+extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth)
 {
-    if (!m || grid < 0 || variant < 0) return CELTY_EINVAL;
+    if (!m || grid < 0 || variant < 0 || variant > 1 || groups < 0 || groups > 32 || depth < 0 || depth > 16)
+        return CELTY_EINVAL;
     m->grid = grid;
     m->variant = variant;
+    m->groups = groups;
+    m->depth = depth;
     return CELTY_OK;
 }
 

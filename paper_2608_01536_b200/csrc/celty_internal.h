@@ -18,7 +18,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Workspace layout (device): all offsets multiples of 256.
 struct WorkspaceLayout {
-    size_t status_off;   // uint32 status, int32 count (and spare words)
+    size_t status_off;   // uint32 status, int32 count, uint32 tickets[2] (and spare words)
     size_t idx_off;      // int32[K]
     size_t val_off;      // uint16[K]
     size_t scratch_off;  // uint32[T + 2] for celty_decode_device
@@ -61,5 +61,5 @@ struct celty_matrix {
     uint8_t *d_image = nullptr;
     uint8_t *d_ws = nullptr;
     celty::WorkspaceLayout ws{};
-    int32_t grid = 0, variant = 0;
+    int32_t grid = 0, variant = 0, groups = 0, depth = 0;
 };

@@ -372,6 +372,8 @@ int ensure_smem(Kernel kernel, size_t bytes, int *granted /* [64], per device */
     return CELTY_OK;
 }
 
+#include "celty_fused.cuh"
+
 int launch_compact(const void *x, int64_t K, float tau, int32_t *idx, uint16_t *val, int32_t *count, float *y,
                    int64_t M, cudaStream_t st)
 {
@@ -380,9 +382,48 @@ int launch_compact(const void *x, int64_t K, float tau, int32_t *idx, uint16_t *
     return CELTY_OK;
 }
 
+// Shape of the fused launch: P row parts of Sc slabs, G warp groups, D ring slots per warp.
+int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
+{
+    FusedPlan pl{};
+    const int S = (int)m->S;
+    pl.P = (S + 3) / 4;
+    pl.Sc = (S + pl.P - 1) / pl.P;
+    pl.slot_bytes = (int)round_up((size_t)m->max_unit16 * 16, 128);
+    pl.cap = 64;
+    const size_t budget = (size_t)di.max_smem_optin;
+    const int g_max = std::max(1, std::min(32 / pl.Sc, m->groups > 0 ? m->groups : std::max(1, 8 / pl.Sc)));
+    const int d_want = m->depth > 0 ? m->depth : 3;
+    pl.G = 0;
+    for (int d = d_want; d >= 1 && pl.G == 0; --d)
+        for (int g = g_max; g >= 1; --g)
+            if (fused_smem_bytes(m->R, (int)m->K, g, pl.Sc, d, pl.slot_bytes, pl.cap) <= budget) {
+                // prefer keeping two copies in flight over a wider block
+                if (d >= 2 || g == 1 || d_want == 1) { pl.G = g; pl.D = d; break; }
+            }
+    if (pl.G == 0) return CELTY_EINVAL;
+    pl.threads = 32 * pl.G * pl.Sc;
+    pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
+    int blocks = di.sms;                       // every block must be resident: they wait for one another's tickets
+    if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
+    pl.grid = std::max(1, blocks / pl.P) * pl.P;
+    if (pl.grid > di.sms) return CELTY_EINVAL;
+    *out = pl;
+    return CELTY_OK;
+}
+
 }  // namespace
 
 extern "C" int celty_last_cuda_error(void) { return g_last_cuda; }
+
+#ifdef CELTY_TRACE
+// Development builds only: where the fused kernel stores its phase timestamps (device pointer, 16 per block).
+extern "C" int celty_debug_set_trace(long long *trace_dev)
+{
+    CELTY_CUDA(cudaMemcpyToSymbol(g_celty_trace, &trace_dev, sizeof(trace_dev)));
+    return CELTY_OK;
+}
+#endif
 
 extern "C" int celty_bind_device(celty_matrix *m, void *image_dev, size_t image_bytes, void *workspace_dev,
                                  size_t workspace_bytes, celty_stream_t stream)
@@ -422,9 +463,30 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
     int32_t *idx = reinterpret_cast<int32_t *>(m->d_ws + m->ws.idx_off);
     uint16_t *val = reinterpret_cast<uint16_t *>(m->d_ws + m->ws.val_off);
     float *y = static_cast<float *>(y_dev);
+    const uint8_t *stream_base = m->d_image + m->meta_bytes;
+    if (m->layout == CELTY_LAYOUT_LANE_TILE && m->variant == 0) {
+        FusedPlan plan;
+        rc = plan_fused(m, di, &plan);
+        if (rc) return rc;
+        static int granted[64];
+        rc = ensure_smem(k_spmspv_fused, plan.smem, granted);
+        if (rc) return rc;
+        FusedParams fp;
+        fp.meta = reinterpret_cast<const uint32_t *>(m->d_image);
+        fp.stream = stream_base;
+        fp.x = static_cast<const uint16_t *>(x_dev);
+        fp.tau = tau;
+        fp.y = y;
+        fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
+        fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.T = (int)m->T;
+        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D;
+        fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
+        k_spmspv_fused<<<plan.grid, plan.threads, plan.smem, st>>>(fp);
+        CELTY_CUDA(cudaGetLastError());
+        return CELTY_OK;
+    }
     rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);
     if (rc) return rc;
-    const uint8_t *stream_base = m->d_image + m->meta_bytes;
     if (m->layout == CELTY_LAYOUT_COLUMN) {
         const size_t smem = (size_t)m->M * 4;
         if (smem > (size_t)di.max_smem_optin) return CELTY_EINVAL;
@@ -435,11 +497,11 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         const int grid = m->grid > 0 ? m->grid : di.sms * per_sm;
         k_spmspv_column<<<grid, 256, smem, st>>>(reinterpret_cast<const uint2 *>(m->d_image), stream_base, idx, val,
                                                   count, y, (int)m->M, status);
-    } else {
+    } else if (m->variant == 1) {
         const size_t group_bytes = (size_t)m->S * (m->R + kTileSlack) * 32 * 4;
-        if (group_bytes > (size_t)di.max_smem_optin || m->S > 32) return CELTY_EINVAL;
+        if (group_bytes > (size_t)di.max_smem_optin) return CELTY_EINVAL;
         int G = (int)std::min<size_t>((size_t)di.max_smem_optin / group_bytes, (size_t)(32 / m->S));
-        G = std::max(1, std::min(G, m->variant > 0 ? m->variant : (int)std::max<int64_t>(1, 8 / m->S)));
+        G = std::max(1, std::min(G, m->groups > 0 ? m->groups : (int)std::max<int64_t>(1, 8 / m->S)));
         const size_t smem = group_bytes * G;
         static int granted[64];
         rc = ensure_smem(k_spmspv_lane, smem, granted);
@@ -509,7 +571,9 @@ extern "C" int celty_last_status(celty_matrix *m, celty_stream_t stream)
     CELTY_CUDA(cudaMemcpyAsync(&word, m->d_ws + m->ws.status_off, 4, cudaMemcpyDeviceToHost, st));
     CELTY_CUDA(cudaStreamSynchronize(st));
     if (word) {
+        // also reset the fused kernel's tickets, which a run that gave up may have left mid-count
         CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off, 0, 4, st));
+        CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
         CELTY_CUDA(cudaStreamSynchronize(st));
     }
     if (word & kStatusTimeout) return CELTY_ETIMEOUT;

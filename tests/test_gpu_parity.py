@@ -13,7 +13,19 @@ from paper_2608_01536_b200 import build, celty, synth
 
 pytestmark = pytest.mark.gpu
 
-LAYOUTS = [celty.LAYOUT_COLUMN, celty.LAYOUT_LANE_TILE]
+# (layout, variant): the published column formulation, the fused lane-tile kernel, and the
+# two-launch lane-tile path
+LAYOUTS = [(celty.LAYOUT_COLUMN, 0), (celty.LAYOUT_LANE_TILE, 0), (celty.LAYOUT_LANE_TILE, 1)]
+DECODE_LAYOUTS = [celty.LAYOUT_COLUMN, celty.LAYOUT_LANE_TILE]
+
+
+def _matrix(W, mask, lv, tile_rows=0):
+    layout, variant = lv
+    m = celty.Matrix(W, mask, layout=layout, tile_rows=0 if layout == celty.LAYOUT_COLUMN else tile_rows,
+                     device="cuda")
+    m.set_launch(variant=variant)
+    m.variant = variant
+    return m
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -72,7 +84,7 @@ def test_compaction_ties_are_dropped():
 
 
 # ----------------------------------------------------------------------------- decode
-@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("layout", DECODE_LAYOUTS)
 @pytest.mark.parametrize("M,K,d_w,tile_rows", [(257, 9, 0.5, 0), (4097, 6, 0.03, 0), (1000, 5, 1.0, 0),
                                                (3000, 7, 0.3, 40), (28672, 3, 0.5, 0), (2100, 4, 0.9, 7)])
 def test_device_decode_bit_exact(layout, M, K, d_w, tile_rows):
@@ -116,7 +128,7 @@ def test_spmspv_random_within_bound(layout, M, K, d_w, d_a):
     mask = synth.mask_bernoulli(seed, M, K, d_w)
     x = synth.activations(seed, K, "laplace")
     tau = synth.threshold_for_density(x, d_a)
-    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    m = _matrix(W, mask, layout)
     y = _run(m, x, tau)
     _check_y(y, W, mask, x, tau)
     idx, val = m.last_compaction()
@@ -131,15 +143,13 @@ def test_spmspv_random_within_bound(layout, M, K, d_w, d_a):
 def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows):
     """Small-integer W and x keep every partial sum below 2^24: FP32 addition is then exact in any
     order, so the result must equal the fp64 definition bit for bit."""
-    if layout == celty.LAYOUT_COLUMN:
-        tile_rows = 0
     W = synth.integer_weights(M + K, M, K)
     mask = synth.mask_bernoulli(M + K, M, K, d_w)
     x = synth.integer_activations(M + K, K)
     tau = synth.threshold_for_density(x, d_a)
-    m = celty.Matrix(W, mask, layout=layout, tile_rows=tile_rows, device="cuda")
-    for grid in (0, 1, 3, 37):
-        m.set_launch(grid=grid)
+    m = _matrix(W, mask, layout, tile_rows)
+    for grid, groups, depth in ((0, 0, 0), (1, 0, 0), (3, 1, 1), (37, 3, 2), (148, 2, 4)):
+        m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth)
         y = _run(m, x, tau)
         _check_y(y, W, mask, x, tau, exact=True)
 
@@ -154,7 +164,7 @@ def test_degenerate_cases(layout):
     mask[-1, 8] = 1                                   # only the last row
     mask[:, 9] = 1                                    # dense column
     x = synth.activations(11, K, "laplace")
-    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    m = _matrix(W, mask, layout)
     amax = float(np.abs(x.astype(np.float32)).max())
     # no survivor: y must be overwritten with zeros
     y = m.spmspv(_dev(x), amax, y=torch.full((M,), 7.0, device="cuda"))
@@ -186,7 +196,7 @@ def test_identity_returns_thresholded_x(layout):
     K = 300
     W = np.eye(K, dtype=np.float16)
     x = synth.activations(2, K, "laplace")
-    m = celty.Matrix(W, None, layout=layout, device="cuda")
+    m = _matrix(W, None, layout)
     y = _run(m, x, 0.6)
     xf = x.astype(np.float32)
     assert np.array_equal(y, np.where(np.abs(xf) > np.float32(0.6), xf, np.float32(0)))
@@ -206,7 +216,7 @@ def test_longest_column_and_power_law_rows(layout):
     tau = synth.threshold_for_density(x, 0.7)
     x[0] = np.float16(2.0)
     x[1] = np.float16(-3.0)
-    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    m = _matrix(W, mask, layout)
     _check_y(_run(m, x, tau), W, mask, x, tau)
 
 
@@ -219,7 +229,7 @@ def test_llama7b_attention_shape_in_bench_configuration(layout):
     mask = synth.mask_magnitude(W, 0.5)
     x = synth.activations(synth.point_seed(2, 4), K, "laplace")
     tau = synth.threshold_for_density(x, 0.5)
-    m = celty.Matrix(W, mask, layout=layout, device="cuda")
+    m = _matrix(W, mask, layout)
     _check_y(_run(m, x, tau), W, mask, x, tau)
 
 
