@@ -113,8 +113,8 @@ int celty_host_image(const celty_matrix *m, const void **image, size_t *image_by
 /*
  * celty_device_bytes -- how much device memory the caller must provide:
  *   image_bytes      the packed matrix as the kernels read it (column metadata + entry stream)
- *   workspace_bytes  per-handle scratch: compacted activation list (indices, values, count) and
- *                    the status word
+ *   workspace_bytes  per-handle scratch: compacted activation list (indices, values, count), the
+ *                    status word, and the per-block partial sums of the split-K merge
  * Both are multiples of 256; the buffers must be 256-byte aligned.
  */
 int celty_device_bytes(const celty_matrix *m, size_t *image_bytes, size_t *workspace_bytes);
@@ -144,9 +144,10 @@ int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *idx_dev, uin
 
 /*
  * celty_spmspv -- the hot path: y = W . threshold(x, tau), batch 1 (Sections 3.1-3.3).
- * Enqueues on `stream`: activation compaction (+ clearing y), then the SpMSpV kernel that visits
- * only the surviving columns, decodes their runs to rows, accumulates value * x_j in shared memory
- * in FP32 (fmaf) and reduces the partial sums into y.
+ * Enqueues on `stream` one kernel (LANE_TILE layout) that thresholds and compacts x, visits only
+ * the surviving columns, decodes their runs to rows, accumulates value * x_j in shared memory in
+ * FP32 (fmaf) and reduces the per-block partial sums into y; the COLUMN layout uses a compaction
+ * kernel followed by the SpMSpV kernel.
  *   x_dev  K FP16 (device, 16-byte aligned), not modified
  *   y_dev  M FP32 (device, 16-byte aligned), overwritten
  * The order of FP32 additions is not fixed (Section 4.2: scatter-accumulation is order-
@@ -187,8 +188,9 @@ int celty_decode_device(celty_matrix *m, int64_t col, int32_t *rows_dev, uint16_
 /*
  * celty_fetched_bytes -- algorithmic HBM bytes of one celty_spmspv call for a given surviving
  * column list (host array of n ascending indices): entry stream of those columns as laid out
- * (including alignment padding and per-block headers), their metadata words, x, the list written
- * and read back, and y written (cleared + reduced).  Host-only arithmetic on the handle's tables.
+ * (including alignment padding and per-block headers), their metadata words, x read once, the
+ * list written, y written once.  Scratch traffic of the split-K merge is not counted.  Host-only
+ * arithmetic on the handle's tables.
  */
 int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx_host, int64_t n, int64_t *stream_bytes,
                         int64_t *total_bytes);

@@ -2,6 +2,7 @@
 // host-side decoding for round-trip tests and byte accounting.  No CUDA calls in this file.
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -206,7 +207,11 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
                 }
         }
         if (m->layout == CELTY_LAYOUT_COLUMN) pack_column(m, lg); else pack_lane_tile(m, lg);
-        m->ws = workspace_layout(K, T);
+        int spb = kSlabsPerBlock;
+        if (const char *e = std::getenv("CELTY_SLABS_PER_BLOCK")) spb = std::max(1, std::atoi(e));
+        m->P = (int32_t)((m->S + spb - 1) / spb);
+        m->Sc = (int32_t)((m->S + m->P - 1) / m->P);
+        m->ws = workspace_layout(K, T, m->layout == CELTY_LAYOUT_LANE_TILE ? (int64_t)m->Sc * m->R * 32 : 0);
         *out = m;
         return CELTY_OK;
     } catch (const std::bad_alloc &) {
@@ -331,14 +336,15 @@ extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, in
         }
     }
     if (stream_bytes) *stream_bytes = sb;
-    // x read, list written then read (4-byte index + 2-byte value each way), y cleared and reduced
-    if (total_bytes) *total_bytes = sb + mb + 2 * m->K + 12 * n + 8 * m->M;
+    // x read once, the list written (4-byte index + 2-byte value), y written once.  Scratch traffic of
+    // the split-K merge (per-block partial sums) is not counted: it is overhead, not work.
+    if (total_bytes) *total_bytes = sb + mb + 2 * m->K + 6 * n + 4 * m->M;
     return CELTY_OK;
 }
 
 extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth)
 {
-    if (!m || grid < 0 || variant < 0 || variant > 1 || groups < 0 || groups > 32 || depth < 0 || depth > 16)
+    if (!m || grid < 0 || variant < 0 || variant > 7 || groups < 0 || groups > 32 || depth < 0 || depth > 16)
         return CELTY_EINVAL;
     m->grid = grid;
     m->variant = variant;

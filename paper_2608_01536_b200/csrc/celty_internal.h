@@ -13,6 +13,8 @@ constexpr int kChunkGroups = 32;     // COLUMN layout: groups per warp-wide chun
 constexpr int kTileSlack = 8;        // LANE_TILE: spare accumulator rows per slab for group-tail slots
 constexpr int64_t kMaxM = 49152;     // accumulators of one thread block must fit shared memory
 constexpr size_t kAlign = 256;
+constexpr int kMaxBlocks = 192;      // blocks of the fused kernel the workspace has partial vectors for
+constexpr int kSlabsPerBlock = 4;    // LANE_TILE: a thread block covers at most this many slabs of rows
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -22,17 +24,19 @@ struct WorkspaceLayout {
     size_t idx_off;      // int32[K]
     size_t val_off;      // uint16[K]
     size_t scratch_off;  // uint32[T + 2] for celty_decode_device
+    size_t partial_off;  // float[kMaxBlocks][part_words]: per-block partial sums of the fused kernel
     size_t total;
 };
 
-inline WorkspaceLayout workspace_layout(int64_t K, int64_t T)
+inline WorkspaceLayout workspace_layout(int64_t K, int64_t T, int64_t part_words)
 {
     WorkspaceLayout w{};
     w.status_off = 0;
     w.idx_off = kAlign;
     w.val_off = w.idx_off + round_up((size_t)K * 4, kAlign);
     w.scratch_off = w.val_off + round_up((size_t)K * 2, kAlign);
-    w.total = w.scratch_off + round_up((size_t)(T + 2) * 4, kAlign);
+    w.partial_off = w.scratch_off + round_up((size_t)(T + 2) * 4, kAlign);
+    w.total = w.partial_off + round_up((size_t)kMaxBlocks * part_words * 4, kAlign);
     return w;
 }
 
@@ -46,6 +50,7 @@ struct celty_matrix {
     int32_t R = 0;          // rows per tile (LANE_TILE) or M (COLUMN)
     int64_t T = 1;          // tiles per column
     int64_t S = 1;          // slabs of 32 tiles per column (LANE_TILE), 1 for COLUMN
+    int32_t P = 1, Sc = 1;  // LANE_TILE: row parts per column and slabs per part (P * Sc >= S)
     int64_t nnz = 0, n_pad = 0;
     std::vector<uint32_t> block_ptr;   // K*T + 1, stored entries before block (j, t)
     std::vector<uint8_t> pad_bits;     // one bit per stored entry (logical order): 1 = padding entry

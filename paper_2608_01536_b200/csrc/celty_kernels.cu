@@ -386,13 +386,12 @@ int launch_compact(const void *x, int64_t K, float tau, int32_t *idx, uint16_t *
 int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
 {
     FusedPlan pl{};
-    const int S = (int)m->S;
-    pl.P = (S + 3) / 4;
-    pl.Sc = (S + pl.P - 1) / pl.P;
+    pl.P = m->P;
+    pl.Sc = m->Sc;
     pl.slot_bytes = (int)round_up((size_t)m->max_unit16 * 16, 128);
     pl.cap = 64;
     const size_t budget = (size_t)di.max_smem_optin;
-    const int g_max = std::max(1, std::min(32 / pl.Sc, m->groups > 0 ? m->groups : std::max(1, 8 / pl.Sc)));
+    const int g_max = std::max(1, std::min(16 / pl.Sc, m->groups > 0 ? m->groups : std::max(1, 8 / pl.Sc)));
     const int d_want = m->depth > 0 ? m->depth : 3;
     pl.G = 0;
     for (int d = d_want; d >= 1 && pl.G == 0; --d)
@@ -402,9 +401,11 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
                 if (d >= 2 || g == 1 || d_want == 1) { pl.G = g; pl.D = d; break; }
             }
     if (pl.G == 0) return CELTY_EINVAL;
-    pl.threads = 32 * pl.G * pl.Sc;
+    // streaming warps first; with variant bit 2 the block is filled up to 512 threads with warps that
+    // only help with the data-parallel phases
+    pl.threads = (m->variant & 4) ? std::max(512, 32 * pl.G * pl.Sc) : 32 * pl.G * pl.Sc;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
-    int blocks = di.sms;                       // every block must be resident: they wait for one another's tickets
+    int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
     pl.grid = std::max(1, blocks / pl.P) * pl.P;
     if (pl.grid > di.sms) return CELTY_EINVAL;
@@ -416,7 +417,7 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
 
 extern "C" int celty_last_cuda_error(void) { return g_last_cuda; }
 
-#ifdef CELTY_TRACE
+#if defined(CELTY_TRACE) || defined(CELTY_GUARD)
 // Development builds only: where the fused kernel stores its phase timestamps (device pointer, 16 per block).
 extern "C" int celty_debug_set_trace(long long *trace_dev)
 {
@@ -464,7 +465,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
     uint16_t *val = reinterpret_cast<uint16_t *>(m->d_ws + m->ws.val_off);
     float *y = static_cast<float *>(y_dev);
     const uint8_t *stream_base = m->d_image + m->meta_bytes;
-    if (m->layout == CELTY_LAYOUT_LANE_TILE && m->variant == 0) {
+    if (m->layout == CELTY_LAYOUT_LANE_TILE && (m->variant & 1) == 0) {
         FusedPlan plan;
         rc = plan_fused(m, di, &plan);
         if (rc) return rc;
@@ -478,9 +479,12 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.tau = tau;
         fp.y = y;
         fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
+        fp.partials = reinterpret_cast<float *>(m->d_ws + m->ws.partial_off);
         fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.T = (int)m->T;
         fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
+        fp.stream_bytes = (long long)m->stream_bytes;
+        fp.flags = (m->variant & 2) ? 1 : 0;
         k_spmspv_fused<<<plan.grid, plan.threads, plan.smem, st>>>(fp);
         CELTY_CUDA(cudaGetLastError());
         return CELTY_OK;
@@ -497,7 +501,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         const int grid = m->grid > 0 ? m->grid : di.sms * per_sm;
         k_spmspv_column<<<grid, 256, smem, st>>>(reinterpret_cast<const uint2 *>(m->d_image), stream_base, idx, val,
                                                   count, y, (int)m->M, status);
-    } else if (m->variant == 1) {
+    } else {
         const size_t group_bytes = (size_t)m->S * (m->R + kTileSlack) * 32 * 4;
         if (group_bytes > (size_t)di.max_smem_optin) return CELTY_EINVAL;
         int G = (int)std::min<size_t>((size_t)di.max_smem_optin / group_bytes, (size_t)(32 / m->S));

@@ -99,5 +99,5 @@ def test_fetched_bytes_accounting():
     expect = sum(((int(n) + 7) // 8 * 20 + 15) // 16 * 16 for n in n_j)
     assert sb == expect
     assert abs(sb - 2.5 * n_j.sum()) <= 2.5 * 8 * idx.size + 16 * idx.size
-    assert tb == sb + 8 * idx.size + 2 * K + 12 * idx.size + 8 * M
-    assert m.fetched_bytes(np.zeros(0, np.int32)) == (0, 2 * K + 8 * M)
+    assert tb == sb + 8 * idx.size + 2 * K + 6 * idx.size + 4 * M
+    assert m.fetched_bytes(np.zeros(0, np.int32)) == (0, 2 * K + 4 * M)
