@@ -208,8 +208,8 @@ def run_celty(args):
     for c in range(copies):
         W, mask = distinct[c % args.distinct]
         m = celty.Matrix(W, mask, layout=layout, tile_rows=args.tile_rows, device=dev)
-        if args.grid or args.variant or args.groups or args.depth:
-            m.set_launch(args.grid, args.variant, args.groups, args.depth)
+        if args.grid or args.variant or args.groups or args.depth or args.team:
+            m.set_launch(args.grid, args.variant, args.groups, args.depth, args.team)
         x, tau = make_x(name, c)
         mats.append(m)
         xs.append(torch.from_numpy(x).to(dev))
@@ -384,6 +384,7 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--groups", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
+    ap.add_argument("--team", type=int, default=0)
     ap.add_argument("--tile-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-dense", action="store_true")

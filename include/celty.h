@@ -57,7 +57,7 @@ enum { CELTY_LAYOUT_COLUMN = 0, CELTY_LAYOUT_LANE_TILE = 1 };
 typedef struct {
     int32_t run_bits;    /* must be 4 (Section 3.2: "Celty uses 4-bit RLC-CSC")                      */
     int32_t layout;      /* CELTY_LAYOUT_COLUMN or CELTY_LAYOUT_LANE_TILE                             */
-    int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: rows per tile, 1..2040, or 0 = choose      */
+    int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: rows per tile, 1..240, or 0 = choose       */
     int32_t reserved;    /* must be 0                                                                 */
 } celty_encode_opts;
 
@@ -206,11 +206,12 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *   grid     thread blocks per launch (rounded down to what fits the device at once)
  *   variant  LANE_TILE only: 0 = single fused launch (compaction + bulk-copy pipeline + reduction),
  *            1 = two launches (compaction kernel, then a kernel that loads straight from global memory)
- *   groups   fused kernel: warp groups per block working on different columns
- *   depth    fused kernel: bulk copies each warp keeps in flight (ring slots)
+ *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
+ *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
+ *   team     fused kernel: warps that share one sub-block and one accumulator (1, 2 or 4)
  * Errors: CELTY_EINVAL.
  */
-int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth);
+int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth, int32_t team);
 
 /* The cudaError_t of the last failing CUDA call made through this library (0 if none). */
 int celty_last_cuda_error(void);

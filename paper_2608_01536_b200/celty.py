@@ -38,7 +38,7 @@ SIGNATURES = {
     "celty_decode_device": (ctypes.c_int, [_vp, _i64, _vp, _vp, _i64, _vp, _vp]),
     "celty_fetched_bytes": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
     "celty_last_status": (ctypes.c_int, [_vp, _vp]),
-    "celty_set_launch": (ctypes.c_int, [_vp, _i32, _i32, _i32, _i32]),
+    "celty_set_launch": (ctypes.c_int, [_vp, _i32, _i32, _i32, _i32, _i32]),
     "celty_last_cuda_error": (ctypes.c_int, []),
     "celty_strerror": (ctypes.c_char_p, [ctypes.c_int]),
 }
@@ -162,8 +162,8 @@ class Matrix:
                "celty_fetched_bytes")
         return s.value, t.value
 
-    def set_launch(self, grid: int = 0, variant: int = 0, groups: int = 0, depth: int = 0):
-        _check(load().celty_set_launch(self._h, grid, variant, groups, depth), "celty_set_launch")
+    def set_launch(self, grid: int = 0, variant: int = 0, groups: int = 0, depth: int = 0, team: int = 0):
+        _check(load().celty_set_launch(self._h, grid, variant, groups, depth, team), "celty_set_launch")
 
     # ---------------------------------------------------------------- device side
     def to(self, device="cuda", stream=None):

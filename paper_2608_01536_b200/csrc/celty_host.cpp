@@ -95,7 +95,7 @@ void pack_lane_tile(celty_matrix *m, const Logical &lg)
                 G += (n + kGroup - 1) / kGroup;
             }
             size_t b = j * S + s;
-            off[b + 1] = off[b] + round_up(32 + (size_t)G * 20, 16);
+            off[b + 1] = off[b] + round_up(kSubHeader + (size_t)G * 20, 16);
             m->max_unit16 = std::max<uint32_t>(m->max_unit16, (uint32_t)((off[b + 1] - off[b]) / 16));
         }
     m->stream_bytes = round_up((size_t)off[K * S], kAlign);
@@ -120,7 +120,27 @@ void pack_lane_tile(celty_matrix *m, const Logical &lg)
                 G += g[L];
                 steps = std::max(steps, g[L]);
             }
-            uint8_t *vbase = sub + 32, *rbase = vbase + 16 * G;
+            // split points for up to four cooperating warps (see kSubHeader)
+            for (int k = 1; k <= 3; ++k) {
+                const uint64_t qk = (k * steps + 3) / 4;
+                uint64_t before = 0;
+                for (int L = 0; L < 32; ++L) {
+                    const uint64_t gq = std::min<uint64_t>(g[L], qk);        // groups of this lane before step q_k
+                    before += gq;
+                    uint64_t row = 0;                                          // rows those groups span
+                    for (uint64_t e = 0; e < std::min<uint64_t>(n[L], gq * kGroup); ++e) row += lg.runs[e0[L] + e] + 1;
+                    if (gq * kGroup > n[L]) row += gq * kGroup - n[L];         // zero-run slots that fill the last group
+                    sub[32 * k + L] = (uint8_t)row;
+                }
+                const uint16_t b16 = (uint16_t)before;
+                std::memcpy(sub + 128 + 2 * (k - 1), &b16, 2);
+            }
+            {
+                const uint16_t g16 = (uint16_t)G;
+                std::memcpy(sub + 134, &g16, 2);
+                sub[136] = (uint8_t)steps;
+            }
+            uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * G;
             uint64_t slot = 0;
             for (uint64_t q = 0; q < steps; ++q)
                 for (int L = 0; L < 32; ++L) {
@@ -145,7 +165,7 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
     if (o.run_bits != 4 || o.reserved != 0) return CELTY_EINVAL;
     if (o.layout != CELTY_LAYOUT_COLUMN && o.layout != CELTY_LAYOUT_LANE_TILE) return CELTY_EINVAL;
     if (o.layout == CELTY_LAYOUT_COLUMN && o.tile_rows != 0) return CELTY_EINVAL;
-    if (o.layout == CELTY_LAYOUT_LANE_TILE && (o.tile_rows < 0 || o.tile_rows > 2040)) return CELTY_EINVAL;
+    if (o.layout == CELTY_LAYOUT_LANE_TILE && (o.tile_rows < 0 || o.tile_rows > kMaxTileRows)) return CELTY_EINVAL;
     *out = nullptr;
     try {
         celty_matrix *m = new celty_matrix();
@@ -276,7 +296,7 @@ extern "C" int celty_decode_host(const celty_matrix *m, int64_t col, int32_t *ro
             const uint8_t *sub = stream + (size_t)meta[col * m->S + sl] * 16;
             int64_t G = 0;
             for (int L = 0; L < 32; ++L) G += sub[L];
-            const uint8_t *vbase = sub + 32, *rbase = vbase + 16 * G;
+            const uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * G;
             for (int L = 0; L < 32; ++L) {
                 const int64_t t = 32 * sl + L;
                 if (t >= T) break;
@@ -342,14 +362,17 @@ extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, in
     return CELTY_OK;
 }
 
-extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth)
+extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth,
+                                int32_t team)
 {
-    if (!m || grid < 0 || variant < 0 || variant > 7 || groups < 0 || groups > 32 || depth < 0 || depth > 16)
+    if (!m || grid < 0 || variant < 0 || variant > 1 || groups < 0 || groups > 15 || depth < 0 || depth > 16 ||
+        !(team == 0 || team == 1 || team == 2 || team == 4))
         return CELTY_EINVAL;
     m->grid = grid;
     m->variant = variant;
     m->groups = groups;
     m->depth = depth;
+    m->team = team;
     return CELTY_OK;
 }
 

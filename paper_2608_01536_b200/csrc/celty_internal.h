@@ -11,10 +11,19 @@ namespace celty {
 constexpr int kGroup = 8;            // entries per 16-byte value vector / 32-bit run word
 constexpr int kChunkGroups = 32;     // COLUMN layout: groups per warp-wide chunk (256 entries)
 constexpr int kTileSlack = 8;        // LANE_TILE: spare accumulator rows per slab for group-tail slots
+// LANE_TILE sub-block header (bytes), ahead of the value vectors and run words:
+//   [0,32)    groups of 8 entries that lane L's tile holds (u8)
+//   [32,128)  for k = 1,2,3: the lane's local row after its first q_k groups (u8 each), where
+//             q_k = ceil(k * steps / 4) and steps = the largest group count -- lets up to four warps
+//             start decoding the same sub-block at those steps without reading the runs before them
+//   [128,134) for k = 1,2,3: vectors stored before step q_k (u16)
+//   [134,136) vectors in the sub-block (u16);  [136] steps (u8);  rest zero
+constexpr int kSubHeader = 144;
+constexpr int kMaxTileRows = 240;    // keeps local rows (and the spare rows after them) in a byte
 constexpr int64_t kMaxM = 49152;     // accumulators of one thread block must fit shared memory
 constexpr size_t kAlign = 256;
 constexpr int kMaxBlocks = 192;      // blocks of the fused kernel the workspace has partial vectors for
-constexpr int kSlabsPerBlock = 4;    // LANE_TILE: a thread block covers at most this many slabs of rows
+constexpr int kSlabsPerBlock = 8;    // LANE_TILE: a thread block covers at most this many slabs of rows
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -66,5 +75,5 @@ struct celty_matrix {
     uint8_t *d_image = nullptr;
     uint8_t *d_ws = nullptr;
     celty::WorkspaceLayout ws{};
-    int32_t grid = 0, variant = 0, groups = 0, depth = 0;
+    int32_t grid = 0, variant = 0, groups = 0, depth = 0, team = 0;
 };

@@ -287,7 +287,7 @@ k_spmspv_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ str
         const uint32_t gl = sub[lane];
         const uint32_t steps = __reduce_max_sync(kFull, gl);
         const uint32_t Gs = __reduce_add_sync(kFull, gl);
-        const uint8_t *vbase = sub + 32, *rbase = vbase + 16 * (size_t)Gs;
+        const uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * (size_t)Gs;
         uint32_t slot0 = 0, row = 0;
         for (uint32_t q = 0; q < steps; ++q) {
             const bool active = gl > q;
@@ -330,7 +330,7 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
     const uint32_t gl = sub[lane];
     const uint32_t steps = __reduce_max_sync(kFull, gl);
     const uint32_t Gs = __reduce_add_sync(kFull, gl);
-    const uint8_t *vbase = sub + 32, *rbase = vbase + 16 * (size_t)Gs;
+    const uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * (size_t)Gs;
     const int t = 32 * s + lane;
     const uint32_t out0 = t < T ? scratch[t] - scratch[0] : 0u;
     const uint32_t nt = t < T ? scratch[t + 1] - scratch[t] : 0u;
@@ -382,28 +382,41 @@ int launch_compact(const void *x, int64_t K, float tau, int32_t *idx, uint16_t *
     return CELTY_OK;
 }
 
-// Shape of the fused launch: P row parts of Sc slabs, G warp groups, D ring slots per warp.
+// Shape of the fused launch: P row parts of Sc slabs, G groups (teams = G * Sc, one accumulator slab and one
+// ring of D slots each), W warps per team.
 int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
 {
     FusedPlan pl{};
     pl.P = m->P;
     pl.Sc = m->Sc;
+    if (pl.Sc > 15) return CELTY_EINVAL;      // one hardware named barrier per team
     pl.slot_bytes = (int)round_up((size_t)m->max_unit16 * 16, 128);
     pl.cap = 64;
     const size_t budget = (size_t)di.max_smem_optin;
-    const int g_max = std::max(1, std::min(16 / pl.Sc, m->groups > 0 ? m->groups : std::max(1, 8 / pl.Sc)));
-    const int d_want = m->depth > 0 ? m->depth : 3;
+    // Warps per team: measurements on B200 show no gain from sharing a sub-block between warps at the
+    // configured sizes, so one warp per team unless asked otherwise.  Groups first (each needs its own
+    // accumulator), then as many ring slots as still fit (at least two, to keep a copy in flight).
+    pl.W = m->team > 0 ? m->team : 1;
+    while (pl.W > 1 && pl.Sc * pl.W > 16) pl.W >>= 1;       // a requested team size that does not fit is reduced
+    if (pl.Sc * pl.W > 16) return CELTY_EINVAL;
+    const int g_cap = std::min(15 / pl.Sc, std::max(1, 16 / (pl.Sc * pl.W)));
+    const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
+    const int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 4;
     pl.G = 0;
-    for (int d = d_want; d >= 1 && pl.G == 0; --d)
-        for (int g = g_max; g >= 1; --g)
+    for (int g = g_max; g >= 1 && pl.G == 0; --g)
+        for (int d = d_max; d >= d_min; --d)
             if (fused_smem_bytes(m->R, (int)m->K, g, pl.Sc, d, pl.slot_bytes, pl.cap) <= budget) {
-                // prefer keeping two copies in flight over a wider block
-                if (d >= 2 || g == 1 || d_want == 1) { pl.G = g; pl.D = d; break; }
+                pl.G = g;
+                pl.D = d;
+                break;
             }
+    if (pl.G == 0 && m->depth == 0 && fused_smem_bytes(m->R, (int)m->K, 1, pl.Sc, 1, pl.slot_bytes, pl.cap) <= budget) {
+        pl.G = 1;
+        pl.D = 1;
+    }
     if (pl.G == 0) return CELTY_EINVAL;
-    // streaming warps first; with variant bit 2 the block is filled up to 512 threads with warps that
-    // only help with the data-parallel phases
-    pl.threads = (m->variant & 4) ? std::max(512, 32 * pl.G * pl.Sc) : 32 * pl.G * pl.Sc;
+    pl.threads = std::max(512, 32 * pl.G * pl.Sc * pl.W);
+    if (pl.threads > 512) return CELTY_EINVAL;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
@@ -465,7 +478,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
     uint16_t *val = reinterpret_cast<uint16_t *>(m->d_ws + m->ws.val_off);
     float *y = static_cast<float *>(y_dev);
     const uint8_t *stream_base = m->d_image + m->meta_bytes;
-    if (m->layout == CELTY_LAYOUT_LANE_TILE && (m->variant & 1) == 0) {
+    if (m->layout == CELTY_LAYOUT_LANE_TILE && m->variant == 0) {
         FusedPlan plan;
         rc = plan_fused(m, di, &plan);
         if (rc) return rc;
@@ -481,10 +494,9 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
         fp.partials = reinterpret_cast<float *>(m->d_ws + m->ws.partial_off);
         fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.T = (int)m->T;
-        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D;
+        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.W = plan.W;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         fp.stream_bytes = (long long)m->stream_bytes;
-        fp.flags = (m->variant & 2) ? 1 : 0;
         k_spmspv_fused<<<plan.grid, plan.threads, plan.smem, st>>>(fp);
         CELTY_CUDA(cudaGetLastError());
         return CELTY_OK;

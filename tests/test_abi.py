@@ -46,7 +46,7 @@ def test_argument_errors(lib):
     with pytest.raises(celty.CeltyError):
         celty.Matrix(W, layout=7)
     with pytest.raises(celty.CeltyError):
-        celty.Matrix(W, layout=celty.LAYOUT_LANE_TILE, tile_rows=4000)
+        celty.Matrix(W, layout=celty.LAYOUT_LANE_TILE, tile_rows=241)
     h = ctypes.c_void_p()
     assert lib.celty_encode(None, 4, None, 4, 4, None, ctypes.byref(h)) == -1
     assert lib.celty_encode(W.ctypes.data_as(ctypes.c_void_p), 4, None, 0, 4, None, ctypes.byref(h)) == -1

@@ -148,8 +148,8 @@ def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows):
     x = synth.integer_activations(M + K, K)
     tau = synth.threshold_for_density(x, d_a)
     m = _matrix(W, mask, layout, tile_rows)
-    for grid, groups, depth in ((0, 0, 0), (1, 0, 0), (3, 1, 1), (37, 3, 2), (148, 2, 4)):
-        m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth)
+    for grid, groups, depth, team in ((0, 0, 0, 0), (1, 0, 0, 1), (3, 1, 1, 4), (37, 3, 2, 2), (148, 2, 4, 1)):
+        m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth, team=team)
         y = _run(m, x, tau)
         _check_y(y, W, mask, x, tau, exact=True)
 
