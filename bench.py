@@ -39,6 +39,13 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_spmspv_fused launch, from the ncu captures
+# summarised under profiles/ (small-case captures of the same kernel and workload).
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "llama7b_attn_4096x4096_s50_a50": 11.33e6,
+    "llama70b_mlp_28672x8192_s50_a50": 165.7e6,
+}
+
 
 def make_layer(name: str, variant: int):
     M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
@@ -333,6 +340,7 @@ def run_celty(args):
             dist.destroy_process_group()
         return
     peak, peak_src = measured_peaks()
+    launches_per_step = 1 if (layout == celty.LAYOUT_LANE_TILE and args.variant == 0) else 2
     out = {
         "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": sec_per_call * 1e3, "us_per_call": sec_per_call * 1e6,
@@ -348,11 +356,12 @@ def run_celty(args):
         "bytes_per_call": {"entry_stream": stream_bytes, "total": total_bytes, "dense_fp16": 2.0 * M * K,
                            "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad},
         "roofline": {"bound": "hbm", "achieved": total_bytes / sec_per_call / 1e9, "peak": peak, "unit": "GB/s",
-                     "frac": total_bytes / sec_per_call / 1e9 / peak, "traffic": None, "peak_source": peak_src,
-                     "note": "time per call covers every kernel of the call"},
+                     "frac": total_bytes / sec_per_call / 1e9 / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(name),
+                     "peak_source": peak_src, "kernel": "k_spmspv_fused" if launches_per_step == 1 else "all kernels of the call",
+                     "note": "one launch per call: algorithmic bytes per call / CUDA-event time per call"},
         "e2e": {"value": world * total_bytes / e2e_sec / 1e9, "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
                 "h2d_bytes_per_step": 2 * K, "d2h_bytes_per_step": 4 * M},
-        "gpu_launches": (1 if (layout == celty.LAYOUT_LANE_TILE and args.variant == 0) else 2) * args.steps,
+        "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks.summary(),
         "context": {"us_per_call_stream_enqueued": us_enqueued, "us_per_call_l2_warm": us_warm,
                     "cublas_gemv_fp16_us": dense_us,
