@@ -118,6 +118,23 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Largest `value` over all ranks of the default process group (the value itself without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(bytes_per_call_per_rank: float, world: int, seconds_per_call: float) -> float:
+    """Replicas only: every rank processes its own calls, so the job moves world x the bytes in the
+    (max-over-ranks) time of one call.  GB/s."""
+    return world * bytes_per_call_per_rank / seconds_per_call / 1e9
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -270,13 +287,9 @@ def run_celty(args):
         timed_region()
         e1.record()
         barrier()
-    ms = e0.elapsed_time(e1)
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
     sec_per_call = ms / 1e3 / args.steps
-    gbs = world * total_bytes / sec_per_call / 1e9
+    gbs = aggregate_throughput(total_bytes, world, sec_per_call)
 
     # ---- stream-enqueued (no graph) and L2-warm numbers, for context
     def time_calls(fn, n):
@@ -312,11 +325,7 @@ def run_celty(args):
         c = i % copies
         mats[c].spmspv_host(xh[c], taus[c], yh, xstage, ys[0])
     barrier()
-    e2e_sec = (time.perf_counter() - t0) / n_e2e
-    t = torch.tensor([e2e_sec], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_sec = float(t.item())
+    e2e_sec = max_over_ranks((time.perf_counter() - t0) / n_e2e, dev)
 
     # ---- dense cuBLAS GEMV on the same GPU, same rotation (context, not the target)
     dense_us = None
@@ -359,7 +368,7 @@ def run_celty(args):
                      "frac": total_bytes / sec_per_call / 1e9 / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(name),
                      "peak_source": peak_src, "kernel": "k_spmspv_fused" if launches_per_step == 1 else "all kernels of the call",
                      "note": "one launch per call: algorithmic bytes per call / CUDA-event time per call"},
-        "e2e": {"value": world * total_bytes / e2e_sec / 1e9, "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
+        "e2e": {"value": aggregate_throughput(total_bytes, world, e2e_sec), "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
                 "h2d_bytes_per_step": 2 * K, "d2h_bytes_per_step": 4 * M},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks.summary(),
