@@ -39,7 +39,8 @@ typedef enum {
     CELTY_ECUDA = -3,      /* a CUDA runtime call failed; celty_last_cuda_error() returns its code */
     CELTY_ESTATE = -4,     /* handle not bound to device memory yet */
     CELTY_ETIMEOUT = -5,   /* device status word: a bounded wait inside a kernel ran out */
-    CELTY_EBOUNDS = -6     /* device status word: a decoded row or list index was out of range */
+    CELTY_EBOUNDS = -6,    /* device status word: a decoded row or list index was out of range */
+    CELTY_ELIMIT = -7      /* a size exceeds the fixed scratch of celty_spmspv_static */
 } celty_status;
 
 /* Device-image layouts.  Both hold exactly the (value, 4-bit run) entries that Section 3.2
@@ -166,6 +167,37 @@ int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, cel
  */
 int celty_spmspv_host(celty_matrix *m, const void *x_host, float tau, void *y_host, void *x_stage_dev,
                       void *y_stage_dev, celty_stream_t stream);
+
+/*
+ * celty_spmspv_static -- the same product for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Some callers of this library run where cudaMalloc is not available to them: inside a stream
+ * capture, under a memory pool that owns every byte of the device, in a plugin whose host forbids
+ * allocations on its inference path.  celty_spmspv needs a caller-provided workspace for its
+ * scratch (the compacted activation list); this variant keeps that scratch in a fixed array that
+ * is part of the library image instead, so the caller passes only inputs and outputs:
+ *   m          a LANE_TILE handle (host side only is used: sizes and table offsets)
+ *   image_dev  the packed image on the device (image_bytes of celty_device_bytes; the caller
+ *              copied celty_host_image there, or it is the buffer given to celty_bind_device)
+ *   x_dev      K FP16 (device, 16-byte aligned), not modified
+ *   y_dev      M FP32 (device, 16-byte aligned), overwritten
+ * It runs the two-launch path (thresholding/compaction kernel, then the lane-tile SpMSpV kernel
+ * that loads straight from global memory and merges with atomic adds) and calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ * Limit: K <= 32768 (the scratch array holds 196 864 bytes: a header, int32 indices and FP16 values
+ * for that many columns; every GPU that loads the library carries it until the process exits);
+ * larger K returns CELTY_ELIMIT.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current); make that first call before any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's contents; nothing in it
+ * has to start at zero (count and list are rewritten by every call), but two calls that overlap on
+ * the GPU (different streams, or one stream of another thread) race on it: serialise them.
+ * Errors: CELTY_EINVAL (null, misaligned, tau < 0 or not finite, COLUMN-layout handle), CELTY_ELIMIT,
+ * CELTY_ECUDA.
+ */
+int celty_spmspv_static(const celty_matrix *m, const void *image_dev, const void *x_dev, float tau, void *y_dev,
+                        celty_stream_t stream);
 
 /*
  * celty_last_compaction -- device pointers into the handle's workspace holding the list the last

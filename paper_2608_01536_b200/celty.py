@@ -33,6 +33,7 @@ SIGNATURES = {
     "celty_bind_device": (ctypes.c_int, [_vp, _vp, _sz, _vp, _sz, _vp]),
     "celty_compact": (ctypes.c_int, [_vp, _i64, _f32, _vp, _vp, _vp, _vp]),
     "celty_spmspv": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp]),
+    "celty_spmspv_static": (ctypes.c_int, [_vp, _vp, _vp, _f32, _vp, _vp]),
     "celty_spmspv_host": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp, _vp]),
     "celty_last_compaction": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
     "celty_decode_device": (ctypes.c_int, [_vp, _i64, _vp, _vp, _i64, _vp, _vp]),
@@ -186,6 +187,19 @@ class Matrix:
         assert x.dtype == torch.float16 and x.numel() == self.K and x.is_contiguous()
         assert y.dtype == torch.float32 and y.numel() == self.M and y.is_contiguous()
         _check(load().celty_spmspv(self._h, x.data_ptr(), tau, y.data_ptr(), _stream_ptr(stream)), "celty_spmspv")
+        return y
+
+    def spmspv_static(self, x, tau: float, y=None, stream=None):
+        """Same product through the entry point that needs no workspace: its scratch is a fixed array inside
+        the library, for callers that cannot allocate device memory.  K <= 32768; calls that overlap on the
+        GPU race on that array.  The matrix's packed image must be on the device (`to()`)."""
+        import torch
+        if y is None:
+            y = torch.empty(self.M, dtype=torch.float32, device=x.device)
+        assert x.dtype == torch.float16 and x.numel() == self.K and x.is_contiguous()
+        assert y.dtype == torch.float32 and y.numel() == self.M and y.is_contiguous()
+        _check(load().celty_spmspv_static(self._h, self._image.data_ptr(), x.data_ptr(), tau, y.data_ptr(),
+                                          _stream_ptr(stream)), "celty_spmspv_static")
         return y
 
     def spmspv_host(self, x_host, tau: float, y_host, x_stage, y_stage, stream=None):

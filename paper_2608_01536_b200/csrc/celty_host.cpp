@@ -386,6 +386,7 @@ extern "C" const char *celty_strerror(int status)
         case CELTY_ESTATE: return "handle is not bound to device memory";
         case CELTY_ETIMEOUT: return "a bounded wait inside a kernel ran out";
         case CELTY_EBOUNDS: return "a decoded index was out of range";
+        case CELTY_ELIMIT: return "size exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

@@ -531,6 +531,76 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
     return CELTY_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// celty_spmspv_static: scratch in a file-scope device array instead of a caller-provided workspace,
+// for callers that cannot allocate device memory.  Layout of the array: [256 B header: status, count]
+// [int32 idx[kStaticMaxK]][uint16 val[kStaticMaxK]].
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t kStaticMaxK = 32768;
+constexpr size_t kStaticScratchBytes = 256 + (size_t)kStaticMaxK * 4 + (size_t)kStaticMaxK * 2;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code the array's name is only a stand-in: the device address comes from the runtime, once
+// per device, with that device current.
+int static_scratch_address(uint8_t **out)
+{
+    static std::mutex mu;
+    static uint8_t *address[64];
+    int dev = 0;
+    CELTY_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CELTY_EINVAL;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!address[dev]) {
+        void *p = nullptr;
+        CELTY_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        address[dev] = static_cast<uint8_t *>(p);
+    }
+    *out = address[dev];
+    return CELTY_OK;
+}
+
+}  // namespace
+
+extern "C" int celty_spmspv_static(const celty_matrix *m, const void *image_dev, const void *x_dev, float tau,
+                                   void *y_dev, celty_stream_t stream)
+{
+    if (!m || !image_dev || !x_dev || !y_dev) return CELTY_EINVAL;
+    if (!(tau >= 0.f) || !std::isfinite(tau)) return CELTY_EINVAL;
+    if (((uintptr_t)x_dev | (uintptr_t)y_dev | (uintptr_t)image_dev) & 15) return CELTY_EINVAL;
+    if (m->layout != CELTY_LAYOUT_LANE_TILE) return CELTY_EINVAL;
+    if (m->K > kStaticMaxK) return CELTY_ELIMIT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    uint8_t *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    int32_t *count = reinterpret_cast<int32_t *>(scratch) + 1;
+    int32_t *idx = reinterpret_cast<int32_t *>(scratch + 256);
+    uint16_t *val = reinterpret_cast<uint16_t *>(scratch + 256 + (size_t)kStaticMaxK * 4);
+    float *y = static_cast<float *>(y_dev);
+    rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);     // also clears y
+    if (rc) return rc;
+    const size_t group_bytes = (size_t)m->S * (m->R + kTileSlack) * 32 * 4;
+    if (group_bytes > (size_t)di.max_smem_optin || m->S > 32) return CELTY_ELIMIT;
+    const int G = (int)std::max<size_t>(1, std::min<size_t>((size_t)di.max_smem_optin / group_bytes,
+                                                             (size_t)std::max<int64_t>(1, 8 / m->S)));
+    const size_t smem = group_bytes * G;
+    static int granted[64];
+    rc = ensure_smem(k_spmspv_lane, smem, granted);
+    if (rc) return rc;
+    const uint8_t *image = static_cast<const uint8_t *>(image_dev);
+    k_spmspv_lane<<<di.sms, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(image),
+                                                            image + m->meta_bytes, idx, val, count, y, (int)m->M, m->R,
+                                                            (int)m->S, (int)m->T, G);
+    CELTY_CUDA(cudaGetLastError());
+    return CELTY_OK;
+}
+
 extern "C" int celty_spmspv_host(celty_matrix *m, const void *x_host, float tau, void *y_host, void *x_stage_dev,
                                  void *y_stage_dev, celty_stream_t stream)
 {
