@@ -201,6 +201,93 @@ def run_reference(args):
     }))
 
 
+# ----------------------------------------------------------------------------- sweeps (documentation runs)
+SWEEPS = {
+    # config 2: 4096 x 4096, magnitude-pruned, all 9 (weight sparsity, activation density) pairs
+    "cfg2": [dict(M=4096, K=4096, s=s, family="magnitude", dist="laplace", d_a=d, cfg=2)
+             for s in (0.3, 0.5, 0.7) for d in (0.7, 0.5, 0.3)],
+    # config 3: Llama-2-7B MLP shapes
+    "cfg3": [dict(M=11008, K=4096, s=0.5, family="magnitude", dist="laplace", d_a=0.5, cfg=3),
+             dict(M=4096, K=11008, s=0.5, family="magnitude", dist="swiglu", d_a=0.5, cfg=3)],
+    # config 4: the three shapes of a Llama-2-13B decode layer (q/k/v/o, gate/up, down)
+    "cfg4": [dict(M=5120, K=5120, s=0.5, family="bernoulli", dist="laplace", d_a=0.4, cfg=4),
+             dict(M=13824, K=5120, s=0.5, family="bernoulli", dist="laplace", d_a=0.4, cfg=4),
+             dict(M=5120, K=13824, s=0.5, family="bernoulli", dist="laplace", d_a=0.4, cfg=4)],
+    # config 5: Llama-70B-shaped MLP, sparsity x density x mask family
+    "cfg5": [dict(M=M, K=K, s=s, family=f, dist="laplace", d_a=d, cfg=5)
+             for (M, K) in ((28672, 8192), (8192, 28672)) for f in ("bernoulli", "powerlaw")
+             for s in (0.3, 0.5, 0.7) for d in (0.1, 0.3, 0.5, 0.7)],
+}
+
+
+def run_sweep(args):
+    """Times every point of one configured sweep, one call at a time with the L2 flushed before each call
+    (a 256 MB memset), CUDA events around the call; the dense cuBLAS GEMV is timed the same way."""
+    import torch
+    from paper_2608_01536_b200 import build as lib_build, celty
+    lib_build.build()
+    celty.load()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    reps = args.sweep_reps
+
+    def timed(fn):
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return float(np.median(ts)), float(np.min(ts))
+
+    points, cache_W, cache_m = [], {}, {}
+    for i, pt in enumerate(SWEEPS[args.sweep]):
+        M, K, s, fam = pt["M"], pt["K"], pt["s"], pt["family"]
+        seed = synth.point_seed(pt["cfg"], 0)
+        if (M, K) not in cache_W:
+            cache_W.clear()
+            cache_m.clear()
+            cache_W[(M, K)] = synth.weights(seed, M, K)
+        W = cache_W[(M, K)]
+        if (s, fam) not in cache_m:
+            cache_m.clear()                                    # one encoded matrix on the device at a time
+            mask = (synth.mask_magnitude(W, s) if fam == "magnitude" else
+                    synth.mask_bernoulli(seed, M, K, 1.0 - s) if fam == "bernoulli" else
+                    synth.mask_powerlaw(seed, M, K, 1.0 - s))
+            m = celty.Matrix(W, mask, device=dev)
+            Wd = torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev)
+            cache_m[(s, fam)] = (m, Wd)
+            del mask
+        m, Wd = cache_m[(s, fam)]
+        x = synth.activations(synth.point_seed(pt["cfg"], 50 + i), K, pt["dist"])
+        tau = synth.threshold_for_density(x, pt["d_a"])
+        xd = torch.from_numpy(x).to(dev)
+        y = torch.empty(M, dtype=torch.float32, device=dev)
+        yd = torch.empty(M, dtype=torch.float16, device=dev)
+        for _ in range(3):
+            m.spmspv(xd, tau, y)
+            torch.mv(Wd, xd, out=yd)
+        idx, _ = m.last_compaction()
+        assert m.last_status() == 0
+        sb, tb = m.fetched_bytes(idx.cpu().numpy())
+        us, us_min = timed(lambda: m.spmspv(xd, tau, y))
+        dus, dus_min = timed(lambda: torch.mv(Wd, xd, out=yd))
+        info = m.info()
+        points.append({"M": M, "K": K, "weight_sparsity": s, "mask": fam, "activation_density": pt["d_a"],
+                       "survivors": int(idx.numel()), "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad,
+                       "fetched_bytes": tb, "us_per_call": us, "us_min": us_min, "GBps": tb / us / 1e3,
+                       "roofline_frac": tb / us / 1e3 / peak, "cublas_gemv_us": dus,
+                       "speedup_vs_cublas": dus / us, "combined_sparsity": 1.0 - (1.0 - s) * pt["d_a"]})
+        print(json.dumps(points[-1]), file=sys.stderr, flush=True)
+    print(json.dumps({"sweep": args.sweep, "protocol": "one call at a time, 256 MB memset before each call, CUDA events, "
+                      f"median of {reps}", "peak_GBps": peak, "points": points}))
+
+
 def run_celty(args):
     import torch
     import torch.distributed as dist
@@ -408,8 +495,12 @@ def main():
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS), help="time every point of a configured sweep")
+    ap.add_argument("--sweep-reps", type=int, default=30)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_celty(args)

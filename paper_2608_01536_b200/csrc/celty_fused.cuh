@@ -128,7 +128,8 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
 // Barrier among the 32 * nwarps threads of one team (hardware named barrier `id`, 1..15).
 __device__ __forceinline__ void team_sync(int id, int nthreads)
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+    if (nthreads == 32) __syncwarp();
+    else asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 // One lane's work on a range of steps of a sub-block, as a three-stage software pipeline (a step =
@@ -172,7 +173,8 @@ __device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t
 {
     uint32_t even, odd, total;
     decode_group(b.w, even, odd, total);
-    // cell address = cell + 128 * offset byte: one dot-product-accumulate per entry
+    // cell address = cell + 128 * offset byte: one dot-product-accumulate per entry (measured faster on
+    // B200 than a byte permute followed by a multiply-add)
     b.a[0] = __dp4a(even, 0x00000080u, cell);
     b.a[1] = __dp4a(odd, 0x00000080u, cell);
     b.a[2] = __dp4a(even, 0x00008000u, cell);
@@ -269,11 +271,13 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
 
     CELTY_MARK(0);
-    // The sub-block offsets are needed right after the ranks are known: start pulling the table into L2 now.
+    // The sub-block offsets are needed right after the ranks are known: start pulling the table into L2
+    // now, each block its own share of the lines (L2 is shared by all blocks).
     {
-        const size_t meta_bytes = ((size_t)p.K * p.S + 1) * 4;
-        for (size_t o = (size_t)tid * 128; o < meta_bytes; o += (size_t)nthreads * 128)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + o));
+        const size_t lines = (((size_t)p.K * p.S + 1) * 4 + 127) / 128;
+        const size_t per = (lines + gridDim.x - 1) / gridDim.x, l0 = (size_t)blockIdx.x * per;
+        for (size_t l = l0 + tid; l < min(lines, l0 + per); l += nthreads)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + l * 128));
     }
     // ---- a1: threshold all of x; byte q of the keep words = keep bits of activations 8q .. 8q+7.
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
@@ -308,6 +312,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             kb[q] = (uint8_t)keep;
         }
     }
+    CELTY_MARK(10);
     // clear the accumulators while those loads are in flight
     {
         float4 *acc4 = reinterpret_cast<float4 *>(acc);
@@ -352,8 +357,15 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
         const uint32_t bar0 = smem_u32(&bars[team * p.D]);
         const uint32_t lt_mask = (1u << lane) - 1u;
+        const uint32_t items0 = smem_u32(items);
         uint32_t issued = 0, consumed = 0;                            // ring positions of this team
         bool failed = false;
+        long long dbg_wait = 0, dbg_head = 0, dbg_loop = 0, dbg_tail = 0, dbg_steps = 0;   // development builds
+        (void)dbg_wait; (void)dbg_head; (void)dbg_loop; (void)dbg_tail; (void)dbg_steps;
+        StepBuf b0, b1;                                               // pipeline registers, live across items
+        b0.v = make_uint4(0, 0, 0, 0); b0.w = 0; b1.v = b0.v; b1.w = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { b0.c[e] = 0.f; b1.c[e] = 0.f; }
 
         for (int rb = r_begin; rb < r_end; rb += p.cap) {
             const int cnt = min(p.cap, r_end - rb);
@@ -403,25 +415,27 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             CELTY_MARK(3);
             for (int i = 0; i < cnt; ++i) {
                 const uint32_t slot = consumed % (uint32_t)p.D, parity = (consumed / (uint32_t)p.D) & 1u;
+                const long long t_a = CELTY_CLOCK();
                 // A warp that gave up on a copy keeps walking the items (and the team barriers) without
                 // touching them, so that the warps of a team never wait for one another in vain.
                 if (!failed && !mbar_wait_bounded(bar0 + 8u * slot, parity)) failed = true;
                 failed = __any_sync(kFull, failed);
                 if (i == 0) CELTY_MARK(4);
+                const long long t_b = CELTY_CLOCK();
                 ++consumed;
                 if (failed) {
                     team_sync(bar_id, team_threads);
                     continue;
                 }
                 const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
-                const float xj = __half2float(__ushort_as_half((uint16_t)items[i].y));
+                uint32_t xbits;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(items0 + 8u * (uint32_t)i + 4u));
+                const float xj = __half2float(__ushort_as_half((uint16_t)xbits));
                 // ---- a3 + a4.  Header: groups per lane, split points, totals (see kSubHeader).
-                uint32_t gl, hw0, hw1, hw2;
+                uint32_t gl, hw;
                 asm volatile("ld.shared.u8 %0, [%1];" : "=r"(gl) : "r"(sub + lane));
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw0) : "r"(sub + 128));     // cum1 | cum2 << 16
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw1) : "r"(sub + 132));     // cum3 | vectors << 16
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw2) : "r"(sub + 136));     // steps
-                const uint32_t steps = hw2 & 0xFFu, Gs = hw1 >> 16;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw) : "r"(sub + 136));      // vectors | steps << 16
+                const uint32_t steps = hw >> 16, Gs = hw & 0xFFFFu;
                 const uint32_t vbase = sub + kSubHeader, rbase = vbase + 16 * Gs;
                 const uint32_t slot_end = sub + (uint32_t)p.slot_bytes;
                 // this warp's range of steps [q_lo, q_hi), its first vector and its lanes' first rows
@@ -432,15 +446,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                     q_lo = (k_lo * steps + 3) >> 2;
                     q_hi = k_hi >= 4 ? steps : (k_hi * steps + 3) >> 2;
                     if (k_lo) {
-                        cum = k_lo == 1 ? (hw0 & 0xFFFFu) : k_lo == 2 ? (hw0 >> 16) : (hw1 & 0xFFFFu);
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(cum) : "r"(sub + 126 + 2 * k_lo));
                         asm volatile("ld.shared.u8 %0, [%1];" : "=r"(row0) : "r"(sub + 32 * k_lo + lane));
                     }
                 }
                 uint32_t cell = cell0 + row0 * 128u;
-                StepBuf b0, b1;
-                b0.v = make_uint4(0, 0, 0, 0); b0.w = 0; b1.v = b0.v; b1.w = 0;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) { b0.c[e] = 0.f; b1.c[e] = 0.f; }
+                const long long t_c = CELTY_CLOCK();
                 step_fetch(b0, gl, q_lo, q_hi, cum, lt_mask, vbase, rbase, slot_end);
                 step_fetch(b1, gl, q_lo + 1, q_hi, cum, lt_mask, vbase, rbase, slot_end);
                 step_decode(b0, cell, slab0, slab_end);                                    // step q_lo
@@ -453,14 +464,18 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                     step_finish(b1, xj);                                                   // step q
                     step_fetch(b0, gl, q + 3, q_hi, cum, lt_mask, vbase, rbase, slot_end);
                 }
+                const long long t_d = CELTY_CLOCK();
                 // every warp of the team is done with this sub-block (and with its rows) before the
                 // slot is refilled and before anybody touches the accumulator for the next column
                 team_sync(bar_id, team_threads);
-                if (member == 0 && lane == 0 && i + p.D < cnt && !failed) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    issue(i + p.D);
-                }
+                // The slot's contents were consumed by loads whose values have been used, and the barrier
+                // above orders every team member's reads before this point: the copy may overwrite it.
+                if (member == 0 && lane == 0 && i + p.D < cnt && !failed) issue(i + p.D);
+                dbg_wait += t_b - t_a; dbg_head += t_c - t_b; dbg_loop += t_d - t_c; dbg_tail += CELTY_CLOCK() - t_d;
+                dbg_steps += q_hi - q_lo;
             }
+            CELTY_STORE(11, dbg_wait); CELTY_STORE(12, dbg_head); CELTY_STORE(13, dbg_loop); CELTY_STORE(14, dbg_tail);
+            CELTY_STORE(15, dbg_steps);
             issued = __shfl_sync(kFull, issued, 0);
             team_sync(bar_id, team_threads);                      // items / imeta are rewritten by the next batch
         }

@@ -2,7 +2,6 @@
 // host-side decoding for round-trip tests and byte accounting.  No CUDA calls in this file.
 #include <algorithm>
 #include <cmath>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -32,12 +31,15 @@ struct Logical {                 // one run per byte, block-major (column, tile)
 
 int choose_tile_rows(int64_t M)
 {
-    // about 128 rows per lane keeps a lane's run stream at ~8 groups per column at 50% density;
-    // slabs of 32 lanes then cover M with at most one partly filled slab.
+    // About 128 rows per lane keeps a lane's run stream at ~8 groups per column at 50% density.  Slabs of
+    // 32 lanes then cover M; when a column needs more slabs than one thread block takes, the slab count is
+    // rounded up to a multiple of the number of row parts so that every part gets the same number.
     int64_t S = std::max<int64_t>(1, (M + 2048) / 4096);
+    const int64_t P = (S + kSlabsPerBlock - 1) / kSlabsPerBlock;
+    S = (S + P - 1) / P * P;
     int64_t R = (M + 32 * S - 1) / (32 * S);
-    R = (R + 3) / 4 * 4;                       // keeps 16-byte vector stores of y aligned
-    return (int)std::max<int64_t>(4, R);
+    R = (R + 3) / 4 * 4;                       // keeps 16-byte vector accesses of a tile aligned
+    return (int)std::min<int64_t>(kMaxTileRows, std::max<int64_t>(4, R));
 }
 
 // Build the COLUMN image: meta uint2[K] {off16, entries}, then per column its chunks of up to 32
@@ -136,9 +138,8 @@ void pack_lane_tile(celty_matrix *m, const Logical &lg)
                 std::memcpy(sub + 128 + 2 * (k - 1), &b16, 2);
             }
             {
-                const uint16_t g16 = (uint16_t)G;
-                std::memcpy(sub + 134, &g16, 2);
-                sub[136] = (uint8_t)steps;
+                const uint32_t gs = (uint32_t)G | ((uint32_t)steps << 16);
+                std::memcpy(sub + 136, &gs, 4);
             }
             uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * G;
             uint64_t slot = 0;
@@ -227,9 +228,7 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
                 }
         }
         if (m->layout == CELTY_LAYOUT_COLUMN) pack_column(m, lg); else pack_lane_tile(m, lg);
-        int spb = kSlabsPerBlock;
-        if (const char *e = std::getenv("CELTY_SLABS_PER_BLOCK")) spb = std::max(1, std::atoi(e));
-        m->P = (int32_t)((m->S + spb - 1) / spb);
+        m->P = (int32_t)((m->S + kSlabsPerBlock - 1) / kSlabsPerBlock);
         m->Sc = (int32_t)((m->S + m->P - 1) / m->P);
         m->ws = workspace_layout(K, T, m->layout == CELTY_LAYOUT_LANE_TILE ? (int64_t)m->Sc * m->R * 32 : 0);
         *out = m;

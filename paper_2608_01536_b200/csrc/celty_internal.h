@@ -17,13 +17,13 @@ constexpr int kTileSlack = 8;        // LANE_TILE: spare accumulator rows per sl
 //             q_k = ceil(k * steps / 4) and steps = the largest group count -- lets up to four warps
 //             start decoding the same sub-block at those steps without reading the runs before them
 //   [128,134) for k = 1,2,3: vectors stored before step q_k (u16)
-//   [134,136) vectors in the sub-block (u16);  [136] steps (u8);  rest zero
+//   [136,140) vectors in the sub-block | steps << 16 (u32);  rest zero
 constexpr int kSubHeader = 144;
 constexpr int kMaxTileRows = 240;    // keeps local rows (and the spare rows after them) in a byte
 constexpr int64_t kMaxM = 49152;     // accumulators of one thread block must fit shared memory
 constexpr size_t kAlign = 256;
 constexpr int kMaxBlocks = 192;      // blocks of the fused kernel the workspace has partial vectors for
-constexpr int kSlabsPerBlock = 8;    // LANE_TILE: a thread block covers at most this many slabs of rows
+constexpr int kSlabsPerBlock = 4;    // LANE_TILE: a thread block covers at most this many slabs of rows
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
