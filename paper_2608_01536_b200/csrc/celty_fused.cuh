@@ -37,6 +37,7 @@ struct FusedParams {
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // items a team looks up per batch
+    int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row tiles into y
 };
 
 constexpr uint32_t kSpinLimit = 1u << 21;
@@ -116,6 +117,15 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
+}
+
+// Polling load that goes to L2 every time but carries no ordering (and so leaves the L1 of the other
+// warps alone); the caller fences once after the value it waits for has shown up.
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -271,6 +281,20 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
 
     CELTY_MARK(0);
+    uint32_t y_ticket = 0;
+    // Bulk reduce-add merge: the adds at the end need a cleared y.  The last warp clears this block's share
+    // and announces it right away, so that the fence and the ticket overlap the loads of a1.
+    if (p.merge == 1 && warp == nwarps - 1) {
+        const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
+        for (int i = r0 + lane; i < r1; i += 32) p.y[i] = 0.f;
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence();
+            // The ticket counts modulo 2 * gridDim.x, so it never has to be reset: calls alternate between
+            // waiting for the lower and for the upper half.
+            y_ticket = atomicInc(&p.tickets[0], 2u * gridDim.x - 1u);
+        }
+    }
     // The sub-block offsets are needed right after the ranks are known: start pulling the table into L2
     // now, each block its own share of the lines (L2 is shared by all blocks).
     {
@@ -490,86 +514,142 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     __syncthreads();
     CELTY_MARK(5);
 
-    // ---- a5, stage 1: add the G accumulators, store the block's partial (accumulator layout, no slack rows)
-    const int tile_words = p.R * 32, part_words = p.Sc * tile_words;
-    {
-        float4 *mine4 = reinterpret_cast<float4 *>(p.partials + (size_t)blockIdx.x * part_words);
-        const float4 *acc4 = reinterpret_cast<const float4 *>(acc);
-        const int tile4 = tile_words >> 2, slab4 = slab_words >> 2, group4 = p.Sc * slab4;
-        for (int fsl = 0; fsl < p.Sc; ++fsl)
-            for (int q4 = tid; q4 < tile4; q4 += nthreads) {
-                const float4 *src = acc4 + fsl * slab4 + q4;
-                float4 v = src[0];
-                for (int gg = 1; gg < p.G; ++gg) {
-                    const float4 t = src[gg * group4];
-                    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
-                }
-                __stcg(mine4 + fsl * tile4 + q4, v);
+    if (p.merge == 1) {
+        // ---- a5 by bulk reduce-add: the block adds its G accumulators, transposes each lane's tile into a
+        // row-major staging tile (stride R + 4 words keeps tiles 16-byte aligned and the stores 4-way
+        // conflicted at worst), and the copy engine adds every tile into y (cp.reduce.async.bulk, FP32 add at
+        // L2).  y was cleared by all blocks at the start; the ticket makes sure of it.
+        if (warp == nwarps - 1 && lane == 0) {                      // every block's share of y is cleared by now
+            const bool low_half = y_ticket < gridDim.x;
+            bool ok = false;
+            for (uint32_t it = 0; it < kSpinLimit; ++it) {
+                const uint32_t cur = ld_relaxed_u32(&p.tickets[0]);
+                if (low_half ? (cur >= gridDim.x) : (cur < gridDim.x)) { ok = true; break; }
+                __nanosleep(64);
             }
-    }
-    __syncthreads();
-    CELTY_MARK(6);
-    if (tid == 0) {
-        __threadfence();                                          // the block's stores, ordered by the barrier above
-        atomicAdd(&p.tickets[0], 1u);
-        bool ok = false;
-        for (uint32_t it = 0; it < kSpinLimit; ++it) {
-            if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
-            __nanosleep(32);
+            __threadfence();
+            if (!ok) atomicOr(p.status, kStatusTimeout);
         }
-        if (!ok) atomicOr(p.status, kStatusTimeout);
-    }
-    __syncthreads();
-    CELTY_MARK(7);
+        const int tstride = p.R + 4;
+        float *stage = reinterpret_cast<float *>(smem + lay.ring);
+        const int group_words = p.Sc * slab_words;
+        for (int fsl = 0; fsl < p.Sc; ++fsl) {
+            const float *src = acc + (size_t)fsl * slab_words + lane;
+            float *dst = stage + (size_t)(fsl * 32 + lane) * tstride;
+            for (int i = 2 * warp; i < p.R; i += 2 * nwarps) {      // two rows per pass: all loads first
+                float v0 = 0.f, v1 = 0.f;
+                const bool two = i + 1 < p.R;
+                for (int gg = 0; gg < p.G; ++gg) {
+                    v0 += src[(size_t)gg * group_words + i * 32];
+                    if (two) v1 += src[(size_t)gg * group_words + (i + 1) * 32];
+                }
+                dst[i] = v0;
+                if (two) dst[i + 1] = v1;
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        CELTY_MARK(6);
+        if (tid < p.Sc * 32) {
+            const int fsl = tid >> 5, t = 32 * (part * p.Sc + fsl) + lane;
+            if (t < p.T) {
+                const int row0 = t * p.R, nrows = min(p.R, p.M - row0);
+                const uint32_t bytes = ((uint32_t)nrows * 4u) & ~15u;
+                const float *src = stage + (size_t)(fsl * 32 + lane) * tstride;
+                if (bytes)
+                    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(p.y + row0),
+                                 "r"(smem_u32(src)), "r"(bytes)
+                                 : "memory");
+                for (int i = (int)(bytes >> 2); i < nrows; ++i)
+                    if (src[i] != 0.f) atomicAdd(p.y + row0 + i, src[i]);
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging may go once it has been read
+        }
+        CELTY_MARK(7);
+    } else {
+        // ---- a5, stage 1: add the G accumulators, store the block's partial (accumulator layout, no slack rows)
+        const int tile_words = p.R * 32, part_words = p.Sc * tile_words;
+        {
+            float4 *mine4 = reinterpret_cast<float4 *>(p.partials + (size_t)blockIdx.x * part_words);
+            const float4 *acc4 = reinterpret_cast<const float4 *>(acc);
+            const int tile4 = tile_words >> 2, slab4 = slab_words >> 2, group4 = p.Sc * slab4;
+            for (int fsl = 0; fsl < p.Sc; ++fsl)
+                for (int q4 = tid; q4 < tile4; q4 += nthreads) {
+                    const float4 *src = acc4 + fsl * slab4 + q4;
+                    float4 v = src[0];
+                    for (int gg = 1; gg < p.G; ++gg) {
+                        const float4 t = src[gg * group4];
+                        v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+                    }
+                    __stcg(mine4 + fsl * tile4 + q4, v);
+                }
+        }
+        __syncthreads();
+        CELTY_MARK(6);
+        if (tid == 0) {
+            __threadfence();                                          // the block's stores, ordered by the barrier above
+            atomicAdd(&p.tickets[0], 1u);
+            bool ok = false;
+            for (uint32_t it = 0; it < kSpinLimit; ++it) {
+                if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
+                __nanosleep(32);
+            }
+            if (!ok) atomicOr(p.status, kStatusTimeout);
+        }
+        __syncthreads();
+        CELTY_MARK(7);
 
-    // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
-    // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
-    // every lane has up to 8 loads in flight, then the ranges are added in a fixed order.
-    {
-        float *red = reinterpret_cast<float *>(smem + lay.acc);   // the accumulators are no longer needed
-        const int wpc = (((part_words + nK - 1) / nK) + 31) & ~31;
-        const int wb = kslice * wpc, we = min(part_words, wb + wpc);
-        const int nchunks = max(0, (we - wb + 31) >> 5);
-        const size_t stride = (size_t)p.P * part_words;
-        for (int c0 = 0; c0 < nchunks; c0 += nwarps) {
-            const int pass_chunks = min(nwarps, nchunks - c0);
-            const int nsplit = nwarps / pass_chunks;              // warps per chunk in this pass
-            const int my_chunk = warp % pass_chunks, my_split = warp / pass_chunks;
-            const int word = wb + 32 * (c0 + my_chunk) + lane;
-            if (my_split < nsplit) {
-                float sum = 0.f;
-                if (word < we) {
-                    const int per = (nK + nsplit - 1) / nsplit;
-                    const int b_lo = my_split * per, b_hi = min(nK, b_lo + per);
-                    const float *src = p.partials + (size_t)part * part_words + word;
-                    for (int b0 = b_lo; b0 < b_hi; b0 += 8) {
-                        float t[8];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            t[k] = (b0 + k < b_hi && CELTY_CHECK((size_t)(b0 + k) * stride + (size_t)part * part_words + word <
-                                                                     (size_t)gridDim.x * part_words, 13, b0 + k))
-                                       ? __ldcg(src + (size_t)(b0 + k) * stride) : 0.f;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) sum += t[k];
+        // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
+        // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
+        // every lane has up to 16 loads in flight, then the ranges are added in a fixed order.
+        {
+            float *red = reinterpret_cast<float *>(smem + lay.acc);   // the accumulators are no longer needed
+            const int wpc = (((part_words + nK - 1) / nK) + 31) & ~31;
+            const int wb = kslice * wpc, we = min(part_words, wb + wpc);
+            const int nchunks = max(0, (we - wb + 31) >> 5);
+            const size_t stride = (size_t)p.P * part_words;
+            for (int c0 = 0; c0 < nchunks; c0 += nwarps) {
+                const int pass_chunks = min(nwarps, nchunks - c0);
+                const int nsplit = nwarps / pass_chunks;              // warps per chunk in this pass
+                const int my_chunk = warp % pass_chunks, my_split = warp / pass_chunks;
+                const int word = wb + 32 * (c0 + my_chunk) + lane;
+                if (my_split < nsplit) {
+                    float sum = 0.f;
+                    if (word < we) {
+                        const int per = (nK + nsplit - 1) / nsplit;
+                        const int b_lo = my_split * per, b_hi = min(nK, b_lo + per);
+                        const float *src = p.partials + (size_t)part * part_words + word;
+                        for (int b0 = b_lo; b0 < b_hi; b0 += 16) {
+                            float t[16];
+    #pragma unroll
+                            for (int k = 0; k < 16; ++k)
+                                t[k] = (b0 + k < b_hi && CELTY_CHECK((size_t)(b0 + k) * stride + (size_t)part * part_words + word <
+                                                                         (size_t)gridDim.x * part_words, 13, b0 + k))
+                                           ? __ldcg(src + (size_t)(b0 + k) * stride) : 0.f;
+    #pragma unroll
+                            for (int k = 0; k < 16; ++k) sum += t[k];
+                        }
+                    }
+                    red[(my_split * pass_chunks + my_chunk) * 32 + lane] = sum;
+                }
+                __syncthreads();
+                if (warp < pass_chunks) {
+                    const int w2 = wb + 32 * (c0 + warp) + lane;
+                    if (w2 < we) {
+                        float total = 0.f;
+                        for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
+                        const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
+                        const int i = rem >> 5, t = 32 * (part * p.Sc + fsl) + (rem & 31), row = t * p.R + i;
+                        if (t < p.T && row < p.M) p.y[row] = total;
                     }
                 }
-                red[(my_split * pass_chunks + my_chunk) * 32 + lane] = sum;
+                __syncthreads();
             }
-            __syncthreads();
-            if (warp < pass_chunks) {
-                const int w2 = wb + 32 * (c0 + warp) + lane;
-                if (w2 < we) {
-                    float total = 0.f;
-                    for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
-                    const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
-                    const int i = rem >> 5, t = 32 * (part * p.Sc + fsl) + (rem & 31), row = t * p.R + i;
-                    if (t < p.T && row < p.M) p.y[row] = total;
-                }
-            }
-            __syncthreads();
         }
     }
     CELTY_MARK(8);
+    if (p.merge == 1) return;
     __syncthreads();
     if (tid == 0) {
         const uint32_t t = atomicAdd(&p.tickets[1], 1u);
@@ -582,7 +662,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 }
 
 struct FusedPlan {
-    int G, Sc, P, D, W, slot_bytes, cap, threads, grid;
+    int G, Sc, P, D, W, slot_bytes, cap, threads, grid, merge;
     size_t smem;
 };
 

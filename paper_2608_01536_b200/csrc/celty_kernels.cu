@@ -418,6 +418,10 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     pl.threads = std::max(512, 32 * pl.G * pl.Sc * pl.W);
     if (pl.threads > 512) return CELTY_EINVAL;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
+    // bulk reduce-add merge: its staging tiles reuse the ring area and must fit there
+    pl.merge = (m->merge >= 0 ? m->merge : 1);
+    if ((size_t)pl.Sc * 32 * (m->R + 4) * 4 > (size_t)pl.G * pl.Sc * pl.D * pl.slot_bytes) pl.merge = 0;
+    if (m->R % 4) pl.merge = 0;                // tiles of y and of the staging area must start on 16 bytes
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
     pl.grid = std::max(1, blocks / pl.P) * pl.P;
@@ -497,6 +501,13 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.W = plan.W;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         fp.stream_bytes = (long long)m->stream_bytes;
+        fp.merge = plan.merge;
+        // the tickets count blocks of one launch shape: start them over when the shape changes
+        if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
+            CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
+            m->last_grid = plan.grid;
+            m->last_merge = plan.merge;
+        }
         k_spmspv_fused<<<plan.grid, plan.threads, plan.smem, st>>>(fp);
         CELTY_CUDA(cudaGetLastError());
         return CELTY_OK;
@@ -661,6 +672,7 @@ extern "C" int celty_last_status(celty_matrix *m, celty_stream_t stream)
         CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off, 0, 4, st));
         CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
         CELTY_CUDA(cudaStreamSynchronize(st));
+        m->last_grid = 0;
     }
     if (word & kStatusTimeout) return CELTY_ETIMEOUT;
     if (word & kStatusBounds) return CELTY_EBOUNDS;
