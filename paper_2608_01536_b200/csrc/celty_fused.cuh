@@ -37,6 +37,7 @@ struct FusedParams {
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // items a team looks up per batch
+    int producer;              // 1: the last warp issues every team's bulk copies (needs an idle warp)
     int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row tiles into y
 };
 
@@ -100,6 +101,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 // Wait for a phase of an mbarrier with an iteration limit; false = gave up.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 {
@@ -158,8 +164,20 @@ struct StepBuf {
     uint32_t fin;       // ... of the decoded step
     uint32_t a[8];      // cell addresses of the decoded step
     float c[8];         // accumulator values loaded for the decoded step
-    float f[8];         // its 8 weights in FP32
+    uint4 h;            // its 8 weights (FP16 pairs)
 };
+
+// d = a * x + c with FP16 a (both halves of `pair`) and x, FP32 c and d: the product of two FP16 numbers
+// is exact in FP32, so this rounds once, exactly like converting to FP32 and calling fmaf.
+__device__ __forceinline__ void fma_pair(uint32_t pair, uint16_t x, float c0, float c1, float &d0, float &d1)
+{
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "mov.b32 {lo, hi}, %2;\n\t"
+        "fma.rn.f32.f16 %0, lo, %3, %4;\n\t"
+        "fma.rn.f32.f16 %1, hi, %3, %5;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "r"(pair), "h"(x), "f"(c0), "f"(c1));
+}
 
 __device__ __forceinline__ void step_fetch(StepBuf &b, uint32_t gl, uint32_t q, uint32_t q_end, uint32_t &cum,
                                            uint32_t lt_mask, uint32_t vbase, uint32_t rbase, uint32_t slot_end)
@@ -211,16 +229,16 @@ __device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t
         : "+f"(b.c[0]), "+f"(b.c[1]), "+f"(b.c[2]), "+f"(b.c[3]), "+f"(b.c[4]), "+f"(b.c[5]), "+f"(b.c[6]), "+f"(b.c[7])
         : "r"(b.a[0]), "r"(b.a[1]), "r"(b.a[2]), "r"(b.a[3]), "r"(b.a[4]), "r"(b.a[5]), "r"(b.a[6]), "r"(b.a[7]),
           "r"(b.fin));
-    const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&b.v.x));
-    const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&b.v.y));
-    const float2 f45 = __half22float2(*reinterpret_cast<const __half2 *>(&b.v.z));
-    const float2 f67 = __half22float2(*reinterpret_cast<const __half2 *>(&b.v.w));
-    b.f[0] = f01.x; b.f[1] = f01.y; b.f[2] = f23.x; b.f[3] = f23.y;
-    b.f[4] = f45.x; b.f[5] = f45.y; b.f[6] = f67.x; b.f[7] = f67.y;
+    b.h = b.v;
 }
 
-__device__ __forceinline__ void step_finish(const StepBuf &b, float xj)
+__device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 {
+    float d[8];
+    fma_pair(b.h.x, xj, b.c[0], b.c[1], d[0], d[1]);
+    fma_pair(b.h.y, xj, b.c[2], b.c[3], d[2], d[3]);
+    fma_pair(b.h.z, xj, b.c[4], b.c[5], d[4], d[5]);
+    fma_pair(b.h.w, xj, b.c[6], b.c[7], d[6], d[7]);
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.u32 p, %16, 0;\n\t"
@@ -230,16 +248,14 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, float xj)
         "@p st.shared.f32 [%6], %14;\n\t@p st.shared.f32 [%7], %15;\n\t}"
         :
         : "r"(b.a[0]), "r"(b.a[1]), "r"(b.a[2]), "r"(b.a[3]), "r"(b.a[4]), "r"(b.a[5]), "r"(b.a[6]), "r"(b.a[7]),
-          "f"(fmaf(b.f[0], xj, b.c[0])), "f"(fmaf(b.f[1], xj, b.c[1])), "f"(fmaf(b.f[2], xj, b.c[2])),
-          "f"(fmaf(b.f[3], xj, b.c[3])), "f"(fmaf(b.f[4], xj, b.c[4])), "f"(fmaf(b.f[5], xj, b.c[5])),
-          "f"(fmaf(b.f[6], xj, b.c[6])), "f"(fmaf(b.f[7], xj, b.c[7])), "r"(b.fin)
+          "f"(d[0]), "f"(d[1]), "f"(d[2]), "f"(d[3]), "f"(d[4]), "f"(d[5]), "f"(d[6]), "f"(d[7]), "r"(b.fin)
         : "memory");
 }
 
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, items, imeta, lane_base, keep, total;
+    size_t acc, ring, bars, empty, mail, items, imeta, lane_base, keep, total;
 };
 
 __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
@@ -248,7 +264,9 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     size_t off = 0;
     l.acc = off;       off += (size_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
     l.ring = off;      off += (size_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
-    l.bars = off;      off += (size_t)teams * D * 8;                       // one mbarrier per slot
+    l.bars = off;      off += (size_t)teams * D * 8;                       // one "full" mbarrier per slot
+    l.empty = off;     off += (size_t)teams * D * 8;                       // one "empty" mbarrier per slot (producer warp)
+    l.mail = off;      off += (size_t)teams * 16;                          // per team: batch sequence, batch size, done
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
     l.lane_base = off; off += 256;                                         // rank of each lane's first survivor, n
@@ -271,6 +289,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
+    uint64_t *empties = reinterpret_cast<uint64_t *>(smem + lay.empty);
+    volatile int *mail = reinterpret_cast<volatile int *>(smem + lay.mail);   // [team][4]: seq, cnt, done, -
     int2 *items = reinterpret_cast<int2 *>(smem + lay.items) + (size_t)team * p.cap;      // [cap] {column, x bits}
     uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
     int *lane_base = reinterpret_cast<int *>(smem + lay.lane_base);                       // [32] + [32] = n
@@ -344,6 +364,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     }
     if (streams && member == 0 && lane == 0) {
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
+        for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&empties[team * p.D + d]), (uint32_t)p.W);
+        mail[team * 4 + 0] = 0; mail[team * 4 + 1] = 0; mail[team * 4 + 2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -379,7 +401,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
         const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
         const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
-        const uint32_t bar0 = smem_u32(&bars[team * p.D]);
+        const uint32_t bar0 = smem_u32(&bars[team * p.D]), emp0 = smem_u32(&empties[team * p.D]);
+        int batch_seq = 0;
         const uint32_t lt_mask = (1u << lane) - 1u;
         const uint32_t items0 = smem_u32(items);
         uint32_t issued = 0, consumed = 0;                            // ring positions of this team
@@ -387,7 +410,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         long long dbg_wait = 0, dbg_head = 0, dbg_loop = 0, dbg_tail = 0, dbg_steps = 0;   // development builds
         (void)dbg_wait; (void)dbg_head; (void)dbg_loop; (void)dbg_tail; (void)dbg_steps;
         StepBuf b0, b1;                                               // pipeline registers, live across items
-        b0.v = make_uint4(0, 0, 0, 0); b0.w = 0; b1.v = b0.v; b1.w = 0;
+        b0.v = make_uint4(0, 0, 0, 0); b0.w = 0; b1.v = b0.v; b1.w = 0; b0.h = b0.v; b1.h = b0.v;
 #pragma unroll
         for (int e = 0; e < 8; ++e) { b0.c[e] = 0.f; b1.c[e] = 0.f; }
 
@@ -426,7 +449,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             }
             team_sync(bar_id, team_threads);
             if (s >= p.S) continue;
-            // ---- a2: keep D copies in flight (issued by lane 0 of the team's first warp)
+            if (p.producer && member == 0 && lane == 0) {           // hand the batch to the producer warp
+                mail[team * 4 + 1] = cnt;
+                __threadfence_block();
+                mail[team * 4 + 0] = ++batch_seq;
+            }
+            // ---- a2: keep D copies in flight (issued by lane 0 of the team's first warp, or by the producer warp)
             auto issue = [&](int i) {
                 const uint32_t slot = issued % (uint32_t)p.D;
                 const uint2 im = imeta[i];
@@ -434,7 +462,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 bulk_load(ring0 + slot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y, bar0 + 8u * slot);
                 ++issued;
             };
-            if (member == 0 && lane == 0 && !failed)
+            if (!p.producer && member == 0 && lane == 0 && !failed)
                 for (int i = 0; i < min(cnt, p.D); ++i) issue(i);
             CELTY_MARK(3);
             for (int i = 0; i < cnt; ++i) {
@@ -449,12 +477,13 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 ++consumed;
                 if (failed) {
                     team_sync(bar_id, team_threads);
+                    if (p.producer && lane == 0) mbar_arrive(emp0 + 8u * slot);
                     continue;
                 }
                 const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
                 uint32_t xbits;
                 asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(items0 + 8u * (uint32_t)i + 4u));
-                const float xj = __half2float(__ushort_as_half((uint16_t)xbits));
+                const uint16_t xj = (uint16_t)xbits;
                 // ---- a3 + a4.  Header: groups per lane, split points, totals (see kSubHeader).
                 uint32_t gl, hw;
                 asm volatile("ld.shared.u8 %0, [%1];" : "=r"(gl) : "r"(sub + lane));
@@ -494,7 +523,11 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 team_sync(bar_id, team_threads);
                 // The slot's contents were consumed by loads whose values have been used, and the barrier
                 // above orders every team member's reads before this point: the copy may overwrite it.
-                if (member == 0 && lane == 0 && i + p.D < cnt && !failed) issue(i + p.D);
+                if (p.producer) {
+                    if (lane == 0) mbar_arrive(emp0 + 8u * slot);  // one arrival per warp of the team frees the slot
+                } else if (member == 0 && lane == 0 && i + p.D < cnt && !failed) {
+                    issue(i + p.D);
+                }
                 dbg_wait += t_b - t_a; dbg_head += t_c - t_b; dbg_loop += t_d - t_c; dbg_tail += CELTY_CLOCK() - t_d;
                 dbg_steps += q_hi - q_lo;
             }
@@ -503,13 +536,51 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             issued = __shfl_sync(kFull, issued, 0);
             team_sync(bar_id, team_threads);                      // items / imeta are rewritten by the next batch
         }
+        if (p.producer && member == 0 && lane == 0) mail[team * 4 + 2] = 1;      // no more batches from this team
         if (failed) {
             // give copies that are still in flight a last (bounded) chance to land before the block exits
-            if (member == 0)
+            if (member == 0 && !p.producer)
                 for (; consumed < issued; ++consumed)
                     mbar_wait_bounded(bar0 + 8u * (consumed % (uint32_t)p.D), (consumed / (uint32_t)p.D) & 1u);
             if (lane == 0) atomicOr(p.status, kStatusTimeout);
         }
+    }
+    else if (p.producer && warp == nwarps - 1 && lane < teams) {
+        // ---- producer: lane t issues team t's bulk copies, in order, as its ring slots are handed back
+        const int t = lane;
+        const uint32_t pbar0 = smem_u32(&bars[t * p.D]), pemp0 = smem_u32(&empties[t * p.D]);
+        const uint32_t pring0 = smem_u32(ring + (size_t)t * p.D * p.slot_bytes);
+        const uint2 *pim = reinterpret_cast<const uint2 *>(smem + lay.imeta) + (size_t)t * p.cap;
+        int seq_seen = 0, next = 0, cnt = 0;
+        uint32_t pos = 0;
+        bool done = false;
+        for (uint32_t it = 0; it < 4u * kSpinLimit && !done; ++it) {
+            if (next == cnt) {                                      // look for the team's next batch
+                const int sq = mail[t * 4 + 0];
+                if (sq != seq_seen) {
+                    __threadfence_block();
+                    cnt = mail[t * 4 + 1];
+                    next = 0;
+                    seq_seen = sq;
+                } else if (mail[t * 4 + 2] && mail[t * 4 + 0] == seq_seen) {
+                    done = true;
+                } else {
+                    __nanosleep(64);
+                }
+                continue;
+            }
+            const uint32_t slot = pos % (uint32_t)p.D, use = pos / (uint32_t)p.D;
+            if (use > 0 && !mbar_try_wait(pemp0 + 8u * slot, (use - 1u) & 1u)) {
+                __nanosleep(32);
+                continue;
+            }
+            const uint2 im = pim[next];
+            mbar_expect_tx(pbar0 + 8u * slot, im.y);
+            bulk_load(pring0 + slot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y, pbar0 + 8u * slot);
+            ++pos;
+            ++next;
+        }
+        if (!done) atomicOr(p.status, kStatusTimeout);
     }
     __syncthreads();
     CELTY_MARK(5);
@@ -662,7 +733,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 }
 
 struct FusedPlan {
-    int G, Sc, P, D, W, slot_bytes, cap, threads, grid, merge;
+    int G, Sc, P, D, W, slot_bytes, cap, threads, grid, merge, producer;
     size_t smem;
 };
 

@@ -418,6 +418,8 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     pl.threads = std::max(512, 32 * pl.G * pl.Sc * pl.W);
     if (pl.threads > 512) return CELTY_EINVAL;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
+    // a warp that does not stream can issue all the bulk copies (variant bit 3 turns that off)
+    pl.producer = (32 * pl.G * pl.Sc * pl.W < pl.threads && !m->no_producer) ? 1 : 0;
     // bulk reduce-add merge: its staging tiles reuse the ring area and must fit there
     pl.merge = (m->merge >= 0 ? m->merge : 1);
     if ((size_t)pl.Sc * 32 * (m->R + 4) * 4 > (size_t)pl.G * pl.Sc * pl.D * pl.slot_bytes) pl.merge = 0;
@@ -502,6 +504,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
+        fp.producer = plan.producer;
         // the tickets count blocks of one launch shape: start them over when the shape changes
         if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
             CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
