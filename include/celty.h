@@ -48,17 +48,26 @@ typedef enum {
  *   CELTY_LAYOUT_COLUMN     tile_rows must be 0: runs are counted along the whole column.
  *                           A warp decodes 256 consecutive entries at a time with the intra-warp
  *                           prefix sum of Algorithm 1 and scatters with shared-memory atomics.
- *   CELTY_LAYOUT_LANE_TILE  tile_rows = R > 0: the rule of Section 3.2 is applied separately to
- *                           consecutive tiles of R rows (the row partition of Section 3.1 taken
- *                           down to one tile per lane).  Lane L of a warp owns tile 32*s + L, so
- *                           every lane writes its own shared-memory bank: no conflicts, no atomics.
+ *   CELTY_LAYOUT_LANE_TILE  tile_rows = R > 0: the rows are partitioned into tiles of R rows (the
+ *                           row partition of Section 3.1 taken down to one tile per lane) and the
+ *                           rule of Section 3.2 is applied to every tile separately.  Lane L of the
+ *                           warp that works on slab s owns tile 32*s + L, so every lane writes its
+ *                           own shared-memory bank: no conflicts, no atomics.  A tile is not a block
+ *                           of consecutive rows: rows are dealt out like cards, row r to lane r mod 32
+ *                           and every group of 32 rows, C groups at a time, to the S slabs in turn
+ *                           (celty_row_map gives S, R and C):
+ *                               row(s, L, i) = (((i / C) * S + s) * C + i mod C) * 32 + L
+ *                           is local row i (0 <= i < R) of tile 32*s + L; values >= M do not exist.
+ *                           Within a tile the rows grow with i, and "dropped rows since the previous
+ *                           entry" counts local rows.  Every lane and every slab thus samples the
+ *                           whole height of the matrix, whatever the row-wise density profile.
  */
 enum { CELTY_LAYOUT_COLUMN = 0, CELTY_LAYOUT_LANE_TILE = 1 };
 
 typedef struct {
     int32_t run_bits;    /* must be 4 (Section 3.2: "Celty uses 4-bit RLC-CSC")                      */
     int32_t layout;      /* CELTY_LAYOUT_COLUMN or CELTY_LAYOUT_LANE_TILE                             */
-    int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: rows per tile, 1..240, or 0 = choose       */
+    int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: local rows per tile, 1..240, or 0 = choose */
     int32_t reserved;    /* must be 0                                                                 */
 } celty_encode_opts;
 
@@ -94,9 +103,18 @@ int celty_info(const celty_matrix *m, int64_t *M, int64_t *K, int64_t *nnz, int6
                int64_t *compressed_bytes, int32_t *layout, int32_t *tile_rows);
 
 /*
+ * celty_row_map -- the parameters of the LANE_TILE row map (see CELTY_LAYOUT_LANE_TILE): slabs S of
+ * 32 tiles, local rows per tile R, chunk C.  The paper partitions rows into contiguous tiles
+ * (Section 3.1); this library's tiles are the interleaved row sets given above.  For a COLUMN handle
+ * the answer is S = 1, R = M, C = 1 (the single tile is the column).  Output pointers may be NULL.
+ */
+int celty_row_map(const celty_matrix *m, int32_t *slabs, int32_t *tile_rows, int32_t *chunk);
+
+/*
  * celty_decode_host -- the stored entries of column `col`, decoded on the host from the handle's
  * own packed image (round-trip tests): absolute row (Algorithm 1: prefix sum of runs + ordinal),
- * FP16 bit pattern, run and pad flag of each entry, row tiles concatenated in ascending order.
+ * FP16 bit pattern, run and pad flag of each entry, row tiles concatenated in ascending tile order
+ * (LANE_TILE: tile 32*s + L, its entries by ascending local row).
  * cap = capacity of the output arrays (entries); *n receives the entry count even when it exceeds
  * cap (then nothing is written and CELTY_ENOMEM is returned).  Output pointers may be NULL.
  */
@@ -236,8 +254,12 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
 /*
  * celty_set_launch -- tuning knobs for experiments and tests; 0 = the library's choice.
  *   grid     thread blocks per launch (rounded down to what fits the device at once)
- *   variant  LANE_TILE only: 0 = single fused launch (compaction + bulk-copy pipeline + reduction),
- *            1 = two launches (compaction kernel, then a kernel that loads straight from global memory)
+ *   variant  LANE_TILE only, a sum of: 1 = two launches (compaction kernel, then a kernel that loads
+ *            straight from global memory) instead of the single fused launch; for the fused launch
+ *            2 = merge the blocks' results through per-block partial vectors summed in a fixed
+ *            order (bit-reproducible) instead of adding them into y with bulk reduce-add copies,
+ *            4 = force the bulk reduce-add merge, 8 = every warp team issues its own bulk copies
+ *            instead of leaving that to an idle warp
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   team     fused kernel: warps that share one sub-block and one accumulator (1, 2 or 4)

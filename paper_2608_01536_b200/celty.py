@@ -27,6 +27,7 @@ SIGNATURES = {
     "celty_encode": (ctypes.c_int, [_vp, _i64, _vp, _i64, _i64, _vp, ctypes.POINTER(_vp)]),
     "celty_destroy": (None, [_vp]),
     "celty_info": (ctypes.c_int, [_vp] + [ctypes.POINTER(_i64)] * 5 + [ctypes.POINTER(_i32)] * 2),
+    "celty_row_map": (ctypes.c_int, [_vp] + [ctypes.POINTER(_i32)] * 3),
     "celty_decode_host": (ctypes.c_int, [_vp, _i64, _vp, _vp, _vp, _vp, _i64, ctypes.POINTER(_i64)]),
     "celty_host_image": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
     "celty_device_bytes": (ctypes.c_int, [_vp, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
@@ -129,6 +130,12 @@ class Matrix:
         _check(load().celty_info(self._h, *[ctypes.byref(a) for a in v + w]), "celty_info")
         return SimpleNamespace(M=v[0].value, K=v[1].value, nnz=v[2].value, n_pad=v[3].value,
                                compressed_bytes=v[4].value, layout=w[0].value, tile_rows=w[1].value)
+
+    def row_map(self):
+        """(slabs S, local rows per tile R, chunk C) of the LANE_TILE row map."""
+        w = [_i32() for _ in range(3)]
+        _check(load().celty_row_map(self._h, *[ctypes.byref(a) for a in w]), "celty_row_map")
+        return w[0].value, w[1].value, w[2].value
 
     def host_image(self):
         """(uint8 copy of the packed image, offset of the entry stream in it)."""

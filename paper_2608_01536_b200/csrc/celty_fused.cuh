@@ -32,7 +32,7 @@ struct FusedParams {
     uint32_t *status;
     uint32_t *tickets;         // [0] partial stored, [1] departed
     float *partials;           // gridDim.x vectors of Sc * R * 32 floats (accumulator layout)
-    int M, K, R, S, T;
+    int M, K, R, S, C;         // rows, columns, local rows per tile, slabs, chunk of the row map (tile_row)
     int G, Sc, P, D, W;        // groups, slabs per block, row parts, ring depth, warps per team (1, 2 or 4)
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
@@ -151,21 +151,35 @@ __device__ __forceinline__ void team_sync(int id, int nthreads)
 // One lane's work on a range of steps of a sub-block, as a three-stage software pipeline (a step =
 // one group of 8 entries of every lane that still has one):
 //   fetch(q+2)   128-bit value vector + 32-bit run word from the ring slot
-//   decode(q)    run-length decode on packed bytes, cell addresses, FP16 -> FP32; the 8 accumulator
-//                loads are issued here ...
-//   finish(q-1)  ... and consumed one step later: fmaf + store.
+//   decode(q)    run-length decode on packed bytes, cell addresses; the 8 accumulator loads are
+//                issued here ...
+//   finish(q-1)  ... and consumed one step later: multiply-add + store.
 // Rows of one lane only grow within a column, so the cells of different steps never coincide and the
-// loads of step q may overtake the stores of step q-1.  Every shared-memory access of a lane that has
-// no group in a step is predicated off.
+// loads of step q may overtake the stores of step q-1.
+// Nothing is predicated: a lane without a group in a step fetches an all-zero group (zero values, zero
+// runs) from a zero block instead and adds 0 to the 8 spare rows at the end of its tile (its own bank;
+// no real entry lives there, so it does not matter who else does the same at the same time).  Such a
+// lane has no group in any later step of the item either, so its running row is dead from then on.
 struct StepBuf {
     uint4 v;            // fetched values
     uint32_t w;         // fetched runs
-    uint32_t act;       // this lane has a group in the step (fetched, then kept for finish)
-    uint32_t fin;       // ... of the decoded step
+    bool act;           // this lane has a group in the fetched step
     uint32_t a[8];      // cell addresses of the decoded step
     float c[8];         // accumulator values loaded for the decoded step
     uint4 h;            // its 8 weights (FP16 pairs)
 };
+
+__device__ __forceinline__ float lds_f32(uint32_t a)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+    return v;
+}
+
+__device__ __forceinline__ void sts_f32(uint32_t a, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
 
 // d = a * x + c with FP16 a (both halves of `pair`) and x, FP32 c and d: the product of two FP16 numbers
 // is exact in FP32, so this rounds once, exactly like converting to FP32 and calling fmaf.
@@ -180,27 +194,27 @@ __device__ __forceinline__ void fma_pair(uint32_t pair, uint16_t x, float c0, fl
 }
 
 __device__ __forceinline__ void step_fetch(StepBuf &b, uint32_t gl, uint32_t q, uint32_t q_end, uint32_t &cum,
-                                           uint32_t lt_mask, uint32_t vbase, uint32_t rbase, uint32_t slot_end)
+                                           uint32_t lt_mask, uint32_t vbase, uint32_t rbase, uint32_t slot_end,
+                                           uint32_t zeros)
 {
-    const bool act = gl > q && q < q_end;
+    bool act = gl > q && q < q_end;
     const uint32_t bal = __ballot_sync(kFull, act);
     const uint32_t k = cum + __popc(bal & lt_mask);
     cum += __popc(bal);
-    b.act = (act && CELTY_CHECK(vbase + 16 * k + 16 <= slot_end && rbase + 4 * k + 4 <= slot_end, 1, k)) ? 1u : 0u;
+    if (!CELTY_CHECK(!act || (vbase + 16 * k + 16 <= slot_end && rbase + 4 * k + 4 <= slot_end), 1, k)) act = false;
     (void)slot_end;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.u32 p, %5, 0;\n\t"
-        "@p ld.shared.v4.u32 {%0, %1, %2, %3}, [%6];\n\t"
-        "@p ld.shared.u32 %4, [%7];\n\t}"
-        : "+r"(b.v.x), "+r"(b.v.y), "+r"(b.v.z), "+r"(b.v.w), "+r"(b.w)
-        : "r"(b.act), "r"(vbase + 16 * k), "r"(rbase + 4 * k));
+    b.act = act;
+    const uint32_t va = act ? vbase + 16 * k : zeros, ra = act ? rbase + 4 * k : zeros;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(b.v.x), "=r"(b.v.y), "=r"(b.v.z), "=r"(b.v.w) : "r"(va));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(b.w) : "r"(ra));
 }
 
-__device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t slab_begin, uint32_t slab_end)
+__device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t spare, uint32_t slab_begin,
+                                            uint32_t slab_end)
 {
     uint32_t even, odd, total;
     decode_group(b.w, even, odd, total);
+    cell = b.act ? cell : spare;
     // cell address = cell + 128 * offset byte: one dot-product-accumulate per entry (measured faster on
     // B200 than a byte permute followed by a multiply-add)
     b.a[0] = __dp4a(even, 0x00000080u, cell);
@@ -211,25 +225,18 @@ __device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t
     b.a[5] = __dp4a(odd, 0x00800000u, cell);
     b.a[6] = __dp4a(even, 0x80000000u, cell);
     b.a[7] = __dp4a(odd, 0x80000000u, cell);
-    b.fin = b.act;
+    b.h = b.v;
 #ifdef CELTY_GUARD
     for (int e = 0; e < 8; ++e)
-        if (b.fin && !CELTY_CHECK(b.a[e] >= slab_begin && b.a[e] + 4 <= slab_end, 2, b.a[e])) b.fin = 0;
+        if (!CELTY_CHECK(b.a[e] >= slab_begin && b.a[e] + 4 <= slab_end, 2, b.a[e])) {
+            b.a[e] = slab_begin + (b.a[e] & 124u);                 // a cell of this lane's bank; add nothing
+            b.h = make_uint4(0, 0, 0, 0);
+        }
 #endif
     (void)slab_begin; (void)slab_end;
-    // a lane without a group in this step decodes garbage, but it has none in any later step either
     cell += (total + kGroup) * 128u;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.u32 p, %16, 0;\n\t"
-        "@p ld.shared.f32 %0, [%8];\n\t@p ld.shared.f32 %1, [%9];\n\t"
-        "@p ld.shared.f32 %2, [%10];\n\t@p ld.shared.f32 %3, [%11];\n\t"
-        "@p ld.shared.f32 %4, [%12];\n\t@p ld.shared.f32 %5, [%13];\n\t"
-        "@p ld.shared.f32 %6, [%14];\n\t@p ld.shared.f32 %7, [%15];\n\t}"
-        : "+f"(b.c[0]), "+f"(b.c[1]), "+f"(b.c[2]), "+f"(b.c[3]), "+f"(b.c[4]), "+f"(b.c[5]), "+f"(b.c[6]), "+f"(b.c[7])
-        : "r"(b.a[0]), "r"(b.a[1]), "r"(b.a[2]), "r"(b.a[3]), "r"(b.a[4]), "r"(b.a[5]), "r"(b.a[6]), "r"(b.a[7]),
-          "r"(b.fin));
-    b.h = b.v;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) b.c[e] = lds_f32(b.a[e]);
 }
 
 __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
@@ -239,17 +246,8 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
     fma_pair(b.h.y, xj, b.c[2], b.c[3], d[2], d[3]);
     fma_pair(b.h.z, xj, b.c[4], b.c[5], d[4], d[5]);
     fma_pair(b.h.w, xj, b.c[6], b.c[7], d[6], d[7]);
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.u32 p, %16, 0;\n\t"
-        "@p st.shared.f32 [%0], %8;\n\t@p st.shared.f32 [%1], %9;\n\t"
-        "@p st.shared.f32 [%2], %10;\n\t@p st.shared.f32 [%3], %11;\n\t"
-        "@p st.shared.f32 [%4], %12;\n\t@p st.shared.f32 [%5], %13;\n\t"
-        "@p st.shared.f32 [%6], %14;\n\t@p st.shared.f32 [%7], %15;\n\t}"
-        :
-        : "r"(b.a[0]), "r"(b.a[1]), "r"(b.a[2]), "r"(b.a[3]), "r"(b.a[4]), "r"(b.a[5]), "r"(b.a[6]), "r"(b.a[7]),
-          "f"(d[0]), "f"(d[1]), "f"(d[2]), "f"(d[3]), "f"(d[4]), "f"(d[5]), "f"(d[6]), "f"(d[7]), "r"(b.fin)
-        : "memory");
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sts_f32(b.a[e], d[e]);
 }
 
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
@@ -269,7 +267,7 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     l.mail = off;      off += (size_t)teams * 16;                          // per team: batch sequence, batch size, done
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
-    l.lane_base = off; off += 256;                                         // rank of each lane's first survivor, n
+    l.lane_base = off; off += 256;                // rank of each lane's first survivor, n; 16 zero bytes at +240
     l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
     l.total = off;
     return l;
@@ -362,6 +360,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         float4 *acc4 = reinterpret_cast<float4 *>(acc);
         for (int i = tid; i < teams * slab_words / 4; i += nthreads) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    if (tid < 4) lane_base[60 + tid] = 0;                         // the zero group of idle lanes
     if (streams && member == 0 && lane == 0) {
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&empties[team * p.D + d]), (uint32_t)p.W);
@@ -406,13 +405,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         const uint32_t lt_mask = (1u << lane) - 1u;
         const uint32_t items0 = smem_u32(items);
         uint32_t issued = 0, consumed = 0;                            // ring positions of this team
+        uint32_t slot = 0, parity = 0, islot = 0;                     // consumed % D, (consumed / D) & 1, issued % D
         bool failed = false;
         long long dbg_wait = 0, dbg_head = 0, dbg_loop = 0, dbg_tail = 0, dbg_steps = 0;   // development builds
         (void)dbg_wait; (void)dbg_head; (void)dbg_loop; (void)dbg_tail; (void)dbg_steps;
         StepBuf b0, b1;                                               // pipeline registers, live across items
-        b0.v = make_uint4(0, 0, 0, 0); b0.w = 0; b1.v = b0.v; b1.w = 0; b0.h = b0.v; b1.h = b0.v;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) { b0.c[e] = 0.f; b1.c[e] = 0.f; }
+        const uint32_t zeros = smem_u32(lane_base) + 240u;            // 16 bytes of zeros
 
         for (int rb = r_begin; rb < r_end; rb += p.cap) {
             const int cnt = min(p.cap, r_end - rb);
@@ -456,17 +454,16 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             }
             // ---- a2: keep D copies in flight (issued by lane 0 of the team's first warp, or by the producer warp)
             auto issue = [&](int i) {
-                const uint32_t slot = issued % (uint32_t)p.D;
                 const uint2 im = imeta[i];
-                mbar_expect_tx(bar0 + 8u * slot, im.y);
-                bulk_load(ring0 + slot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y, bar0 + 8u * slot);
+                mbar_expect_tx(bar0 + 8u * islot, im.y);
+                bulk_load(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y, bar0 + 8u * islot);
                 ++issued;
+                if (++islot == (uint32_t)p.D) islot = 0;
             };
             if (!p.producer && member == 0 && lane == 0 && !failed)
                 for (int i = 0; i < min(cnt, p.D); ++i) issue(i);
             CELTY_MARK(3);
             for (int i = 0; i < cnt; ++i) {
-                const uint32_t slot = consumed % (uint32_t)p.D, parity = (consumed / (uint32_t)p.D) & 1u;
                 const long long t_a = CELTY_CLOCK();
                 // A warp that gave up on a copy keeps walking the items (and the team barriers) without
                 // touching them, so that the warps of a team never wait for one another in vain.
@@ -478,6 +475,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 if (failed) {
                     team_sync(bar_id, team_threads);
                     if (p.producer && lane == 0) mbar_arrive(emp0 + 8u * slot);
+                    if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
                     continue;
                 }
                 const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
@@ -504,18 +502,19 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                     }
                 }
                 uint32_t cell = cell0 + row0 * 128u;
+                const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
                 const long long t_c = CELTY_CLOCK();
-                step_fetch(b0, gl, q_lo, q_hi, cum, lt_mask, vbase, rbase, slot_end);
-                step_fetch(b1, gl, q_lo + 1, q_hi, cum, lt_mask, vbase, rbase, slot_end);
-                step_decode(b0, cell, slab0, slab_end);                                    // step q_lo
-                step_fetch(b0, gl, q_lo + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end);
+                step_fetch(b0, gl, q_lo, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                step_fetch(b1, gl, q_lo + 1, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                step_decode(b0, cell, spare, slab0, slab_end);                                    // step q_lo
+                step_fetch(b0, gl, q_lo + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 for (uint32_t q = q_lo + 1; q <= q_hi; q += 2) {
-                    step_decode(b1, cell, slab0, slab_end);                                // step q
+                    step_decode(b1, cell, spare, slab0, slab_end);                                // step q
                     step_finish(b0, xj);                                                   // step q-1
-                    step_fetch(b1, gl, q + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end);
-                    step_decode(b0, cell, slab0, slab_end);                                // step q+1
+                    step_fetch(b1, gl, q + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                    step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
                     step_finish(b1, xj);                                                   // step q
-                    step_fetch(b0, gl, q + 3, q_hi, cum, lt_mask, vbase, rbase, slot_end);
+                    step_fetch(b0, gl, q + 3, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 }
                 const long long t_d = CELTY_CLOCK();
                 // every warp of the team is done with this sub-block (and with its rows) before the
@@ -528,12 +527,14 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 } else if (member == 0 && lane == 0 && i + p.D < cnt && !failed) {
                     issue(i + p.D);
                 }
+                if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
                 dbg_wait += t_b - t_a; dbg_head += t_c - t_b; dbg_loop += t_d - t_c; dbg_tail += CELTY_CLOCK() - t_d;
                 dbg_steps += q_hi - q_lo;
             }
             CELTY_STORE(11, dbg_wait); CELTY_STORE(12, dbg_head); CELTY_STORE(13, dbg_loop); CELTY_STORE(14, dbg_tail);
             CELTY_STORE(15, dbg_steps);
             issued = __shfl_sync(kFull, issued, 0);
+            islot = __shfl_sync(kFull, islot, 0);
             team_sync(bar_id, team_threads);                      // items / imeta are rewritten by the next batch
         }
         if (p.producer && member == 0 && lane == 0) mail[team * 4 + 2] = 1;      // no more batches from this team
@@ -552,7 +553,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         const uint32_t pring0 = smem_u32(ring + (size_t)t * p.D * p.slot_bytes);
         const uint2 *pim = reinterpret_cast<const uint2 *>(smem + lay.imeta) + (size_t)t * p.cap;
         int seq_seen = 0, next = 0, cnt = 0;
-        uint32_t pos = 0;
+        uint32_t slot = 0, use = 0;                                 // ring position = use * D + slot
         bool done = false;
         for (uint32_t it = 0; it < 4u * kSpinLimit && !done; ++it) {
             if (next == cnt) {                                      // look for the team's next batch
@@ -569,7 +570,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 }
                 continue;
             }
-            const uint32_t slot = pos % (uint32_t)p.D, use = pos / (uint32_t)p.D;
             if (use > 0 && !mbar_try_wait(pemp0 + 8u * slot, (use - 1u) & 1u)) {
                 __nanosleep(32);
                 continue;
@@ -577,7 +577,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             const uint2 im = pim[next];
             mbar_expect_tx(pbar0 + 8u * slot, im.y);
             bulk_load(pring0 + slot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y, pbar0 + 8u * slot);
-            ++pos;
+            if (++slot == (uint32_t)p.D) { slot = 0; ++use; }
             ++next;
         }
         if (!done) atomicOr(p.status, kStatusTimeout);
@@ -601,32 +601,35 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             __threadfence();
             if (!ok) atomicOr(p.status, kStatusTimeout);
         }
-        const int tstride = p.R + 4;
-        float *stage = reinterpret_cast<float *>(smem + lay.ring);
-        const int group_words = p.Sc * slab_words;
-        for (int fsl = 0; fsl < p.Sc; ++fsl) {
-            const float *src = acc + (size_t)fsl * slab_words + lane;
-            float *dst = stage + (size_t)(fsl * 32 + lane) * tstride;
-            for (int i = 2 * warp; i < p.R; i += 2 * nwarps) {      // two rows per pass: all loads first
-                float v0 = 0.f, v1 = 0.f;
-                const bool two = i + 1 < p.R;
-                for (int gg = 0; gg < p.G; ++gg) {
-                    v0 += src[(size_t)gg * group_words + i * 32];
-                    if (two) v1 += src[(size_t)gg * group_words + (i + 1) * 32];
+        // add the G accumulators into the first one
+        if (p.G > 1) {
+            float4 *acc4 = reinterpret_cast<float4 *>(acc);
+            const int group4 = p.Sc * slab_words / 4;
+            for (int q4 = tid; q4 < group4; q4 += nthreads) {
+                float4 v = acc4[q4];
+                for (int gg = 1; gg < p.G; ++gg) {
+                    const float4 t = acc4[(size_t)gg * group4 + q4];
+                    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
                 }
-                dst[i] = v0;
-                if (two) dst[i + 1] = v1;
+                acc4[q4] = v;
             }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
         CELTY_MARK(6);
-        if (tid < p.Sc * 32) {
-            const int fsl = tid >> 5, t = 32 * (part * p.Sc + fsl) + lane;
-            if (t < p.T) {
-                const int row0 = t * p.R, nrows = min(p.R, p.M - row0);
+        // The row map makes local rows [kC, kC + C) of a slab 32*C consecutive rows of y, in accumulator
+        // order (with one slab the whole accumulator is y itself): each such segment is one bulk reduce-add.
+        {
+            const int seg = p.S == 1 ? 16 : p.C, nseg = (p.R + seg - 1) / seg;
+            for (int sg = tid; sg < p.Sc * nseg; sg += nthreads) {
+                const int fsl = sg / nseg, k = sg - fsl * nseg, sfull = part * p.Sc + fsl;
+                if (sfull >= p.S) continue;
+                const int i0 = k * seg, i1 = min(p.R, i0 + seg);
+                const int64_t row0 = tile_row(p.S, p.C, sfull, 0, i0);
+                if (row0 >= p.M) continue;
+                const int nrows = min((i1 - i0) * 32, p.M - (int)row0);
                 const uint32_t bytes = ((uint32_t)nrows * 4u) & ~15u;
-                const float *src = stage + (size_t)(fsl * 32 + lane) * tstride;
+                const float *src = acc + (size_t)fsl * slab_words + (size_t)i0 * 32;
                 if (bytes)
                     asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(p.y + row0),
                                  "r"(smem_u32(src)), "r"(bytes)
@@ -635,7 +638,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                     if (src[i] != 0.f) atomicAdd(p.y + row0 + i, src[i]);
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging may go once it has been read
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may go once it has been read
         }
         CELTY_MARK(7);
     } else {
@@ -711,8 +714,9 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                         float total = 0.f;
                         for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
                         const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
-                        const int i = rem >> 5, t = 32 * (part * p.Sc + fsl) + (rem & 31), row = t * p.R + i;
-                        if (t < p.T && row < p.M) p.y[row] = total;
+                        const int sfull = part * p.Sc + fsl;
+                        const int64_t row = tile_row(p.S, p.C, sfull, rem & 31, rem >> 5);
+                        if (sfull < p.S && row < p.M) p.y[row] = total;
                     }
                 }
                 __syncthreads();

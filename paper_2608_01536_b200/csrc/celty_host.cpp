@@ -29,17 +29,28 @@ struct Logical {                 // one run per byte, block-major (column, tile)
     std::vector<uint8_t> runs;
 };
 
-int choose_tile_rows(int64_t M)
+// Slabs S, local rows per tile R and chunk C of the LANE_TILE row map for M rows (tile_rows = 0: library's
+// choice).  About 128 local rows per lane keep a lane's run stream at ~8 groups per column at 50% density;
+// when a column needs more slabs than one thread block takes, the slab count is rounded up to a multiple
+// of the number of row parts so that every part gets the same number.
+void choose_shape(int64_t M, int tile_rows, int64_t *S_out, int32_t *R_out, int32_t *C_out)
 {
-    // About 128 rows per lane keeps a lane's run stream at ~8 groups per column at 50% density.  Slabs of
-    // 32 lanes then cover M; when a column needs more slabs than one thread block takes, the slab count is
-    // rounded up to a multiple of the number of row parts so that every part gets the same number.
-    int64_t S = std::max<int64_t>(1, (M + 2048) / 4096);
-    const int64_t P = (S + kSlabsPerBlock - 1) / kSlabsPerBlock;
-    S = (S + P - 1) / P * P;
-    int64_t R = (M + 32 * S - 1) / (32 * S);
-    R = (R + 3) / 4 * 4;                       // keeps 16-byte vector accesses of a tile aligned
-    return (int)std::min<int64_t>(kMaxTileRows, std::max<int64_t>(4, R));
+    const int64_t Q = (M + 31) / 32;                                  // groups of 32 rows
+    int64_t S, R;
+    if (tile_rows > 0) {
+        R = tile_rows;
+        S = (Q + R - 1) / R;
+    } else {
+        S = std::max<int64_t>(1, (M + 2048) / 4096);
+        const int64_t P = (S + kSlabsPerBlock - 1) / kSlabsPerBlock;
+        S = (S + P - 1) / P * P;
+        R = ((Q + S - 1) / S + 3) / 4 * 4;
+        while (R > kMaxTileRows) { S += P; R = ((Q + S - 1) / S + 3) / 4 * 4; }
+        R = std::max<int64_t>(4, R);
+    }
+    *S_out = S;
+    *R_out = (int32_t)R;
+    *C_out = R % 4 == 0 ? 4 : 1;                                      // chunks of 4 groups = 512 bytes of y
 }
 
 // Build the COLUMN image: meta uint2[K] {off16, entries}, then per column its chunks of up to 32
@@ -174,30 +185,34 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
         if (o.layout == CELTY_LAYOUT_COLUMN) {
             m->R = (int32_t)M; m->T = 1; m->S = 1;
         } else {
-            m->R = o.tile_rows > 0 ? o.tile_rows : choose_tile_rows(M);
-            m->T = (M + m->R - 1) / m->R;
-            m->S = (m->T + 31) / 32;
+            choose_shape(M, o.tile_rows, &m->S, &m->R, &m->C);
+            m->T = 32 * m->S;
             if (m->S > 32) { delete m; return CELTY_EINVAL; }   // one warp per slab, 32 warps per block
         }
         const int64_t R = m->R, T = m->T;
+        const bool lane_tile = m->layout == CELTY_LAYOUT_LANE_TILE;
+        // local row i of tile t -> row of W (COLUMN: the one tile is the column itself)
+        auto row_of = [&](int64_t t, int64_t i) { return lane_tile ? tile_row(m->S, m->C, t / 32, t % 32, i) : i; };
         // Pass 1: one sweep over the rows of W keeps, per column, the last kept row; the gap before a
         // kept weight is split into floor(gap/16) pads and a run of gap mod 16 (Section 3.2).
         std::vector<uint32_t> cnt((size_t)(K * T), 0);
         std::vector<int32_t> last((size_t)K);
         uint64_t total = 0;
         for (int64_t t = 0; t < T; ++t) {
-            const int64_t r0 = t * R, r1 = std::min<int64_t>(M, r0 + R);
-            std::fill(last.begin(), last.end(), (int32_t)r0 - 1);
-            for (int64_t r = r0; r < r1; ++r)
+            std::fill(last.begin(), last.end(), -1);
+            for (int64_t i = 0; i < R; ++i) {
+                const int64_t r = row_of(t, i);
+                if (r >= M) break;                                    // a tile's rows grow with i
                 for (int64_t j = 0; j < K; ++j) {
                     if (!kept(W, ldw, mask, K, r, j)) continue;
-                    const uint32_t gap = (uint32_t)(r - last[j] - 1);
+                    const uint32_t gap = (uint32_t)(i - last[j] - 1);
                     cnt[j * T + t] += (gap >> 4) + 1;
                     total += (gap >> 4) + 1;
                     m->n_pad += gap >> 4;
                     m->nnz += 1;
-                    last[j] = (int32_t)r;
+                    last[j] = (int32_t)i;
                 }
+            }
         }
         if (total > 0xFFFFFFFFull) { delete m; return CELTY_EINVAL; }
         m->block_ptr.resize((size_t)(K * T + 1));
@@ -211,12 +226,13 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
         m->pad_bits.assign((size_t)(total + 7) / 8, 0);
         std::vector<uint32_t> cur(m->block_ptr.begin(), m->block_ptr.end() - 1);
         for (int64_t t = 0; t < T; ++t) {
-            const int64_t r0 = t * R, r1 = std::min<int64_t>(M, r0 + R);
-            std::fill(last.begin(), last.end(), (int32_t)r0 - 1);
-            for (int64_t r = r0; r < r1; ++r)
+            std::fill(last.begin(), last.end(), -1);
+            for (int64_t i = 0; i < R; ++i) {
+                const int64_t r = row_of(t, i);
+                if (r >= M) break;
                 for (int64_t j = 0; j < K; ++j) {
                     if (!kept(W, ldw, mask, K, r, j)) continue;
-                    uint32_t gap = (uint32_t)(r - last[j] - 1);
+                    uint32_t gap = (uint32_t)(i - last[j] - 1);
                     uint32_t &c = cur[j * T + t];
                     for (; gap > 15; gap -= 16) {
                         lg.vals[c] = 0; lg.runs[c] = 15;
@@ -224,8 +240,9 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
                         ++c;
                     }
                     lg.vals[c] = W[r * ldw + j]; lg.runs[c] = (uint8_t)gap; ++c;
-                    last[j] = (int32_t)r;
+                    last[j] = (int32_t)i;
                 }
+            }
         }
         if (m->layout == CELTY_LAYOUT_COLUMN) pack_column(m, lg); else pack_lane_tile(m, lg);
         m->P = (int32_t)((m->S + kSlabsPerBlock - 1) / kSlabsPerBlock);
@@ -251,6 +268,15 @@ extern "C" int celty_info(const celty_matrix *m, int64_t *M, int64_t *K, int64_t
     if (compressed_bytes) *compressed_bytes = (m->nnz + m->n_pad) * 5 / 2 + 4 * (m->K + 1);
     if (layout) *layout = m->layout;
     if (tile_rows) *tile_rows = m->layout == CELTY_LAYOUT_COLUMN ? 0 : m->R;
+    return CELTY_OK;
+}
+
+extern "C" int celty_row_map(const celty_matrix *m, int32_t *slabs, int32_t *tile_rows, int32_t *chunk)
+{
+    if (!m) return CELTY_EINVAL;
+    if (slabs) *slabs = (int32_t)m->S;
+    if (tile_rows) *tile_rows = m->R;
+    if (chunk) *chunk = m->C;
     return CELTY_OK;
 }
 
@@ -311,7 +337,7 @@ extern "C" int celty_decode_host(const celty_matrix *m, int64_t col, int32_t *ro
                     std::memcpy(&w, rbase + 4 * slot, 4);
                     const uint8_t run = (w >> (4 * (e % kGroup))) & 15u;
                     s += run;
-                    emit((uint64_t)m->block_ptr[col * T + t] + e, t * m->R + s + e, v, run);
+                    emit((uint64_t)m->block_ptr[col * T + t] + e, tile_row(m->S, m->C, sl, L, s + e), v, run);
                 }
             }
         }

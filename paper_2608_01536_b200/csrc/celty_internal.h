@@ -27,6 +27,25 @@ constexpr int kSlabsPerBlock = 4;    // LANE_TILE: a thread block covers at most
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+#ifdef __CUDACC__
+#define CELTY_HD __host__ __device__
+#else
+#define CELTY_HD
+#endif
+
+// LANE_TILE row map.  Rows are dealt to the 32 lanes one at a time (row r belongs to lane r mod 32), and
+// the groups of 32 consecutive rows are dealt to the S slabs in chunks of C groups, round robin.  Tile
+// t = 32*s + L is the ordered set of rows that lane L of slab s receives; local row i of that tile is
+//     row = (((i / C) * S + s) * C + i mod C) * 32 + L.
+// A lane's local rows grow with the row number, every slab samples the whole height of the matrix (so a
+// mask whose density drifts with the row index still gives every lane and every slab the same share),
+// and local rows [kC, kC + C) of a slab are the 32*C consecutive rows that start at ((k*S + s)*C)*32:
+// the accumulator word (i*32 + L) order of a slab is the order of y, C*32 rows at a time.
+CELTY_HD inline int64_t tile_row(int64_t S, int64_t C, int64_t s, int64_t lane, int64_t i)
+{
+    return (((i / C) * S + s) * C + i % C) * 32 + lane;
+}
+
 // Workspace layout (device): all offsets multiples of 256.
 struct WorkspaceLayout {
     size_t status_off;   // uint32 status, int32 count, uint32 tickets[2] (and spare words)
@@ -56,8 +75,9 @@ inline WorkspaceLayout workspace_layout(int64_t K, int64_t T, int64_t part_words
 struct celty_matrix {
     int64_t M = 0, K = 0;
     int32_t layout = 0;
-    int32_t R = 0;          // rows per tile (LANE_TILE) or M (COLUMN)
-    int64_t T = 1;          // tiles per column
+    int32_t R = 0;          // local rows per tile (LANE_TILE) or M (COLUMN)
+    int32_t C = 1;          // LANE_TILE: groups of 32 rows that go to the same slab in a row (see tile_row)
+    int64_t T = 1;          // tiles per column (LANE_TILE: 32 * S)
     int64_t S = 1;          // slabs of 32 tiles per column (LANE_TILE), 1 for COLUMN
     int32_t P = 1, Sc = 1;  // LANE_TILE: row parts per column and slabs per part (P * Sc >= S)
     int64_t nnz = 0, n_pad = 0;

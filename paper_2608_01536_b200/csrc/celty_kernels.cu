@@ -256,8 +256,8 @@ __global__ void k_decode_column(const uint2 *__restrict__ meta, const uint8_t *_
 }
 
 // ------------------------------------------------------------------------------------------------
-// LANE_TILE layout kernel.  Rows are partitioned into tiles of R rows and the rule of Section 3.2
-// restarts in every tile.  Warp s of a warp group owns slab s (tiles 32s .. 32s+31), lane L owns tile
+// LANE_TILE layout kernel.  Rows are partitioned into tiles of R rows each (the row map tile_row deals
+// them out lane by lane and slab by slab) and the rule of Section 3.2 restarts in every tile.  Warp s of a warp group owns slab s (tiles 32s .. 32s+31), lane L owns tile
 // 32s+L: each lane walks its own run stream with a running row sum (no cross-lane scan is needed),
 // and local row i of lane L lives at accumulator word (s*(R+8) + i)*32 + L, i.e. in bank L -- every
 // scatter instruction touches 32 distinct banks, and no two threads ever touch the same word, so the
@@ -268,7 +268,7 @@ __global__ void k_decode_column(const uint2 *__restrict__ meta, const uint8_t *_
 __global__ void __launch_bounds__(1024)
 k_spmspv_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ stream,
               const int32_t *__restrict__ idx, const uint16_t *__restrict__ val,
-              const int32_t *__restrict__ count, float *__restrict__ y, int M, int R, int S, int T, int G)
+              const int32_t *__restrict__ count, float *__restrict__ y, int M, int R, int S, int C, int G)
 {
     extern __shared__ float acc[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -311,8 +311,8 @@ k_spmspv_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ str
     __syncthreads();
     for (int w = warp; w < S * R; w += nwarps) {
         const int sl = w / R, i = w - sl * R;
-        const int t = 32 * sl + lane, r = t * R + i;
-        if (t < T && r < M) {
+        const int64_t r = tile_row(S, C, sl, lane, i);
+        if (r < M) {
             float v = 0.f;
             for (int gg = 0; gg < G; ++gg) v += acc[gg * group_words + sl * slab_words + i * 32 + lane];
             if (v != 0.f) atomicAdd(&y[r], v);
@@ -322,7 +322,7 @@ k_spmspv_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ str
 
 // scratch[0 .. T] = the column's logical block pointers (entries before each tile), relative to scratch[0]
 __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ stream, int j,
-                              int R, int S, int T, const uint32_t *__restrict__ scratch, int32_t *rows,
+                              int S, int C, const uint32_t *__restrict__ scratch, int32_t *rows,
                               uint16_t *vals, int cap, int32_t *count)
 {
     const int lane = threadIdx.x & 31, s = threadIdx.x >> 5;
@@ -331,9 +331,9 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
     const uint32_t steps = __reduce_max_sync(kFull, gl);
     const uint32_t Gs = __reduce_add_sync(kFull, gl);
     const uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * (size_t)Gs;
-    const int t = 32 * s + lane;
-    const uint32_t out0 = t < T ? scratch[t] - scratch[0] : 0u;
-    const uint32_t nt = t < T ? scratch[t + 1] - scratch[t] : 0u;
+    const int t = 32 * s + lane, T = 32 * S;
+    const uint32_t out0 = scratch[t] - scratch[0];
+    const uint32_t nt = scratch[t + 1] - scratch[t];
     uint32_t slot0 = 0, row = 0;
     for (uint32_t q = 0; q < steps; ++q) {
         const bool active = gl > q;
@@ -347,7 +347,7 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
             for (int e = 0; e < kGroup; ++e) {
                 const uint32_t k = q * kGroup + e;
                 if (k < nt && out0 + k < (uint32_t)cap) {
-                    rows[out0 + k] = (int32_t)(t * R + row + entry_offset(even, odd, e));
+                    rows[out0 + k] = (int32_t)tile_row(S, C, s, lane, row + entry_offset(even, odd, e));
                     vals[out0 + k] = entry_bits(v, e);
                 }
             }
@@ -420,10 +420,7 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
     // a warp that does not stream can issue all the bulk copies (variant bit 3 turns that off)
     pl.producer = (32 * pl.G * pl.Sc * pl.W < pl.threads && !m->no_producer) ? 1 : 0;
-    // bulk reduce-add merge: its staging tiles reuse the ring area and must fit there
     pl.merge = (m->merge >= 0 ? m->merge : 1);
-    if ((size_t)pl.Sc * 32 * (m->R + 4) * 4 > (size_t)pl.G * pl.Sc * pl.D * pl.slot_bytes) pl.merge = 0;
-    if (m->R % 4) pl.merge = 0;                // tiles of y and of the staging area must start on 16 bytes
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
     pl.grid = std::max(1, blocks / pl.P) * pl.P;
@@ -499,7 +496,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.y = y;
         fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
         fp.partials = reinterpret_cast<float *>(m->d_ws + m->ws.partial_off);
-        fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.T = (int)m->T;
+        fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.C = m->C;
         fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.W = plan.W;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         fp.stream_bytes = (long long)m->stream_bytes;
@@ -539,7 +536,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         const int grid = m->grid > 0 ? m->grid : di.sms;
         k_spmspv_lane<<<grid, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(m->d_image),
                                                               stream_base, idx, val, count, y, (int)m->M, m->R,
-                                                              (int)m->S, (int)m->T, G);
+                                                              (int)m->S, m->C, G);
     }
     CELTY_CUDA(cudaGetLastError());
     return CELTY_OK;
@@ -610,7 +607,7 @@ extern "C" int celty_spmspv_static(const celty_matrix *m, const void *image_dev,
     const uint8_t *image = static_cast<const uint8_t *>(image_dev);
     k_spmspv_lane<<<di.sms, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(image),
                                                             image + m->meta_bytes, idx, val, count, y, (int)m->M, m->R,
-                                                            (int)m->S, (int)m->T, G);
+                                                            (int)m->S, m->C, G);
     CELTY_CUDA(cudaGetLastError());
     return CELTY_OK;
 }
@@ -655,7 +652,7 @@ extern "C" int celty_decode_device(celty_matrix *m, int64_t col, int32_t *rows_d
         CELTY_CUDA(cudaMemcpyAsync(scratch, &m->block_ptr[(size_t)col * m->T], (size_t)(m->T + 1) * 4,
                                    cudaMemcpyHostToDevice, st));
         k_decode_lane<<<1, 32 * (int)m->S, 0, st>>>(reinterpret_cast<const uint32_t *>(m->d_image), stream_base,
-                                                    (int)col, m->R, (int)m->S, (int)m->T, scratch, rows_dev, vals_dev,
+                                                    (int)col, (int)m->S, m->C, scratch, rows_dev, vals_dev,
                                                     (int)cap, count_dev);
     }
     CELTY_CUDA(cudaGetLastError());

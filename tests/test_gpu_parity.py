@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+from conftest import permute_for_lane_tiles
 from oracle import celty_oracle as orc
 from paper_2608_01536_b200 import build, celty, synth
 
@@ -97,10 +98,18 @@ def test_device_decode_bit_exact(layout, M, K, d_w, tile_rows):
     mask[-1, 1] = 1                     # only the last row: maximum number of pads
     mask[:, 2] = 1                      # dense column
     m = celty.Matrix(W, mask, layout=layout, tile_rows=tile_rows, device="cuda")
-    enc = orc.rlc_encode(W, mask, 4, tile_rows=m.info().tile_rows)
+    rowmap = None
+    if layout == celty.LAYOUT_LANE_TILE:
+        S, R, C = m.row_map()
+        Wp, mp, rowmap = permute_for_lane_tiles(W, mask, S, R, C)
+        enc = orc.rlc_encode(Wp, mp, 4, tile_rows=R)
+    else:
+        enc = orc.rlc_encode(W, mask, 4, tile_rows=0)
     for j in range(K):
         rows, vals = m.decode_device(j)
         orows, ovals, _, _ = orc.column_entries(enc, j)
+        if rowmap is not None:
+            orows = rowmap[orows]
         assert np.array_equal(rows, orows), j
         assert np.array_equal(vals, ovals), j
 

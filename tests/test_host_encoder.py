@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from conftest import read_golden
+from conftest import permute_for_lane_tiles, read_golden
 from oracle import celty_oracle as orc
 from paper_2608_01536_b200 import build, celty, synth
 
@@ -33,13 +33,24 @@ def test_encoder_matches_oracle(M, K, d_w, layout, tile_rows):
     info = m.info()
     R = info.tile_rows
     assert (R == 0) == (layout == celty.LAYOUT_COLUMN)
-    enc = orc.rlc_encode(W, mask, 4, tile_rows=R)
+    rowmap = None
+    if layout == celty.LAYOUT_LANE_TILE:
+        S, R2, C = m.row_map()
+        assert R2 == R and (tile_rows == 0 or R == tile_rows) and 32 * S * R >= M
+        Wp, mp, rowmap = permute_for_lane_tiles(W, mask, S, R, C)
+        enc = orc.rlc_encode(Wp, mp, 4, tile_rows=R)
+    else:
+        assert m.row_map() == (1, M, 1)
+        enc = orc.rlc_encode(W, mask, 4, tile_rows=R)
     assert info.nnz == int(mask.sum())
     assert info.n_pad == int(enc.is_pad.sum())
     assert info.compressed_bytes == enc.vals.size * 5 // 2 + 4 * (K + 1)
     for j in range(K):
         rows, vals, runs, pad = m.decode_host(j)
         orows, ovals, opad, oruns = orc.column_entries(enc, j)
+        if rowmap is not None:
+            orows = rowmap[orows]
+            assert orows.min(initial=0) >= 0
         assert np.array_equal(rows, orows)
         assert np.array_equal(vals, ovals)
         assert np.array_equal(runs, oruns)
@@ -62,15 +73,20 @@ def test_null_mask_keeps_nonzero_weights():
 def test_library_encoder_on_hand_vectors(name, layout):
     c = read_golden("rlc_hand_vectors_4bit.txt")[name]
     M = c["M"][0]
-    W = np.zeros((M, 1), np.float16)
-    mask = np.zeros((M, 1), np.uint8)
+    # LANE_TILE with one slab deals row r to lane r mod 32: rows 32*i are lane 0's tile, local row i, so
+    # the hand vector stretched by 32 must come back as lane 0's encoding
+    stretch = 1 if layout == celty.LAYOUT_COLUMN else 32
+    W = np.zeros((M * stretch, 1), np.float16)
+    mask = np.zeros((M * stretch, 1), np.uint8)
     for r in c["kept_rows"]:
-        W[r, 0] = r + 1
-        mask[r, 0] = 1
-    # one tile covering the whole column reproduces the whole-column encoding
+        W[r * stretch, 0] = r + 1
+        mask[r * stretch, 0] = 1
     m = celty.Matrix(W, mask, layout=layout, tile_rows=0 if layout == celty.LAYOUT_COLUMN else max(4, M))
+    if layout == celty.LAYOUT_LANE_TILE:
+        assert m.row_map()[0] == 1
     rows, vals, runs, pad = m.decode_host(0)
-    assert rows.tolist() == c["rows"] and runs.tolist() == c["runs"] and pad.tolist() == c["is_pad"]
+    assert rows.tolist() == [r * stretch for r in c["rows"]]
+    assert runs.tolist() == c["runs"] and pad.tolist() == c["is_pad"]
 
 
 def test_packed_run_nibbles_are_little_endian():
