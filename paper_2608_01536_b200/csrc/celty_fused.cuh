@@ -37,6 +37,8 @@ struct FusedParams {
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // items a team looks up per batch
+    int units;                 // groups that share the survivor list: (grid / P) * G; units_inv = floor(2^32 / units)
+    uint32_t units_inv;
     int producer;              // 1: the last warp issues every team's bulk copies (needs an idle warp)
     int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row tiles into y
 };
@@ -253,7 +255,7 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, empty, mail, items, imeta, lane_base, keep, total;
+    size_t acc, ring, bars, empty, mail, items, imeta, lane_base, keep, wrel, blk, total;
 };
 
 __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
@@ -267,8 +269,10 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     l.mail = off;      off += (size_t)teams * 16;                          // per team: batch sequence, batch size, done
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
-    l.lane_base = off; off += 256;                // rank of each lane's first survivor, n; 16 zero bytes at +240
+    l.lane_base = off; off += 256;                // [32] survivors n, [33] n / units, [34] n mod units; 16 zero bytes at +240
     l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
+    l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 8
+    l.blk = off;       off += ((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16; // survivors before each block of 8 keep words
     l.total = off;
     return l;
 }
@@ -291,7 +295,9 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     volatile int *mail = reinterpret_cast<volatile int *>(smem + lay.mail);   // [team][4]: seq, cnt, done, -
     int2 *items = reinterpret_cast<int2 *>(smem + lay.items) + (size_t)team * p.cap;      // [cap] {column, x bits}
     uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
-    int *lane_base = reinterpret_cast<int *>(smem + lay.lane_base);                       // [32] + [32] = n
+    int *lane_base = reinterpret_cast<int *>(smem + lay.lane_base);                       // see fused_smem_layout
+    int *wrel = reinterpret_cast<int *>(smem + lay.wrel);                                 // [nwords]
+    int *blk = reinterpret_cast<int *>(smem + lay.blk);                                   // [nwords / 8]
     uint32_t *kbw = reinterpret_cast<uint32_t *>(smem + lay.keep);
 
     const int part = blockIdx.x % p.P, kslice = blockIdx.x / p.P, nK = gridDim.x / p.P;
@@ -321,13 +327,17 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         for (size_t l = l0 + tid; l < min(lines, l0 + per); l += nthreads)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + l * 128));
     }
-    // ---- a1: threshold all of x; byte q of the keep words = keep bits of activations 8q .. 8q+7.
+    // ---- a1: threshold all of x.  A thread takes 8 activations (one 128-bit load) and makes one keep byte,
+    // four neighbouring lanes assemble a keep word, and the warp scans the survivor counts of its 8 words:
+    //   kbw[w]  keep bits of activations 32w .. 32w+31,
+    //   wrel[w] survivors in the words before w of the same block of 8 words,
+    //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
-    const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5;
+    const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 7) >> 3;
     {
-        uint8_t *kb = reinterpret_cast<uint8_t *>(kbw);
         const __half2 tau2 = __half2half2(__float2half_rd(p.tau));
-        for (int q = tid; q < nwords * 4; q += nthreads) {
+        for (int q0 = 0; q0 < nwords * 4; q0 += nthreads) {       // the same trip count for every thread
+            const int q = q0 + tid;
             uint32_t keep = 0;
             if (q < ngroups) {
                 uint32_t h[4];
@@ -351,57 +361,75 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                     if ((bits >> 16) == 0 && 8 * q + 2 * k + 1 < p.K) keep |= 2u << (2 * k);
                 }
             }
-            kb[q] = (uint8_t)keep;
+            uint32_t word = keep << (8 * (lane & 3));
+            word |= __shfl_xor_sync(kFull, word, 1);
+            word |= __shfl_xor_sync(kFull, word, 2);
+            const int cnt = (lane & 3) == 0 ? __popc(word) : 0;
+            int incl = cnt;
+#pragma unroll
+            for (int d = 4; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(kFull, incl, d);
+                if (lane >= d) incl += up;
+            }
+            const int w = q >> 2;
+            if ((lane & 3) == 0 && w < nwords) {
+                kbw[w] = word;
+                wrel[w] = incl - cnt;
+            }
+            if (lane == 28 && (w >> 3) < nblk) blk[w >> 3] = incl;
         }
     }
     CELTY_MARK(10);
-    // clear the accumulators while those loads are in flight
-    {
-        float4 *acc4 = reinterpret_cast<float4 *>(acc);
-        for (int i = tid; i < teams * slab_words / 4; i += nthreads) acc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     if (tid < 4) lane_base[60 + tid] = 0;                         // the zero group of idle lanes
     if (streams && member == 0 && lane == 0) {
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&empties[team * p.D + d]), (uint32_t)p.W);
-        mail[team * 4 + 0] = 0; mail[team * 4 + 1] = 0; mail[team * 4 + 2] = 0;
+        mail[team * 4 + 0] = 0; mail[team * 4 + 1] = 0; mail[team * 4 + 2] = 0; mail[team * 4 + 3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
     CELTY_MARK(1);
-    // ---- ranks: lane L of warp 0 owns keep words [L*wpl, (L+1)*wpl); lane_base[L] = rank of its first survivor
-    const int wpl = (nwords + 31) >> 5;
+    // ---- ranks: warp 0 turns the block counts into survivors before each block, 32 blocks at a time; the
+    // list is then cut into equal shares for the groups that work on different columns.
     if (warp == 0) {
-        const int w0 = min(nwords, lane * wpl), w1 = min(nwords, w0 + wpl);
-        int mine = 0;
-        for (int w = w0; w < w1; ++w) mine += __popc(kbw[w]);
-        int incl = mine;
+        int carry = 0;
+        for (int e0 = 0; e0 < nblk; e0 += 32) {
+            const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
+            int incl = cnt;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int up = __shfl_up_sync(kFull, incl, d);
-            if (lane >= d) incl += up;
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(kFull, incl, d);
+                if (lane >= d) incl += up;
+            }
+            if (e < nblk) blk[e] = carry + incl - cnt;
+            carry += __shfl_sync(kFull, incl, 31);
         }
-        lane_base[lane] = incl - mine;
-        if (lane == 31) {
-            lane_base[32] = incl;
-            if (blockIdx.x == 0) *p.count = incl;
+        if (lane == 0) {
+            // n / units without a division: units_inv = floor(2^32 / units) gives a quotient that is at most
+            // one too small
+            uint32_t share = __umulhi((uint32_t)carry, p.units_inv), extra = (uint32_t)carry - share * (uint32_t)p.units;
+            if (extra >= (uint32_t)p.units) { ++share; extra -= (uint32_t)p.units; }
+            lane_base[32] = carry;
+            lane_base[33] = (int)share;
+            lane_base[34] = (int)extra;
+            if (blockIdx.x == 0) *p.count = carry;
         }
     }
     __syncthreads();
     CELTY_MARK(2);
 
     if (streams) {
-        const int n = lane_base[32];
-        // group u of nK * G owns ranks [u*n/units, (u+1)*n/units)
-        const int64_t units = (int64_t)nK * p.G, u = (int64_t)kslice * p.G + g;
-        const int r_begin = (int)(u * n / units), r_end = (int)((u + 1) * n / units);
+        // group u of nK * G owns n / units ranks, the first n mod units groups one more
+        const int u = kslice * p.G + g, share = lane_base[33], extra = lane_base[34];
+        const int r_begin = u * share + min(u, extra), r_end = r_begin + share + (u < extra ? 1 : 0);
         const int team_threads = 32 * p.W, bar_id = 1 + team;
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
         const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
         const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
         const uint32_t bar0 = smem_u32(&bars[team * p.D]), emp0 = smem_u32(&empties[team * p.D]);
         int batch_seq = 0;
+        bool zeroed = false;
         const uint32_t lt_mask = (1u << lane) - 1u;
         const uint32_t items0 = smem_u32(items);
         uint32_t issued = 0, consumed = 0;                            // ring positions of this team
@@ -417,19 +445,26 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             // ---- column of rank r: the lane whose words hold it, then the word, then the bit
             for (int i = member * 32 + lane; i < cnt; i += team_threads) {
                 const int r = rb + i;
-                int o = 0;
+                // the block of 8 keep words that holds rank r (the last one with blk[e] <= r), the word in it
+                // (the last one with wrel[w] <= what is left) ...
+                int e = 0;
+                for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
+                    if (e + step < nblk && blk[e + step] <= r) e += step;
+                int k = r - blk[e], w = 8 * e;
 #pragma unroll
-                for (int step = 16; step; step >>= 1)
-                    if (lane_base[o + step] <= r) o += step;
-                int rem = r - lane_base[o], w = o * wpl;
-                for (;;) {
-                    if (!CELTY_CHECK(w >= 0 && w < nwords, 8, w)) { w = 0; rem = 0; break; }
-                    const int pc = __popc(kbw[w]);
-                    if (rem < pc) break;
-                    rem -= pc;
-                    ++w;
+                for (int step = 4; step; step >>= 1)
+                    if (w + step < nwords && wrel[w + step] <= k) w += step;
+                k -= wrel[w];
+                // ... and the bit in it: halve the word, keep the half that holds the wanted set bit
+                const uint32_t word = kbw[w];
+                int pos = 0;
+#pragma unroll
+                for (int sh = 16; sh; sh >>= 1) {
+                    const int c = __popc((word >> pos) & ((1u << sh) - 1u));
+                    if (k >= c) { k -= c; pos += sh; }
                 }
-                int j = 32 * w + (int)__fns(kbw[w], 0, rem + 1);
+                if (!CELTY_CHECK(((word >> pos) & 1u) != 0 && k == 0, 8, w)) pos = 0;
+                int j = 32 * w + pos;
                 if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
                 const uint16_t xb = p.x[j];
                 items[i] = make_int2(j, (int)xb);
@@ -445,14 +480,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                         imeta[i] = make_uint2(0u, (uint32_t)kSubHeader);
                 }
             }
+
             team_sync(bar_id, team_threads);
             if (s >= p.S) continue;
-            if (p.producer && member == 0 && lane == 0) {           // hand the batch to the producer warp
-                mail[team * 4 + 1] = cnt;
-                __threadfence_block();
-                mail[team * 4 + 0] = ++batch_seq;
-            }
-            // ---- a2: keep D copies in flight (issued by lane 0 of the team's first warp, or by the producer warp)
+            // ---- a2: keep D copies in flight.  Lane 0 of the team's first warp issues the first D of the
+            // first batch itself (nobody is closer to the offsets); after that the producer warp takes over,
+            // or, without one, the same lane refills a slot whenever the team has finished with it.
             auto issue = [&](int i) {
                 const uint2 im = imeta[i];
                 mbar_expect_tx(bar0 + 8u * islot, im.y);
@@ -460,9 +493,23 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 ++issued;
                 if (++islot == (uint32_t)p.D) islot = 0;
             };
-            if (!p.producer && member == 0 && lane == 0 && !failed)
-                for (int i = 0; i < min(cnt, p.D); ++i) issue(i);
+            const int pre = (!p.producer || rb == r_begin) ? min(cnt, p.D) : 0;
+            if (member == 0 && lane == 0 && !failed) {
+                for (int i = 0; i < pre; ++i) issue(i);
+                if (p.producer) {                                   // hand the rest of the batch to the producer warp
+                    mail[team * 4 + 1] = cnt;
+                    mail[team * 4 + 3] = pre;
+                    __threadfence_block();
+                    mail[team * 4 + 0] = ++batch_seq;
+                }
+            }
             CELTY_MARK(3);
+            if (!zeroed) {                                          // clear the slab while the first copies fly
+                float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
+                for (int i = member * 32 + lane; i < slab_words / 4; i += team_threads) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                zeroed = true;
+                team_sync(bar_id, team_threads);
+            }
             for (int i = 0; i < cnt; ++i) {
                 const long long t_a = CELTY_CLOCK();
                 // A warp that gave up on a copy keeps walking the items (and the team barriers) without
@@ -537,6 +584,10 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             islot = __shfl_sync(kFull, islot, 0);
             team_sync(bar_id, team_threads);                      // items / imeta are rewritten by the next batch
         }
+        if (!zeroed && s < p.S) {                                     // a team without columns still owns a slab
+            float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
+            for (int i = member * 32 + lane; i < slab_words / 4; i += team_threads) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         if (p.producer && member == 0 && lane == 0) mail[team * 4 + 2] = 1;      // no more batches from this team
         if (failed) {
             // give copies that are still in flight a last (bounded) chance to land before the block exits
@@ -561,17 +612,19 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 if (sq != seq_seen) {
                     __threadfence_block();
                     cnt = mail[t * 4 + 1];
-                    next = 0;
+                    next = mail[t * 4 + 3];                         // the team issued that many itself
+                    for (int k = 0; k < next; ++k)
+                        if (++slot == (uint32_t)p.D) { slot = 0; ++use; }
                     seq_seen = sq;
                 } else if (mail[t * 4 + 2] && mail[t * 4 + 0] == seq_seen) {
                     done = true;
                 } else {
-                    __nanosleep(64);
+                    __nanosleep(200);
                 }
                 continue;
             }
             if (use > 0 && !mbar_try_wait(pemp0 + 8u * slot, (use - 1u) & 1u)) {
-                __nanosleep(32);
+                __nanosleep(200);                                   // a slot comes back once per item: no hurry
                 continue;
             }
             const uint2 im = pim[next];

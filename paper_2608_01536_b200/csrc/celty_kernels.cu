@@ -502,6 +502,8 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
         fp.producer = plan.producer;
+        fp.units = (plan.grid / plan.P) * plan.G;
+        fp.units_inv = fp.units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / (uint64_t)fp.units);
         // the tickets count blocks of one launch shape: start them over when the shape changes
         if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
             CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
