@@ -258,8 +258,7 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            straight from global memory) instead of the single fused launch; for the fused launch
  *            2 = merge the blocks' results through per-block partial vectors summed in a fixed
  *            order (bit-reproducible) instead of adding them into y with bulk reduce-add copies,
- *            4 = force the bulk reduce-add merge, 8 = every warp team issues its own bulk copies
- *            instead of leaving that to an idle warp
+ *            4 = force the bulk reduce-add merge
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   team     fused kernel: warps that share one sub-block and one accumulator (1, 2 or 4)

@@ -39,7 +39,6 @@ struct FusedParams {
     int cap;                   // items a team looks up per batch
     int units;                 // groups that share the survivor list: (grid / P) * G; units_inv = floor(2^32 / units)
     uint32_t units_inv;
-    int producer;              // 1: the last warp issues every team's bulk copies (needs an idle warp)
     int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row tiles into y
 };
 
@@ -101,11 +100,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // Wait for a phase of an mbarrier with an iteration limit; false = gave up.
@@ -255,7 +249,7 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, empty, mail, items, imeta, lane_base, keep, wrel, blk, total;
+    size_t acc, ring, bars, items, imeta, lane_base, keep, wrel, blk, total;
 };
 
 __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
@@ -265,8 +259,7 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     l.acc = off;       off += (size_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
     l.ring = off;      off += (size_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
     l.bars = off;      off += (size_t)teams * D * 8;                       // one "full" mbarrier per slot
-    l.empty = off;     off += (size_t)teams * D * 8;                       // one "empty" mbarrier per slot (producer warp)
-    l.mail = off;      off += (size_t)teams * 16;                          // per team: batch sequence, batch size, done
+    off = (off + 15) / 16 * 16;
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
     l.lane_base = off; off += 256;                // [32] survivors n, [33] n / units, [34] n mod units; 16 zero bytes at +240
@@ -280,7 +273,10 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
 __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nwarps = nthreads >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x, nwarps = nthreads >> 5;
+    // the warp index through a shuffle: the compiler then knows that it (and every team, slab and loop bound
+    // derived from it) is the same for all lanes, and keeps the streaming loop free of divergence handling
+    const int warp = __shfl_sync(kFull, tid >> 5, 0);
     const int slab_words = (p.R + kTileSlack) * 32;
     // Warps [0, teams * W) stream columns, W warps per team; the others only help with the phases that
     // are plain data-parallel work (thresholding, clearing, storing and summing partial vectors).
@@ -291,8 +287,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
-    uint64_t *empties = reinterpret_cast<uint64_t *>(smem + lay.empty);
-    volatile int *mail = reinterpret_cast<volatile int *>(smem + lay.mail);   // [team][4]: seq, cnt, done, -
     int2 *items = reinterpret_cast<int2 *>(smem + lay.items) + (size_t)team * p.cap;      // [cap] {column, x bits}
     uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
     int *lane_base = reinterpret_cast<int *>(smem + lay.lane_base);                       // see fused_smem_layout
@@ -383,8 +377,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     if (tid < 4) lane_base[60 + tid] = 0;                         // the zero group of idle lanes
     if (streams && member == 0 && lane == 0) {
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
-        for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&empties[team * p.D + d]), (uint32_t)p.W);
-        mail[team * 4 + 0] = 0; mail[team * 4 + 1] = 0; mail[team * 4 + 2] = 0; mail[team * 4 + 3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -427,8 +419,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
         const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
         const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
-        const uint32_t bar0 = smem_u32(&bars[team * p.D]), emp0 = smem_u32(&empties[team * p.D]);
-        int batch_seq = 0;
+        const uint32_t bar0 = smem_u32(&bars[team * p.D]);
         bool zeroed = false;
         const uint32_t lt_mask = (1u << lane) - 1u;
         const uint32_t items0 = smem_u32(items);
@@ -483,9 +474,9 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 
             team_sync(bar_id, team_threads);
             if (s >= p.S) continue;
-            // ---- a2: keep D copies in flight.  Lane 0 of the team's first warp issues the first D of the
-            // first batch itself (nobody is closer to the offsets); after that the producer warp takes over,
-            // or, without one, the same lane refills a slot whenever the team has finished with it.
+            // ---- a2: keep D copies in flight.  Lane 0 of the team's first warp issues the first D of a batch
+            // and refills a slot whenever the team has finished with it.  (A dedicated producer warp that
+            // polled per-slot "empty" barriers was measured and was no faster at any configured shape.)
             auto issue = [&](int i) {
                 const uint2 im = imeta[i];
                 mbar_expect_tx(bar0 + 8u * islot, im.y);
@@ -493,16 +484,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 ++issued;
                 if (++islot == (uint32_t)p.D) islot = 0;
             };
-            const int pre = (!p.producer || rb == r_begin) ? min(cnt, p.D) : 0;
-            if (member == 0 && lane == 0 && !failed) {
-                for (int i = 0; i < pre; ++i) issue(i);
-                if (p.producer) {                                   // hand the rest of the batch to the producer warp
-                    mail[team * 4 + 1] = cnt;
-                    mail[team * 4 + 3] = pre;
-                    __threadfence_block();
-                    mail[team * 4 + 0] = ++batch_seq;
-                }
-            }
+            if (member == 0 && lane == 0 && !failed)
+                for (int i = 0; i < min(cnt, p.D); ++i) issue(i);
             CELTY_MARK(3);
             if (!zeroed) {                                          // clear the slab while the first copies fly
                 float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
@@ -521,7 +504,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 ++consumed;
                 if (failed) {
                     team_sync(bar_id, team_threads);
-                    if (p.producer && lane == 0) mbar_arrive(emp0 + 8u * slot);
                     if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
                     continue;
                 }
@@ -555,6 +537,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 step_fetch(b1, gl, q_lo + 1, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 step_decode(b0, cell, spare, slab0, slab_end);                                    // step q_lo
                 step_fetch(b0, gl, q_lo + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
+#pragma unroll 2
                 for (uint32_t q = q_lo + 1; q <= q_hi; q += 2) {
                     step_decode(b1, cell, spare, slab0, slab_end);                                // step q
                     step_finish(b0, xj);                                                   // step q-1
@@ -569,11 +552,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 team_sync(bar_id, team_threads);
                 // The slot's contents were consumed by loads whose values have been used, and the barrier
                 // above orders every team member's reads before this point: the copy may overwrite it.
-                if (p.producer) {
-                    if (lane == 0) mbar_arrive(emp0 + 8u * slot);  // one arrival per warp of the team frees the slot
-                } else if (member == 0 && lane == 0 && i + p.D < cnt && !failed) {
-                    issue(i + p.D);
-                }
+                if (member == 0 && lane == 0 && i + p.D < cnt && !failed) issue(i + p.D);
                 if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
                 dbg_wait += t_b - t_a; dbg_head += t_c - t_b; dbg_loop += t_d - t_c; dbg_tail += CELTY_CLOCK() - t_d;
                 dbg_steps += q_hi - q_lo;
@@ -588,52 +567,13 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
             for (int i = member * 32 + lane; i < slab_words / 4; i += team_threads) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (p.producer && member == 0 && lane == 0) mail[team * 4 + 2] = 1;      // no more batches from this team
         if (failed) {
             // give copies that are still in flight a last (bounded) chance to land before the block exits
-            if (member == 0 && !p.producer)
+            if (member == 0)
                 for (; consumed < issued; ++consumed)
                     mbar_wait_bounded(bar0 + 8u * (consumed % (uint32_t)p.D), (consumed / (uint32_t)p.D) & 1u);
             if (lane == 0) atomicOr(p.status, kStatusTimeout);
         }
-    }
-    else if (p.producer && warp == nwarps - 1 && lane < teams) {
-        // ---- producer: lane t issues team t's bulk copies, in order, as its ring slots are handed back
-        const int t = lane;
-        const uint32_t pbar0 = smem_u32(&bars[t * p.D]), pemp0 = smem_u32(&empties[t * p.D]);
-        const uint32_t pring0 = smem_u32(ring + (size_t)t * p.D * p.slot_bytes);
-        const uint2 *pim = reinterpret_cast<const uint2 *>(smem + lay.imeta) + (size_t)t * p.cap;
-        int seq_seen = 0, next = 0, cnt = 0;
-        uint32_t slot = 0, use = 0;                                 // ring position = use * D + slot
-        bool done = false;
-        for (uint32_t it = 0; it < 4u * kSpinLimit && !done; ++it) {
-            if (next == cnt) {                                      // look for the team's next batch
-                const int sq = mail[t * 4 + 0];
-                if (sq != seq_seen) {
-                    __threadfence_block();
-                    cnt = mail[t * 4 + 1];
-                    next = mail[t * 4 + 3];                         // the team issued that many itself
-                    for (int k = 0; k < next; ++k)
-                        if (++slot == (uint32_t)p.D) { slot = 0; ++use; }
-                    seq_seen = sq;
-                } else if (mail[t * 4 + 2] && mail[t * 4 + 0] == seq_seen) {
-                    done = true;
-                } else {
-                    __nanosleep(200);
-                }
-                continue;
-            }
-            if (use > 0 && !mbar_try_wait(pemp0 + 8u * slot, (use - 1u) & 1u)) {
-                __nanosleep(200);                                   // a slot comes back once per item: no hurry
-                continue;
-            }
-            const uint2 im = pim[next];
-            mbar_expect_tx(pbar0 + 8u * slot, im.y);
-            bulk_load(pring0 + slot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y, pbar0 + 8u * slot);
-            if (++slot == (uint32_t)p.D) { slot = 0; ++use; }
-            ++next;
-        }
-        if (!done) atomicOr(p.status, kStatusTimeout);
     }
     __syncthreads();
     CELTY_MARK(5);
@@ -790,7 +730,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 }
 
 struct FusedPlan {
-    int G, Sc, P, D, W, slot_bytes, cap, threads, grid, merge, producer;
+    int G, Sc, P, D, W, slot_bytes, cap, threads, grid, merge;
     size_t smem;
 };
 

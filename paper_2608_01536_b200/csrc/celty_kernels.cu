@@ -418,8 +418,6 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     pl.threads = std::max(512, 32 * pl.G * pl.Sc * pl.W);
     if (pl.threads > 512) return CELTY_EINVAL;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
-    // a warp that does not stream can issue all the bulk copies (variant bit 3 turns that off)
-    pl.producer = (32 * pl.G * pl.Sc * pl.W < pl.threads && !m->no_producer) ? 1 : 0;
     pl.merge = (m->merge >= 0 ? m->merge : 1);
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
@@ -501,7 +499,6 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
-        fp.producer = plan.producer;
         fp.units = (plan.grid / plan.P) * plan.G;
         fp.units_inv = fp.units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / (uint64_t)fp.units);
         // the tickets count blocks of one launch shape: start them over when the shape changes
