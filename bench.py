@@ -221,8 +221,9 @@ SWEEPS = {
 
 
 def run_sweep(args):
-    """Times every point of one configured sweep, one call at a time with the L2 flushed before each call
-    (a 256 MB memset), CUDA events around the call; the dense cuBLAS GEMV is timed the same way."""
+    """Times every point of one configured sweep with the protocol of the main run: calls rotate over enough
+    device copies of the layer to exceed 2x L2 (every call finds its matrix cold), one rotation is captured in
+    a CUDA graph, and CUDA events bracket several replays.  The dense cuBLAS GEMV is timed the same way."""
     import torch
     from paper_2608_01536_b200 import build as lib_build, celty
     lib_build.build()
@@ -230,62 +231,104 @@ def run_sweep(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     peak, _ = measured_peaks()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    reps = args.sweep_reps
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
 
-    def timed(fn):
-        ts = []
+    def rotation_us(calls):
+        for f in calls:
+            f()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for f in calls:
+                f()
+        g.replay()
+        torch.cuda.synchronize()
+        reps = max(3, -(-args.sweep_calls // len(calls)))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
         for _ in range(reps):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn()
-            b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b) * 1e3)
-        return float(np.median(ts)), float(np.min(ts))
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / (reps * len(calls))
 
-    points, cache_W, cache_m = [], {}, {}
+    points, key, mats, dense = [], None, [], []
     for i, pt in enumerate(SWEEPS[args.sweep]):
         M, K, s, fam = pt["M"], pt["K"], pt["s"], pt["family"]
-        seed = synth.point_seed(pt["cfg"], 0)
-        if (M, K) not in cache_W:
-            cache_W.clear()
-            cache_m.clear()
-            cache_W[(M, K)] = synth.weights(seed, M, K)
-        W = cache_W[(M, K)]
-        if (s, fam) not in cache_m:
-            cache_m.clear()                                    # one encoded matrix on the device at a time
+        if key != (M, K, s, fam):                              # one layer on the device at a time
+            key = (M, K, s, fam)
+            mats, dense = [], []
+            seed = synth.point_seed(pt["cfg"], 0)
+            W = synth.weights(seed, M, K)
             mask = (synth.mask_magnitude(W, s) if fam == "magnitude" else
                     synth.mask_bernoulli(seed, M, K, 1.0 - s) if fam == "bernoulli" else
                     synth.mask_powerlaw(seed, M, K, 1.0 - s))
-            m = celty.Matrix(W, mask, device=dev)
-            Wd = torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev)
-            cache_m[(s, fam)] = (m, Wd)
-            del mask
-        m, Wd = cache_m[(s, fam)]
-        x = synth.activations(synth.point_seed(pt["cfg"], 50 + i), K, pt["dist"])
-        tau = synth.threshold_for_density(x, pt["d_a"])
-        xd = torch.from_numpy(x).to(dev)
-        y = torch.empty(M, dtype=torch.float32, device=dev)
+            mats.append(celty.Matrix(W, mask, device=dev))
+            copies = int(np.ceil(2.5 * l2 / mats[0].device_bytes()[0])) + 1
+            while len(mats) < copies:
+                mats.append(celty.Matrix(W, mask, device=dev))
+            Wm = torch.from_numpy(np.where(mask != 0, W, np.float16(0)))
+            dense = [Wm.to(dev) for _ in range(min(copies, int(np.ceil(2.5 * l2 / (2 * M * K))) + 1))]
+            del W, mask, Wm
+        copies = len(mats)
+        xs, taus = [], []
+        for c in range(copies):
+            x = synth.activations(synth.point_seed(pt["cfg"], 50 + 16 * i + c), K, pt["dist"])
+            taus.append(synth.threshold_for_density(x, pt["d_a"]))
+            xs.append(torch.from_numpy(x).to(dev))
+        ys = [torch.empty(M, dtype=torch.float32, device=dev) for _ in range(copies)]
         yd = torch.empty(M, dtype=torch.float16, device=dev)
-        for _ in range(3):
-            m.spmspv(xd, tau, y)
-            torch.mv(Wd, xd, out=yd)
-        idx, _ = m.last_compaction()
-        assert m.last_status() == 0
-        sb, tb = m.fetched_bytes(idx.cpu().numpy())
-        us, us_min = timed(lambda: m.spmspv(xd, tau, y))
-        dus, dus_min = timed(lambda: torch.mv(Wd, xd, out=yd))
-        info = m.info()
+        fetched, survivors = [], []
+        for c in range(copies):
+            mats[c].spmspv(xs[c], taus[c], ys[c])
+            idx, _ = mats[c].last_compaction()
+            assert mats[c].last_status() == 0
+            fetched.append(mats[c].fetched_bytes(idx.cpu().numpy())[1])
+            survivors.append(int(idx.numel()))
+        tb = float(np.mean(fetched))
+        us = rotation_us([(lambda c=c: mats[c].spmspv(xs[c], taus[c], ys[c])) for c in range(copies)])
+        dus = rotation_us([(lambda c=c: torch.mv(dense[c % len(dense)], xs[c], out=yd)) for c in range(copies)])
+        info = mats[0].info()
         points.append({"M": M, "K": K, "weight_sparsity": s, "mask": fam, "activation_density": pt["d_a"],
-                       "survivors": int(idx.numel()), "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad,
-                       "fetched_bytes": tb, "us_per_call": us, "us_min": us_min, "GBps": tb / us / 1e3,
-                       "roofline_frac": tb / us / 1e3 / peak, "cublas_gemv_us": dus,
-                       "speedup_vs_cublas": dus / us, "combined_sparsity": 1.0 - (1.0 - s) * pt["d_a"]})
+                       "combined_sparsity": 1.0 - (1.0 - s) * pt["d_a"], "device_copies": copies,
+                       "survivors": float(np.mean(survivors)), "stored_entries": info.nnz + info.n_pad,
+                       "pads": info.n_pad, "fetched_bytes": tb, "us_per_call": us, "GBps": tb / us / 1e3,
+                       "roofline_frac": tb / us / 1e3 / peak, "cublas_gemv_us": dus, "speedup_vs_cublas": dus / us})
         print(json.dumps(points[-1]), file=sys.stderr, flush=True)
-    print(json.dumps({"sweep": args.sweep, "protocol": "one call at a time, 256 MB memset before each call, CUDA events, "
-                      f"median of {reps}", "peak_GBps": peak, "points": points}))
+    extra = {}
+    if args.sweep == "cfg4":
+        # the decode-layer chain of config 4: q, k, v, o (5120 x 5120), gate, up (13824 x 5120), down (5120 x 13824),
+        # 7 calls back to back on one stream, each with its own matrix and its own synthetic x; two layers in
+        # rotation (about 0.8 GB of compressed weights, far beyond L2)
+        del mats, dense
+        shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]
+        chain, dchain, tot_bytes = [], [], 0.0
+        for layer in range(2):
+            for k, (M, K) in enumerate(shapes):
+                seed = synth.point_seed(4, 10 * layer + k)
+                W = synth.weights(seed, M, K)
+                mask = synth.mask_bernoulli(seed, M, K, 0.5)
+                m = celty.Matrix(W, mask, device=dev)
+                x = synth.activations(synth.point_seed(4, 200 + 10 * layer + k), K, "laplace")
+                tau = synth.threshold_for_density(x, 0.4)
+                xd = torch.from_numpy(x).to(dev)
+                y = torch.empty(M, dtype=torch.float32, device=dev)
+                m.spmspv(xd, tau, y)
+                idx, _ = m.last_compaction()
+                assert m.last_status() == 0
+                tot_bytes += m.fetched_bytes(idx.cpu().numpy())[1]
+                chain.append(lambda m=m, xd=xd, tau=tau, y=y: m.spmspv(xd, tau, y))
+                Wd = torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev)
+                yd = torch.empty(M, dtype=torch.float16, device=dev)
+                dchain.append(lambda Wd=Wd, xd=xd, yd=yd: torch.mv(Wd, xd, out=yd))
+        us = rotation_us(chain) * len(shapes)
+        dus = rotation_us(dchain) * len(shapes)
+        extra["chain"] = {"calls_per_layer": len(shapes), "layers_in_rotation": 2, "us_per_layer": us,
+                          "fetched_bytes_per_layer": tot_bytes / 2, "GBps": tot_bytes / 2 / us / 1e3,
+                          "roofline_frac": tot_bytes / 2 / us / 1e3 / peak, "cublas_gemv_us_per_layer": dus,
+                          "speedup_vs_cublas": dus / us}
+    print(json.dumps({"sweep": args.sweep, "protocol": "rotation over device copies of the layer (> 2x L2) captured in one "
+                      "CUDA graph, CUDA events around the replays", "peak_GBps": peak, "points": points, **extra}))
 
 
 def run_celty(args):
@@ -496,7 +539,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS), help="time every point of a configured sweep")
-    ap.add_argument("--sweep-reps", type=int, default=30)
+    ap.add_argument("--sweep-calls", type=int, default=600, help="calls timed per sweep point (at least)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)

@@ -258,7 +258,8 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            straight from global memory) instead of the single fused launch; for the fused launch
  *            2 = merge the blocks' results through per-block partial vectors summed in a fixed
  *            order (bit-reproducible) instead of adding them into y with bulk reduce-add copies,
- *            4 = force the bulk reduce-add merge
+ *            4 = force the bulk reduce-add merge, 8 = plain launch instead of a programmatic dependent
+ *            launch (with which the kernel's set-up overlaps the tail of the previous kernel of the stream)
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   team     fused kernel: warps that share one sub-block and one accumulator (1, 2 or 4)

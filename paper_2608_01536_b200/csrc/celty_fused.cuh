@@ -299,6 +299,25 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
 
     CELTY_MARK(0);
+    // Programmatic dependent launch: let the next kernel of the stream be scheduled as this one's blocks retire,
+    // and do everything that touches neither the caller's vectors nor the workspace (warming L2 with the offset
+    // table, setting up shared memory) before waiting for the previous kernel of the stream to be complete.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // The sub-block offsets are needed right after the ranks are known: start pulling the table into L2
+    // now, each block its own share of the lines (L2 is shared by all blocks).
+    {
+        const size_t lines = (((size_t)p.K * p.S + 1) * 4 + 127) / 128;
+        const size_t per = (lines + gridDim.x - 1) / gridDim.x, l0 = (size_t)blockIdx.x * per;
+        for (size_t l = l0 + tid; l < min(lines, l0 + per); l += nthreads)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + l * 128));
+    }
+    if (tid < 4) lane_base[60 + tid] = 0;                         // the zero group of idle lanes
+    if (streams && member == 0 && lane == 0) {
+        for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     uint32_t y_ticket = 0;
     // Bulk reduce-add merge: the adds at the end need a cleared y.  The last warp clears this block's share
     // and announces it right away, so that the fence and the ticket overlap the loads of a1.
@@ -312,14 +331,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             // waiting for the lower and for the upper half.
             y_ticket = atomicInc(&p.tickets[0], 2u * gridDim.x - 1u);
         }
-    }
-    // The sub-block offsets are needed right after the ranks are known: start pulling the table into L2
-    // now, each block its own share of the lines (L2 is shared by all blocks).
-    {
-        const size_t lines = (((size_t)p.K * p.S + 1) * 4 + 127) / 128;
-        const size_t per = (lines + gridDim.x - 1) / gridDim.x, l0 = (size_t)blockIdx.x * per;
-        for (size_t l = l0 + tid; l < min(lines, l0 + per); l += nthreads)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + l * 128));
     }
     // ---- a1: threshold all of x.  A thread takes 8 activations (one 128-bit load) and makes one keep byte,
     // four neighbouring lanes assemble a keep word, and the warp scans the survivor counts of its 8 words:
@@ -374,12 +385,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         }
     }
     CELTY_MARK(10);
-    if (tid < 4) lane_base[60 + tid] = 0;                         // the zero group of idle lanes
-    if (streams && member == 0 && lane == 0) {
-        for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
     __syncthreads();
     CELTY_MARK(1);
     // ---- ranks: warp 0 turns the block counts into survivors before each block, 32 blocks at a time; the

@@ -390,12 +390,13 @@ extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, in
 extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth,
                                 int32_t team)
 {
-    if (!m || grid < 0 || variant < 0 || variant > 5 || groups < 0 || groups > 15 || depth < 0 || depth > 16 ||
+    if (!m || grid < 0 || variant < 0 || variant > 13 || groups < 0 || groups > 15 || depth < 0 || depth > 16 ||
         !(team == 0 || team == 1 || team == 2 || team == 4))
         return CELTY_EINVAL;
     m->grid = grid;
     // variant: bit 0 selects the two-launch path; 2 / 4 force the ordered two-stage / the bulk reduce-add merge
     m->merge = (variant & 2) ? 0 : (variant & 4) ? 1 : -1;
+    m->no_overlap = (variant & 8) ? 1 : 0;
     m->variant = variant & 1;
     m->groups = groups;
     m->depth = depth;

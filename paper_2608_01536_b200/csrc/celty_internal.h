@@ -97,5 +97,6 @@ struct celty_matrix {
     celty::WorkspaceLayout ws{};
     int32_t grid = 0, variant = 0, groups = 0, depth = 0, team = 0;
     int32_t last_grid = 0, last_merge = -1;   // what the tickets in the workspace were last used with
+    int32_t no_overlap = 0; // fused kernel: 1 = plain launch (no programmatic dependent launch)
     int32_t merge = -1;     // fused kernel: -1 = library's choice, 0 = ordered two-stage sum, 1 = bulk reduce-add
 };

@@ -507,8 +507,19 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
             m->last_grid = plan.grid;
             m->last_merge = plan.merge;
         }
-        k_spmspv_fused<<<plan.grid, plan.threads, plan.smem, st>>>(fp);
-        CELTY_CUDA(cudaGetLastError());
+        // Programmatic dependent launch: the kernel may be scheduled while the previous kernel of the stream
+        // drains; it waits for that kernel (griddepcontrol.wait) before it reads or writes anything of the call.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)plan.grid);
+        cfg.blockDim = dim3((unsigned)plan.threads);
+        cfg.dynamicSmemBytes = plan.smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = m->no_overlap ? 0 : 1;
+        CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused, fp));
         return CELTY_OK;
     }
     rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);
