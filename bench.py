@@ -34,7 +34,10 @@ WORKLOADS = {
     "llama7b_gateup_11008x4096_s50_a50": (11008, 4096, 0.5, "magnitude", "laplace", 0.5, 3),
     "llama7b_down_4096x11008_s50_a50": (4096, 11008, 0.5, "magnitude", "swiglu", 0.5, 3),
     "llama13b_attn_5120x5120_s50_a40": (5120, 5120, 0.5, "bernoulli", "laplace", 0.4, 4),
+    "llama13b_gateup_13824x5120_s50_a40": (13824, 5120, 0.5, "bernoulli", "laplace", 0.4, 4),
+    "llama13b_down_5120x13824_s50_a40": (5120, 13824, 0.5, "bernoulli", "laplace", 0.4, 4),
     "llama70b_mlp_28672x8192_s50_a50": (28672, 8192, 0.5, "bernoulli", "laplace", 0.5, 5),
+    "llama70b_down_8192x28672_s50_a50": (8192, 28672, 0.5, "bernoulli", "laplace", 0.5, 5),
     "small_1024x1024_s50_a50": (1024, 1024, 0.5, "bernoulli", "normal", 0.5, 1),
 }
 DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"

@@ -68,7 +68,8 @@ typedef struct {
     int32_t run_bits;    /* must be 4 (Section 3.2: "Celty uses 4-bit RLC-CSC")                      */
     int32_t layout;      /* CELTY_LAYOUT_COLUMN or CELTY_LAYOUT_LANE_TILE                             */
     int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: local rows per tile, 1..240, or 0 = choose */
-    int32_t reserved;    /* must be 0                                                                 */
+    int32_t slabs_per_block; /* LANE_TILE: slabs of rows one thread block works on, 1..15; 0 = choose (1);
+                                COLUMN: must be 0                                                         */
 } celty_encode_opts;
 
 /*

@@ -88,13 +88,14 @@ def _stream_ptr(stream):
 
 
 class _Opts(ctypes.Structure):
-    _fields_ = [("run_bits", _i32), ("layout", _i32), ("tile_rows", _i32), ("reserved", _i32)]
+    _fields_ = [("run_bits", _i32), ("layout", _i32), ("tile_rows", _i32), ("slabs_per_block", _i32)]
 
 
 class Matrix:
     """An RLC-CSC encoded weight matrix (host handle), optionally bound to device memory."""
 
-    def __init__(self, W, mask=None, layout: int = LAYOUT_LANE_TILE, tile_rows: int = 0, device=None):
+    def __init__(self, W, mask=None, layout: int = LAYOUT_LANE_TILE, tile_rows: int = 0, device=None,
+                 slabs_per_block: int = 0):
         lib = load()
         W = np.asarray(W)
         if W.dtype == np.float16:
@@ -109,7 +110,7 @@ class Matrix:
             if mask.shape != (M, K):
                 raise ValueError("mask shape")
             mptr = _np_ptr(mask)
-        opts = _Opts(4, layout, tile_rows, 0)
+        opts = _Opts(4, layout, tile_rows, slabs_per_block)
         h = _vp()
         _check(lib.celty_encode(_np_ptr(W), K, mptr, M, K, ctypes.byref(opts), ctypes.byref(h)), "celty_encode")
         self._h = h

@@ -23,7 +23,11 @@ constexpr int kMaxTileRows = 240;    // keeps local rows (and the spare rows aft
 constexpr int64_t kMaxM = 49152;     // accumulators of one thread block must fit shared memory
 constexpr size_t kAlign = 256;
 constexpr int kMaxBlocks = 192;      // blocks of the fused kernel the workspace has partial vectors for
-constexpr int kSlabsPerBlock = 4;    // LANE_TILE: a thread block covers at most this many slabs of rows
+// LANE_TILE: a thread block covers at most this many slabs of rows.  The kernels take any value; with one
+// slab per block (row parts = slabs, all of a block's warp teams work on different columns of the same rows)
+// every configured shape ran as fast or faster on B200 than with 2 or 4, mostly because a block then adds
+// fewer rows into y at the end.
+constexpr int kSlabsPerBlock = 1;
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

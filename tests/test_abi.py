@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported_and_bound(lib):
 
 def test_header_is_plain_c(tmp_path):
     src = tmp_path / "t.c"
-    src.write_text('#include "celty.h"\nint main(void){ celty_encode_opts o = {4, CELTY_LAYOUT_COLUMN, 0, 0}; return o.reserved; }\n')
+    src.write_text('#include "celty.h"\nint main(void){ celty_encode_opts o = {4, CELTY_LAYOUT_COLUMN, 0, 0}; return o.slabs_per_block; }\n')
     import subprocess
     subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), "-c", str(src),
                            "-o", str(tmp_path / "t.o")])
@@ -47,6 +47,10 @@ def test_argument_errors(lib):
         celty.Matrix(W, layout=7)
     with pytest.raises(celty.CeltyError):
         celty.Matrix(W, layout=celty.LAYOUT_LANE_TILE, tile_rows=241)
+    with pytest.raises(celty.CeltyError):
+        celty.Matrix(W, layout=celty.LAYOUT_LANE_TILE, slabs_per_block=16)
+    with pytest.raises(celty.CeltyError):
+        celty.Matrix(W, layout=celty.LAYOUT_COLUMN, slabs_per_block=1)
     h = ctypes.c_void_p()
     assert lib.celty_encode(None, 4, None, 4, 4, None, ctypes.byref(h)) == -1
     assert lib.celty_encode(W.ctypes.data_as(ctypes.c_void_p), 4, None, 0, 4, None, ctypes.byref(h)) == -1

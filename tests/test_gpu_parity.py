@@ -20,10 +20,11 @@ LAYOUTS = [(celty.LAYOUT_COLUMN, 0), (celty.LAYOUT_LANE_TILE, 0), (celty.LAYOUT_
 DECODE_LAYOUTS = [celty.LAYOUT_COLUMN, celty.LAYOUT_LANE_TILE]
 
 
-def _matrix(W, mask, lv, tile_rows=0):
+def _matrix(W, mask, lv, tile_rows=0, slabs_per_block=0):
     layout, variant = lv
-    m = celty.Matrix(W, mask, layout=layout, tile_rows=0 if layout == celty.LAYOUT_COLUMN else tile_rows,
-                     device="cuda")
+    lane = layout == celty.LAYOUT_LANE_TILE
+    m = celty.Matrix(W, mask, layout=layout, tile_rows=tile_rows if lane else 0,
+                     slabs_per_block=slabs_per_block if lane else 0, device="cuda")
     m.set_launch(variant=variant)
     m.variant = variant
     return m
@@ -147,16 +148,18 @@ def test_spmspv_random_within_bound(layout, M, K, d_w, d_a):
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
-@pytest.mark.parametrize("M,K,d_w,d_a,tile_rows", [(1000, 1003, 0.5, 0.5, 0), (4096, 512, 0.5, 0.5, 0),
-                                                    (777, 129, 0.2, 0.9, 5), (3000, 200, 0.6, 0.5, 24)])
-def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows):
+@pytest.mark.parametrize("M,K,d_w,d_a,tile_rows,spb", [(1000, 1003, 0.5, 0.5, 0, 0), (4096, 512, 0.5, 0.5, 0, 0),
+                                                        (777, 129, 0.2, 0.9, 5, 0), (3000, 200, 0.6, 0.5, 24, 0),
+                                                        (777, 129, 0.2, 0.9, 5, 2), (3000, 200, 0.6, 0.5, 24, 4),
+                                                        (11008, 96, 0.5, 0.5, 0, 2), (28672, 64, 0.4, 0.6, 0, 3)])
+def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows, spb):
     """Small-integer W and x keep every partial sum below 2^24: FP32 addition is then exact in any
     order, so the result must equal the fp64 definition bit for bit."""
     W = synth.integer_weights(M + K, M, K)
     mask = synth.mask_bernoulli(M + K, M, K, d_w)
     x = synth.integer_activations(M + K, K)
     tau = synth.threshold_for_density(x, d_a)
-    m = _matrix(W, mask, layout, tile_rows)
+    m = _matrix(W, mask, layout, tile_rows, spb)
     for grid, groups, depth, team in ((0, 0, 0, 0), (1, 0, 0, 1), (3, 1, 1, 4), (37, 3, 2, 2), (148, 2, 4, 1)):
         m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth, team=team)
         y = _run(m, x, tau)
