@@ -245,6 +245,37 @@ def test_llama7b_attention_shape_in_bench_configuration(layout):
     _check_y(_run(m, x, tau), W, mask, x, tau)
 
 
+def test_back_to_back_calls_do_not_interfere():
+    """Consecutive calls on one stream overlap at the seams (the next kernel is scheduled while the previous one
+    drains): alternate two handles and several activation vectors, reuse one output buffer for every
+    other call, and compare every result afterwards."""
+    M, K = 4096, 1536
+    mats, refs = [], []
+    for v in range(2):
+        W = synth.weights(40 + v, M, K)
+        mask = synth.mask_bernoulli(40 + v, M, K, 0.5)
+        mats.append((celty.Matrix(W, mask, device="cuda"), W, mask))
+    xs = [synth.activations(60 + i, K, "laplace") for i in range(6)]
+    taus = [synth.threshold_for_density(x, d) for x, d in zip(xs, (0.5, 0.1, 0.9, 0.3, 0.7, 0.5))]
+    xd = [_dev(x) for x in xs]
+    shared = torch.empty(M, dtype=torch.float32, device="cuda")
+    outs = []
+    for rep in range(4):
+        for i in range(6):
+            m = mats[i % 2][0]
+            if i % 2 == 0:
+                y = m.spmspv(xd[i], taus[i], y=shared)
+                outs.append((i, y.clone()))                 # the clone is ordered after the call on the stream
+            else:
+                outs.append((i, m.spmspv(xd[i], taus[i])))
+    torch.cuda.synchronize()
+    for m, _, _ in mats:
+        assert m.last_status() == 0
+    for i, y in outs:
+        _, W, mask = mats[i % 2]
+        _check_y(y.cpu().numpy(), W, mask, xs[i], taus[i])
+
+
 def test_host_buffer_entry_point():
     M, K = 1024, 1024
     W = synth.weights(1, M, K)
