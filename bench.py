@@ -206,6 +206,8 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------- sweeps (documentation runs)
 SWEEPS = {
+    # config 1: the small single layer (latency-bound; microseconds are the figure that means something)
+    "cfg1": [dict(M=1024, K=1024, s=0.5, family="bernoulli", dist="normal", d_a=0.5, cfg=1)],
     # config 2: 4096 x 4096, magnitude-pruned, all 9 (weight sparsity, activation density) pairs
     "cfg2": [dict(M=4096, K=4096, s=s, family="magnitude", dist="laplace", d_a=d, cfg=2)
              for s in (0.3, 0.5, 0.7) for d in (0.7, 0.5, 0.3)],
@@ -255,12 +257,12 @@ def run_sweep(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) * 1e3 / (reps * len(calls))
 
-    points, key, mats, dense = [], None, [], []
+    points, key, mats, dense, dense_t = [], None, [], [], []
     for i, pt in enumerate(SWEEPS[args.sweep]):
         M, K, s, fam = pt["M"], pt["K"], pt["s"], pt["family"]
         if key != (M, K, s, fam):                              # one layer on the device at a time
             key = (M, K, s, fam)
-            mats, dense = [], []
+            mats, dense, dense_t = [], [], []
             seed = synth.point_seed(pt["cfg"], 0)
             W = synth.weights(seed, M, K)
             mask = (synth.mask_magnitude(W, s) if fam == "magnitude" else
@@ -272,6 +274,7 @@ def run_sweep(args):
                 mats.append(celty.Matrix(W, mask, device=dev))
             Wm = torch.from_numpy(np.where(mask != 0, W, np.float16(0)))
             dense = [Wm.to(dev) for _ in range(min(copies, int(np.ceil(2.5 * l2 / (2 * M * K))) + 1))]
+            dense_t = [w.t().contiguous() for w in dense]
             del W, mask, Wm
         copies = len(mats)
         xs, taus = [], []
@@ -290,20 +293,24 @@ def run_sweep(args):
             survivors.append(int(idx.numel()))
         tb = float(np.mean(fetched))
         us = rotation_us([(lambda c=c: mats[c].spmspv(xs[c], taus[c], ys[c])) for c in range(copies)])
-        dus = rotation_us([(lambda c=c: torch.mv(dense[c % len(dense)], xs[c], out=yd)) for c in range(copies)])
+        dus = min(rotation_us([(lambda c=c: torch.mv(dense[c % len(dense)], xs[c], out=yd)) for c in range(copies)]),
+                  rotation_us([(lambda c=c: torch.mv(dense_t[c % len(dense_t)].t(), xs[c], out=yd)) for c in range(copies)]))
         info = mats[0].info()
         points.append({"M": M, "K": K, "weight_sparsity": s, "mask": fam, "activation_density": pt["d_a"],
                        "combined_sparsity": 1.0 - (1.0 - s) * pt["d_a"], "device_copies": copies,
                        "survivors": float(np.mean(survivors)), "stored_entries": info.nnz + info.n_pad,
                        "pads": info.n_pad, "fetched_bytes": tb, "us_per_call": us, "GBps": tb / us / 1e3,
-                       "roofline_frac": tb / us / 1e3 / peak, "cublas_gemv_us": dus, "speedup_vs_cublas": dus / us})
+                       "roofline_frac": tb / us / 1e3 / peak, "roofline_frac_of_nominal_8000": tb / us / 1e3 / 8000.0,
+                       "dense_equivalent_GBps": 2.0 * M * K / us / 1e3, "realised_weight_density": info.nnz / (M * K),
+                       "realised_activation_density": float(np.mean(survivors)) / K,
+                       "cublas_gemv_us": dus, "speedup_vs_cublas": dus / us})
         print(json.dumps(points[-1]), file=sys.stderr, flush=True)
     extra = {}
     if args.sweep == "cfg4":
         # the decode-layer chain of config 4: q, k, v, o (5120 x 5120), gate, up (13824 x 5120), down (5120 x 13824),
         # 7 calls back to back on one stream, each with its own matrix and its own synthetic x; two layers in
         # rotation (about 0.8 GB of compressed weights, far beyond L2)
-        del mats, dense
+        del mats, dense, dense_t
         shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]
         chain, dchain, tot_bytes = [], [], 0.0
         for layer in range(2):
@@ -361,7 +368,7 @@ def run_celty(args):
     copies = max(args.distinct, int(np.ceil(2.5 * l2 / image_bytes)) + 1)
     if args.copies:
         copies = args.copies
-    mats, xs, taus, fetched = [], [], [], []
+    mats, xs, taus, fetched, survivors = [], [], [], [], []
     for c in range(copies):
         W, mask = distinct[c % args.distinct]
         m = celty.Matrix(W, mask, layout=layout, tile_rows=args.tile_rows, device=dev)
@@ -382,6 +389,7 @@ def run_celty(args):
         call(c)
         idx, _ = mats[c].last_compaction()
         fetched.append(mats[c].fetched_bytes(idx.cpu().numpy()))
+        survivors.append(int(idx.numel()))
         assert mats[c].last_status() == 0
     stream_bytes = float(np.mean([f[0] for f in fetched]))
     total_bytes = float(np.mean([f[1] for f in fetched]))
@@ -460,22 +468,39 @@ def run_celty(args):
     barrier()
     e2e_sec = max_over_ranks((time.perf_counter() - t0) / n_e2e, dev)
 
-    # ---- dense cuBLAS GEMV on the same GPU, same rotation (context, not the target)
-    dense_us = None
-    if not args.no_dense:
-        Wd = [torch.from_numpy(distinct[c % args.distinct][0]).to(dev) for c in range(min(copies, 12))]
-        if len(Wd) * Wd[0].numel() * 2 < 2 * l2:
-            Wd = Wd + [w.clone() for w in Wd]
-        yd = torch.empty(M, dtype=torch.float16, device=dev)
-        gd = torch.cuda.CUDAGraph()
-        torch.mv(Wd[0], xs[0], out=yd)
+    # ---- one isolated call, host timer around call + synchronize (launch and sync latency included)
+    iso = []
+    for i in range(50):
+        c = i % copies
         torch.cuda.synchronize()
-        with torch.cuda.graph(gd):
-            for c in range(len(Wd)):
-                torch.mv(Wd[c], xs[c % copies], out=yd)
-        gd.replay()
-        dense_us = time_calls(lambda i: gd.replay(), max(3, n_ctx // len(Wd))) / len(Wd)
-        del Wd
+        t0 = time.perf_counter()
+        call(c)
+        torch.cuda.synchronize()
+        iso.append((time.perf_counter() - t0) * 1e6)
+    us_isolated = float(np.median(iso))
+
+    # ---- dense cuBLAS GEMV on the same GPU, same rotation (context, not the target): W row-major (M x K)
+    # and its transpose stored row-major (K x M), the better of the two is quoted
+    dense_us, dense_both = None, None
+    if not args.no_dense:
+        def dense_rotation(transposed):
+            Wd = [torch.from_numpy(distinct[c % args.distinct][0]).to(dev) for c in range(min(copies, 12))]
+            if transposed:
+                Wd = [w.t().contiguous() for w in Wd]
+            if len(Wd) * Wd[0].numel() * 2 < 2 * l2:
+                Wd = Wd + [w.clone() for w in Wd]
+            op = (lambda w, x, out: torch.mv(w.t(), x, out=out)) if transposed else (lambda w, x, out: torch.mv(w, x, out=out))
+            yd = torch.empty(M, dtype=torch.float16, device=dev)
+            gd = torch.cuda.CUDAGraph()
+            op(Wd[0], xs[0], yd)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(gd):
+                for c in range(len(Wd)):
+                    op(Wd[c], xs[c % copies], yd)
+            gd.replay()
+            return time_calls(lambda i: gd.replay(), max(3, n_ctx // len(Wd))) / len(Wd)
+        dense_both = {"row_major_MxK": dense_rotation(False), "transposed_KxM": dense_rotation(True)}
+        dense_us = min(dense_both.values())
 
     if rank != 0:
         if world > 1:
@@ -499,6 +524,7 @@ def run_celty(args):
                            "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad},
         "roofline": {"bound": "hbm", "achieved": total_bytes / sec_per_call / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": total_bytes / sec_per_call / 1e9 / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(name),
+                     "frac_of_nominal_8000": total_bytes / sec_per_call / 1e9 / 8000.0,
                      "peak_source": peak_src, "kernel": "k_spmspv_fused" if launches_per_step == 1 else "all kernels of the call",
                      "note": "one launch per call: algorithmic bytes per call / CUDA-event time per call"},
         "e2e": {"value": aggregate_throughput(total_bytes, world, e2e_sec), "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
@@ -506,16 +532,22 @@ def run_celty(args):
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks.summary(),
         "context": {"us_per_call_stream_enqueued": us_enqueued, "us_per_call_l2_warm": us_warm,
-                    "cublas_gemv_fp16_us": dense_us,
+                    "us_per_call_isolated_host_timer": us_isolated,
+                    "dense_equivalent_GBps": 2.0 * M * K / sec_per_call / 1e9,
+                    "survivors": float(np.mean(survivors)), "realised_activation_density": float(np.mean(survivors)) / K,
+                    "realised_weight_density": info.nnz / (M * K),
+                    "cublas_gemv_fp16_us": dense_us, "cublas_gemv_fp16_us_by_layout": dense_both,
                     "speedup_vs_cublas_gemv": (dense_us / (sec_per_call * 1e6)) if dense_us else None},
     }
     if world == 1 and not args.no_cpu:
         from oracle import celty_oracle as orc
         threads = orc.max_threads()
         sec, calls = oracle_seconds_per_call(name, args.cpu_seconds, threads)
+        sec1, calls1 = oracle_seconds_per_call(name, args.cpu_seconds / 4, 1)
         out["cpu_baseline"] = {"value": total_bytes / sec / 1e9, "unit": "GB/s", "us_per_call": sec * 1e6,
                                "cores": threads, "kind": "oracle",
-                               "sample": f"{calls} full calls of the fp64 masked product on this workload"}
+                               "sample": f"{calls} full calls of the fp64 masked product on this workload",
+                               "one_thread": {"us_per_call": sec1 * 1e6, "sample": f"{calls1} full calls"}}
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -2,22 +2,25 @@
 // anonymous namespace, after decode_group).
 //
 // One launch does the whole call (Sections 3.1-3.3):
+//   a0  the last warp of every block clears its share of y and takes a ticket (the merge at the end adds into y);
 //   a1  every block thresholds all of x (K <= a few 10k values, served by L2) into one keep bit per
-//       activation and ranks the survivors (popcounts + one warp scan); each warp team then looks up
-//       the columns whose ranks belong to it -- the list is balanced over all teams by count.  The
-//       team that owns a rank also writes it to the global list (index, value, count) for the API;
+//       activation and ranks the survivors (popcounts + warp scans); each warp team then looks up the
+//       columns whose ranks belong to it -- the list is balanced over all teams by count.  The team
+//       that owns a rank on slab 0 also writes it to the global list (index, value, count) for the API;
 //   a2  each team streams the sub-blocks (column j, slab s) of its columns from HBM into its ring of
 //       shared-memory slots with bulk asynchronous copies (cp.async.bulk + mbarrier complete_tx), D deep;
 //   a3  each lane decodes its own tile's runs on packed bytes and keeps a running row; the W warps of a
 //       team split the steps of a sub-block at the split points its header carries;
-//   a4  value * x_j is accumulated with fmaf into the lane's private bank of the team's accumulator;
-//   a5  the block adds its G accumulators and stores them as one partial vector; after a bounded
-//       grid-wide ticket barrier each block sums a share of the rows over all partials in a fixed order
-//       and stores y.  No atomics on y, no clearing of y, and the result is deterministic.
+//   a4  value * x_j is accumulated (FP16 x FP16 + FP32 fused multiply-add) into the lane's private bank of
+//       the team's accumulator;
+//   a5  the block adds its G accumulators; the row map makes a slab's accumulator a sequence of 128-row
+//       segments of y, and each goes out as one bulk reduce-add copy (FP32 add in L2) once the tickets show
+//       that every block has cleared its share of y.  Option: per-block partial vectors, a bounded
+//       grid-wide ticket barrier and a sum in a fixed order (bit-reproducible, no clearing of y).
 //
 // Rows are split over P parts (blockIdx % P) of Sc slabs each, columns over gridDim/P slices; inside a
 // block G groups take different columns, a team = (group, slab) owns one accumulator slab.  Every block
-// must be resident at once (grid <= SM count) because of the ticket barrier.  All waits are bounded:
+// must be resident at once (grid <= SM count) because of the tickets.  All waits are bounded:
 // when one runs out the kernel sets kStatusTimeout in the status word and carries on to a clean exit.
 
 struct FusedParams {
@@ -584,10 +587,9 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     CELTY_MARK(5);
 
     if (p.merge == 1) {
-        // ---- a5 by bulk reduce-add: the block adds its G accumulators, transposes each lane's tile into a
-        // row-major staging tile (stride R + 4 words keeps tiles 16-byte aligned and the stores 4-way
-        // conflicted at worst), and the copy engine adds every tile into y (cp.reduce.async.bulk, FP32 add at
-        // L2).  y was cleared by all blocks at the start; the ticket makes sure of it.
+        // ---- a5 by bulk reduce-add: the block adds its G accumulators and the copy engine adds every 128-row
+        // segment into y (cp.reduce.async.bulk, FP32 add at L2).  y was cleared by all blocks at the start; the
+        // ticket makes sure of it.
         if (warp == nwarps - 1 && lane == 0) {                      // every block's share of y is cleared by now
             const bool low_half = y_ticket < gridDim.x;
             bool ok = false;
