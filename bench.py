@@ -311,32 +311,37 @@ def run_sweep(args):
         # 7 calls back to back on one stream, each with its own matrix and its own synthetic x; two layers in
         # rotation (about 0.8 GB of compressed weights, far beyond L2)
         del mats, dense, dense_t
-        shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]
-        chain, dchain, tot_bytes = [], [], 0.0
-        for layer in range(2):
-            for k, (M, K) in enumerate(shapes):
-                seed = synth.point_seed(4, 10 * layer + k)
-                W = synth.weights(seed, M, K)
-                mask = synth.mask_bernoulli(seed, M, K, 0.5)
-                m = celty.Matrix(W, mask, device=dev)
-                x = synth.activations(synth.point_seed(4, 200 + 10 * layer + k), K, "laplace")
-                tau = synth.threshold_for_density(x, 0.4)
-                xd = torch.from_numpy(x).to(dev)
-                y = torch.empty(M, dtype=torch.float32, device=dev)
-                m.spmspv(xd, tau, y)
-                idx, _ = m.last_compaction()
-                assert m.last_status() == 0
-                tot_bytes += m.fetched_bytes(idx.cpu().numpy())[1]
-                chain.append(lambda m=m, xd=xd, tau=tau, y=y: m.spmspv(xd, tau, y))
-                Wd = torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev)
-                yd = torch.empty(M, dtype=torch.float16, device=dev)
-                dchain.append(lambda Wd=Wd, xd=xd, yd=yd: torch.mv(Wd, xd, out=yd))
-        us = rotation_us(chain) * len(shapes)
-        dus = rotation_us(dchain) * len(shapes)
-        extra["chain"] = {"calls_per_layer": len(shapes), "layers_in_rotation": 2, "us_per_layer": us,
-                          "fetched_bytes_per_layer": tot_bytes / 2, "GBps": tot_bytes / 2 / us / 1e3,
-                          "roofline_frac": tot_bytes / 2 / us / 1e3 / peak, "cublas_gemv_us_per_layer": dus,
-                          "speedup_vs_cublas": dus / us}
+        def chain(shapes, tag):
+            calls, dcalls, tot_bytes = [], [], 0.0
+            for layer in range(2):
+                for k, (M, K) in enumerate(shapes):
+                    seed = synth.point_seed(4, 10 * layer + k + (100 if tag == "stacked" else 0))
+                    W = synth.weights(seed, M, K)
+                    mask = synth.mask_bernoulli(seed, M, K, 0.5)
+                    m = celty.Matrix(W, mask, device=dev)
+                    x = synth.activations(synth.point_seed(4, 200 + 10 * layer + k), K, "laplace")
+                    tau = synth.threshold_for_density(x, 0.4)
+                    xd = torch.from_numpy(x).to(dev)
+                    y = torch.empty(M, dtype=torch.float32, device=dev)
+                    m.spmspv(xd, tau, y)
+                    idx, _ = m.last_compaction()
+                    assert m.last_status() == 0
+                    tot_bytes += m.fetched_bytes(idx.cpu().numpy())[1]
+                    calls.append(lambda m=m, xd=xd, tau=tau, y=y: m.spmspv(xd, tau, y))
+                    Wd = torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev)
+                    yd = torch.empty(M, dtype=torch.float16, device=dev)
+                    dcalls.append(lambda Wd=Wd, xd=xd, yd=yd: torch.mv(Wd, xd, out=yd))
+            us = rotation_us(calls) * len(shapes)
+            dus = rotation_us(dcalls) * len(shapes)
+            return {"calls_per_layer": len(shapes), "layers_in_rotation": 2, "us_per_layer": us,
+                    "fetched_bytes_per_layer": tot_bytes / 2, "GBps": tot_bytes / 2 / us / 1e3,
+                    "roofline_frac": tot_bytes / 2 / us / 1e3 / peak, "cublas_gemv_us_per_layer": dus,
+                    "speedup_vs_cublas": dus / us}
+        # 7 calls per layer, each product its own matrix
+        extra["chain"] = chain([(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)], "separate")
+        # the same layer with the products that share an input stacked row-wise into one matrix ([q; k; v] and
+        # [gate; up]): 4 calls per layer, one thresholding pass per shared x, for the sparse and the dense side alike
+        extra["chain_stacked"] = chain([(15360, 5120), (5120, 5120), (27648, 5120), (5120, 13824)], "stacked")
     print(json.dumps({"sweep": args.sweep, "protocol": "rotation over device copies of the layer (> 2x L2) captured in one "
                       "CUDA graph, CUDA events around the replays", "peak_GBps": peak, "points": points, **extra}))
 
