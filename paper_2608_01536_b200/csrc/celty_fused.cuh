@@ -545,14 +545,22 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 step_fetch(b1, gl, q_lo + 1, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 step_decode(b0, cell, spare, slab0, slab_end);                                    // step q_lo
                 step_fetch(b0, gl, q_lo + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                uint32_t q = q_lo + 1;
 #pragma unroll 2
-                for (uint32_t q = q_lo + 1; q <= q_hi; q += 2) {
+                for (; q + 1 < q_hi; q += 2) {                                             // two real steps per pass
                     step_decode(b1, cell, spare, slab0, slab_end);                                // step q
                     step_finish(b0, xj);                                                   // step q-1
                     step_fetch(b1, gl, q + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
                     step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
                     step_finish(b1, xj);                                                   // step q
                     step_fetch(b0, gl, q + 3, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                }
+                if (q < q_hi) {                                                            // one real step left
+                    step_decode(b1, cell, spare, slab0, slab_end);
+                    step_finish(b0, xj);
+                    step_finish(b1, xj);
+                } else {                                                                   // only the last one to finish
+                    step_finish(b0, xj);
                 }
                 const long long t_d = CELTY_CLOCK();
                 // every warp of the team is done with this sub-block (and with its rows) before the
