@@ -166,13 +166,17 @@ int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *idx_dev, uin
  * celty_spmspv -- the hot path: y = W . threshold(x, tau), batch 1 (Sections 3.1-3.3).
  * Enqueues on `stream` one kernel (LANE_TILE layout) that thresholds and compacts x, visits only
  * the surviving columns, decodes their runs to rows, accumulates value * x_j in shared memory in
- * FP32 (fmaf) and reduces the per-block partial sums into y; the COLUMN layout uses a compaction
- * kernel followed by the SpMSpV kernel.
+ * FP32 (one rounding per multiply-add) and merges the thread blocks' results into y (FP32 adds in L2
+ * by bulk reduce-add copies; celty_set_launch can select a sum in a fixed order instead); the COLUMN
+ * layout uses a compaction kernel followed by the SpMSpV kernel.  On a stream of calls the kernel's
+ * set-up overlaps the end of the previous kernel (programmatic dependent launch); it waits for that
+ * kernel before it reads x or touches y or the workspace.
  *   x_dev  K FP16 (device, 16-byte aligned), not modified
  *   y_dev  M FP32 (device, 16-byte aligned), overwritten
  * The order of FP32 additions is not fixed (Section 4.2: scatter-accumulation is order-
- * independent), so results may differ in the last bits between calls.  Inputs must be finite for
- * the result to equal the definition in every row (a pad times an infinite x_j is NaN).
+ * independent), so results may differ in the last bits between calls.  Activations must be finite
+ * for the result to equal the definition in every row: a zero-valued stored slot (a padding entry,
+ * or a slot that fills a lane's last group of 8) times an infinite or NaN x_j is NaN.
  * Errors: CELTY_EINVAL, CELTY_ESTATE, CELTY_ECUDA.  Device-side problems (a bounded wait that ran
  * out, an out-of-range index) do not fault: they set the status word, see celty_last_status.
  */

@@ -245,6 +245,31 @@ def test_llama7b_attention_shape_in_bench_configuration(layout):
     _check_y(_run(m, x, tau), W, mask, x, tau)
 
 
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_nan_activation_is_kept_and_propagates(layout):
+    """NaN fails the comparison |x| <= tau, so it survives thresholding and every row with a kept weight in that
+    column becomes NaN, as in the dense definition.  Zero-valued stored slots (padding entries, the slots that
+    fill a lane's last group) multiply the NaN too, so a few more rows may turn NaN: the method needs finite
+    activations for exact parity, and what is checked here is that nothing else is disturbed."""
+    M, K = 2000, 160
+    W = synth.weights(21, M, K)
+    mask = synth.mask_bernoulli(21, M, K, 0.5)
+    x = synth.activations(21, K, "laplace")
+    x[77] = np.float16(np.nan)
+    tau = synth.threshold_for_density(np.nan_to_num(x), 0.5)
+    m = _matrix(W, mask, layout)
+    y = _run(m, x, tau)
+    y_ref, a_ref = orc.masked_gemv(W, mask, x, tau, threads=4)
+    assert np.all(np.isnan(y)[np.isnan(y_ref)])
+    ok = ~np.isnan(y)
+    assert ok.sum() > M // 3
+    assert np.all(np.abs(y[ok].astype(np.float64) - y_ref[ok]) <= 2e-3 * a_ref[ok] + 1e-6)
+    idx, val = m.last_compaction()
+    oi, ov, _ = orc.compact(x, tau)
+    assert 77 in oi and np.array_equal(idx.cpu().numpy(), oi)
+    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+
+
 def test_back_to_back_calls_do_not_interfere():
     """Consecutive calls on one stream overlap at the seams (the next kernel is scheduled while the previous one
     drains): alternate two handles and several activation vectors, reuse one output buffer for every
