@@ -10,7 +10,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcelty.so")
 SOURCES = [os.path.join(CSRC, "celty_host.cpp"), os.path.join(CSRC, "celty_kernels.cu")]
-HEADERS = [os.path.join(CSRC, "celty_internal.h"), os.path.join(ROOT, "include", "celty.h")]
+HEADERS = [os.path.join(CSRC, "celty_internal.h"), os.path.join(CSRC, "celty_fused.cuh"),
+           os.path.join(ROOT, "include", "celty.h")]
 
 
 def needs_build() -> bool:

@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <memory>
 #include <new>
 
 #include "celty_internal.h"
@@ -177,14 +178,15 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
     if (o.layout == CELTY_LAYOUT_LANE_TILE && (o.tile_rows < 0 || o.tile_rows > kMaxTileRows)) return CELTY_EINVAL;
     *out = nullptr;
     try {
-        celty_matrix *m = new celty_matrix();
+        std::unique_ptr<celty_matrix> owner(new celty_matrix());   // released to the caller only on success
+        celty_matrix *m = owner.get();
         m->M = M; m->K = K; m->layout = o.layout;
         if (o.layout == CELTY_LAYOUT_COLUMN) {
             m->R = (int32_t)M; m->T = 1; m->S = 1;
         } else {
             choose_shape(M, o.tile_rows, &m->S, &m->R, &m->C);
             m->T = 32 * m->S;
-            if (m->S > 32) { delete m; return CELTY_EINVAL; }   // one warp per slab, 32 warps per block
+            if (m->S > 32) return CELTY_EINVAL;                 // one warp per slab, 32 warps per block
         }
         const int64_t R = m->R, T = m->T;
         const bool lane_tile = m->layout == CELTY_LAYOUT_LANE_TILE;
@@ -211,7 +213,7 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
                 }
             }
         }
-        if (total > 0xFFFFFFFFull) { delete m; return CELTY_EINVAL; }
+        if (total > 0xFFFFFFFFull) return CELTY_EINVAL;
         m->block_ptr.resize((size_t)(K * T + 1));
         uint32_t acc = 0;
         for (int64_t b = 0; b < K * T; ++b) { m->block_ptr[b] = acc; acc += cnt[b]; }
@@ -246,7 +248,7 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
         m->P = (int32_t)((m->S + spb - 1) / spb);
         m->Sc = (int32_t)((m->S + m->P - 1) / m->P);
         m->ws = workspace_layout(K, T, m->layout == CELTY_LAYOUT_LANE_TILE ? (int64_t)m->Sc * m->R * 32 : 0);
-        *out = m;
+        *out = owner.release();
         return CELTY_OK;
     } catch (const std::bad_alloc &) {
         return CELTY_ENOMEM;
