@@ -252,7 +252,7 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, items, imeta, lane_base, keep, wrel, blk, total;
+    size_t acc, ring, bars, items, imeta, lane_base, keep, wrel, blk, blkw, total;
 };
 
 __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
@@ -265,10 +265,11 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     off = (off + 15) / 16 * 16;
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
-    l.lane_base = off; off += 256;                // [32] survivors n, [33] n / units, [34] n mod units; 16 zero bytes at +240
+    l.lane_base = off; off += 256;                // scratch words; 16 zero bytes at +240
     l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
     l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 8
-    l.blk = off;       off += ((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16; // survivors before each block of 8 keep words
+    l.blk = off;       off += ((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16; // survivors in each block of 8 keep words
+    l.blkw = off;      off += 16 * (((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
     l.total = off;
     return l;
 }
@@ -294,7 +295,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
     int *lane_base = reinterpret_cast<int *>(smem + lay.lane_base);                       // see fused_smem_layout
     int *wrel = reinterpret_cast<int *>(smem + lay.wrel);                                 // [nwords]
-    int *blk = reinterpret_cast<int *>(smem + lay.blk);                                   // [nwords / 8]
+    const int *blk = reinterpret_cast<const int *>(smem + lay.blk);                       // [nwords / 8] counts
+    int *myblk = reinterpret_cast<int *>(smem + lay.blkw) + (size_t)warp * ((lay.blkw - lay.blk) / 4);   // this warp's prefix
     uint32_t *kbw = reinterpret_cast<uint32_t *>(smem + lay.keep);
 
     const int part = blockIdx.x % p.P, kslice = blockIdx.x / p.P, nK = gridDim.x / p.P;
@@ -384,15 +386,17 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 kbw[w] = word;
                 wrel[w] = incl - cnt;
             }
-            if (lane == 28 && (w >> 3) < nblk) blk[w >> 3] = incl;
+            if (lane == 28 && (w >> 3) < nblk) const_cast<int *>(blk)[w >> 3] = incl;
         }
     }
     CELTY_MARK(10);
     __syncthreads();
     CELTY_MARK(1);
-    // ---- ranks: warp 0 turns the block counts into survivors before each block, 32 blocks at a time; the
-    // list is then cut into equal shares for the groups that work on different columns.
-    if (warp == 0) {
+    // ---- ranks: every streaming warp turns the block counts into survivors before each block for itself, 32
+    // blocks at a time (a copy per warp costs a few hundred bytes and saves a block-wide barrier behind a single
+    // warp); the list is then cut into equal shares for the groups that work on different columns.
+    int n_surv = 0;
+    if (streams) {
         int carry = 0;
         for (int e0 = 0; e0 < nblk; e0 += 32) {
             const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
@@ -402,27 +406,22 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 const int up = __shfl_up_sync(kFull, incl, d);
                 if (lane >= d) incl += up;
             }
-            if (e < nblk) blk[e] = carry + incl - cnt;
+            if (e < nblk) myblk[e] = carry + incl - cnt;
             carry += __shfl_sync(kFull, incl, 31);
         }
-        if (lane == 0) {
-            // n / units without a division: units_inv = floor(2^32 / units) gives a quotient that is at most
-            // one too small
-            uint32_t share = __umulhi((uint32_t)carry, p.units_inv), extra = (uint32_t)carry - share * (uint32_t)p.units;
-            if (extra >= (uint32_t)p.units) { ++share; extra -= (uint32_t)p.units; }
-            lane_base[32] = carry;
-            lane_base[33] = (int)share;
-            lane_base[34] = (int)extra;
-            if (blockIdx.x == 0) *p.count = carry;
-        }
+        __syncwarp();
+        n_surv = carry;
+        if (blockIdx.x == 0 && warp == 0 && lane == 0) *p.count = carry;
     }
-    __syncthreads();
     CELTY_MARK(2);
 
     if (streams) {
-        // group u of nK * G owns n / units ranks, the first n mod units groups one more
-        const int u = kslice * p.G + g, share = lane_base[33], extra = lane_base[34];
-        const int r_begin = u * share + min(u, extra), r_end = r_begin + share + (u < extra ? 1 : 0);
+        // group u of nK * G owns n / units ranks, the first n mod units groups one more.  n / units without a
+        // division: units_inv = floor(2^32 / units) gives a quotient that is at most one too small
+        uint32_t share = __umulhi((uint32_t)n_surv, p.units_inv), extra = (uint32_t)n_surv - share * (uint32_t)p.units;
+        if (extra >= (uint32_t)p.units) { ++share; extra -= (uint32_t)p.units; }
+        const int u = kslice * p.G + g;
+        const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
         const int team_threads = 32 * p.W, bar_id = 1 + team;
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
         const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
@@ -448,8 +447,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 // (the last one with wrel[w] <= what is left) ...
                 int e = 0;
                 for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
-                    if (e + step < nblk && blk[e + step] <= r) e += step;
-                int k = r - blk[e], w = 8 * e;
+                    if (e + step < nblk && myblk[e + step] <= r) e += step;
+                int k = r - myblk[e], w = 8 * e;
 #pragma unroll
                 for (int step = 4; step; step >>= 1)
                     if (w + step < nwords && wrel[w + step] <= k) w += step;
