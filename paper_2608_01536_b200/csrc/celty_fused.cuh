@@ -252,7 +252,7 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, items, imeta, lane_base, keep, wrel, blk, blkw, total;
+    size_t acc, ring, bars, items, imeta, zero, keep, wrel, blk, blkw, total;
 };
 
 __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
@@ -265,7 +265,7 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     off = (off + 15) / 16 * 16;
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
-    l.lane_base = off; off += 256;                // scratch words; 16 zero bytes at +240
+    l.zero = off;      off += 16;                                          // the all-zero group that idle lanes fetch
     l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
     l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 8
     l.blk = off;       off += ((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16; // survivors in each block of 8 keep words
@@ -293,7 +293,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
     int2 *items = reinterpret_cast<int2 *>(smem + lay.items) + (size_t)team * p.cap;      // [cap] {column, x bits}
     uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
-    int *lane_base = reinterpret_cast<int *>(smem + lay.lane_base);                       // see fused_smem_layout
+    int *zero_group = reinterpret_cast<int *>(smem + lay.zero);                           // 16 bytes of zeros
     int *wrel = reinterpret_cast<int *>(smem + lay.wrel);                                 // [nwords]
     const int *blk = reinterpret_cast<const int *>(smem + lay.blk);                       // [nwords / 8] counts
     int *myblk = reinterpret_cast<int *>(smem + lay.blkw) + (size_t)warp * ((lay.blkw - lay.blk) / 4);   // this warp's prefix
@@ -316,7 +316,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         for (size_t l = l0 + tid; l < min(lines, l0 + per); l += nthreads)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + l * 128));
     }
-    if (tid < 4) lane_base[60 + tid] = 0;                         // the zero group of idle lanes
+    if (tid < 4) zero_group[tid] = 0;
     if (streams && member == 0 && lane == 0) {
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -436,7 +436,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         long long dbg_wait = 0, dbg_head = 0, dbg_loop = 0, dbg_tail = 0, dbg_steps = 0;   // development builds
         (void)dbg_wait; (void)dbg_head; (void)dbg_loop; (void)dbg_tail; (void)dbg_steps;
         StepBuf b0, b1;                                               // pipeline registers, live across items
-        const uint32_t zeros = smem_u32(lane_base) + 240u;            // 16 bytes of zeros
+        const uint32_t zeros = smem_u32(zero_group);
 
         for (int rb = r_begin; rb < r_end; rb += p.cap) {
             const int cnt = min(p.cap, r_end - rb);
