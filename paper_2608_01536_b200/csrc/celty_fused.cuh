@@ -13,7 +13,7 @@
 //       team split the steps of a sub-block at the split points its header carries;
 //   a4  value * x_j is accumulated (FP16 x FP16 + FP32 fused multiply-add) into the lane's private bank of
 //       the team's accumulator;
-//   a5  the block adds its G accumulators; the row map makes a slab's accumulator a sequence of 128-row
+//   a5  the block adds its G accumulators; the row map makes a slab's accumulator a sequence of 32*C-row
 //       segments of y, and each goes out as one bulk reduce-add copy (FP32 add in L2) once the tickets show
 //       that every block has cleared its share of y.  Option: per-block partial vectors, a bounded
 //       grid-wide ticket barrier and a sum in a fixed order (bit-reproducible, no clearing of y).
@@ -594,7 +594,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     CELTY_MARK(5);
 
     if (p.merge == 1) {
-        // ---- a5 by bulk reduce-add: the block adds its G accumulators and the copy engine adds every 128-row
+        // ---- a5 by bulk reduce-add: the block adds its G accumulators and the copy engine adds every 32*C-row
         // segment into y (cp.reduce.async.bulk, FP32 add at L2).  y was cleared by all blocks at the start; the
         // ticket makes sure of it.
         if (warp == nwarps - 1 && lane == 0) {                      // every block's share of y is cleared by now

@@ -43,11 +43,13 @@ void choose_shape(int64_t M, int tile_rows, int64_t *S_out, int32_t *R_out, int3
         S = (Q + R - 1) / R;
     } else {
         S = std::max<int64_t>(1, (M + 4095) / 4096);
-        R = std::max<int64_t>(4, ((Q + S - 1) / S + 3) / 4 * 4);
+        R = std::max<int64_t>(16, ((Q + S - 1) / S + 15) / 16 * 16);
     }
     *S_out = S;
     *R_out = (int32_t)R;
-    *C_out = R % 4 == 0 ? 4 : 1;                                      // chunks of 4 groups = 512 bytes of y
+    // chunks of 16 groups = 2 KB of consecutive rows of y: the merge adds them with one bulk copy each, and 2 KB
+    // copies measured 3-4% faster per call than 512-byte ones on the mid-size shapes
+    *C_out = R % 16 == 0 ? 16 : R % 8 == 0 ? 8 : R % 4 == 0 ? 4 : 1;
 }
 
 // Build the COLUMN image: meta uint2[K] {off16, entries}, then per column its chunks of up to 32
