@@ -7,7 +7,11 @@ A step is one celty_spmspv call (activation compaction, column fetch, run-length
 shared-memory accumulation, reduction to y) on the Llama-2-7B attention shape (4096 x 4096, W
 magnitude-pruned 50% per column, x ~ Laplace thresholded to 50% density).  Calls rotate over
 device copies of the layer whose total size exceeds twice the L2, so every call reads HBM.
-Prints ONE JSON line (see the design doc for the keys).  `--impl reference` times the CPU oracle.
+Prints ONE JSON line: the metric (achieved GB/s on the bytes a call must fetch) with microseconds per call, the
+roofline object (achieved against the measured HBM copy bandwidth, DRAM traffic from the profiler), the
+end-to-end figure through host buffers, the SM clocks sampled while timing, context (stream-enqueued, L2-warm and
+isolated timings, dense cuBLAS GEMV in both weight layouts) and the CPU oracle on the host cores.
+`--impl reference` times the CPU oracle alone; `--sweep cfgN` times every point of a configured sweep.
 """
 from __future__ import annotations
 
