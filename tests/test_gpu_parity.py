@@ -246,6 +246,22 @@ def test_llama7b_attention_shape_in_bench_configuration(layout):
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("M,K,d_a", [(300, 70001, 0.05), (96, 131072, 0.5), (2049, 40000, 0.9)])
+def test_very_wide_layers(layout, M, K, d_a):
+    """Tens of thousands of columns: several passes of the thresholding loop and several chunks of the rank scan."""
+    W = synth.weights(K + M, M, K)
+    mask = synth.mask_bernoulli(K + M, M, K, 0.5)
+    x = synth.activations(K + M, K, "laplace")
+    tau = synth.threshold_for_density(x, d_a)
+    m = _matrix(W, mask, layout)
+    _check_y(_run(m, x, tau), W, mask, x, tau)
+    idx, val = m.last_compaction()
+    oi, ov, _ = orc.compact(x, tau)
+    assert np.array_equal(idx.cpu().numpy(), oi)
+    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
 def test_nan_activation_is_kept_and_propagates(layout):
     """NaN fails the comparison |x| <= tau, so it survives thresholding and every row with a kept weight in that
     column becomes NaN, as in the dense definition.  Zero-valued stored slots (padding entries, the slots that
