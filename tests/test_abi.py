@@ -52,6 +52,8 @@ def test_argument_errors(lib):
     with pytest.raises(celty.CeltyError):
         celty.Matrix(W, layout=celty.LAYOUT_COLUMN, slabs_per_block=1)
     h = ctypes.c_void_p()
+    tall = np.zeros((49153, 1), np.float16)                      # one row more than the library takes
+    assert lib.celty_encode(tall.ctypes.data_as(ctypes.c_void_p), 1, None, 49153, 1, None, ctypes.byref(h)) == -1
     assert lib.celty_encode(None, 4, None, 4, 4, None, ctypes.byref(h)) == -1
     assert lib.celty_encode(W.ctypes.data_as(ctypes.c_void_p), 4, None, 0, 4, None, ctypes.byref(h)) == -1
     assert lib.celty_encode(W.ctypes.data_as(ctypes.c_void_p), 2, None, 4, 4, None, ctypes.byref(h)) == -1

@@ -246,6 +246,20 @@ def test_llama7b_attention_shape_in_bench_configuration(layout):
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
+def test_tallest_layer_the_library_takes(layout):
+    """M = 49152 rows (the documented limit): 12 slabs of 128 local rows."""
+    M, K = 49152, 40
+    W = synth.weights(77, M, K)
+    mask = synth.mask_bernoulli(77, M, K, 0.3)
+    x = synth.activations(77, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.7)
+    m = _matrix(W, mask, layout)
+    if layout[0] == celty.LAYOUT_LANE_TILE:
+        assert m.row_map() == (12, 128, 16)
+    _check_y(_run(m, x, tau), W, mask, x, tau)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
 @pytest.mark.parametrize("M,K,d_a", [(300, 70001, 0.05), (96, 131072, 0.5), (2049, 40000, 0.9)])
 def test_very_wide_layers(layout, M, K, d_a):
     """Tens of thousands of columns: several passes of the thresholding loop and several chunks of the rank scan."""
