@@ -344,3 +344,13 @@ def test_host_buffer_entry_point():
     ys = torch.empty(M, dtype=torch.float32, device="cuda")
     m.spmspv_host(xh, tau, yh, xs, ys)
     _check_y(yh.numpy(), W, mask, x, tau)
+    # ordinary (pageable) host memory
+    xp, yp = torch.from_numpy(x.copy()), torch.zeros(M, dtype=torch.float32)
+    m.spmspv_host(xp, tau, yp, xs, ys)
+    _check_y(yp.numpy(), W, mask, x, tau)
+    # an odd number of activations
+    Wo, mo, xo = W[:, :K - 1].copy(), mask[:, :K - 1].copy(), x[:K - 1].copy()
+    m2 = celty.Matrix(Wo, mo, device="cuda")
+    xh2 = torch.from_numpy(xo).pin_memory()
+    m2.spmspv_host(xh2, tau, yh, xs, ys)
+    _check_y(yh.numpy(), Wo, mo, xo, tau)
