@@ -42,6 +42,8 @@ WORKLOADS = {
     "llama13b_down_5120x13824_s50_a40": (5120, 13824, 0.5, "bernoulli", "laplace", 0.4, 4),
     "llama70b_mlp_28672x8192_s50_a50": (28672, 8192, 0.5, "bernoulli", "laplace", 0.5, 5),
     "llama70b_down_8192x28672_s50_a50": (8192, 28672, 0.5, "bernoulli", "laplace", 0.5, 5),
+    "llama70b_mlp_28672x8192_s30_a50": (28672, 8192, 0.3, "bernoulli", "laplace", 0.5, 5),
+    "llama70b_mlp_28672x8192_s70_a50": (28672, 8192, 0.7, "bernoulli", "laplace", 0.5, 5),
     "small_1024x1024_s50_a50": (1024, 1024, 0.5, "bernoulli", "normal", 0.5, 1),
 }
 DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"

@@ -40,8 +40,9 @@ struct FusedParams {
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // items a team looks up per batch
-    int units;                 // groups that share the survivor list: (grid / P) * G; units_inv = floor(2^32 / units)
-    uint32_t units_inv;
+    // groups that share the survivor list of a row part: units = (column slices of the part) * G;
+    // units_inv = floor(2^32 / units) for parts with grid / P slices, units_inv_long for those with one more
+    uint32_t units_inv, units_inv_long;
     int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row tiles into y
 };
 
@@ -299,7 +300,11 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     int *myblk = reinterpret_cast<int *>(smem + lay.blkw) + (size_t)warp * ((lay.blkw - lay.blk) / 4);   // this warp's prefix
     uint32_t *kbw = reinterpret_cast<uint32_t *>(smem + lay.keep);
 
-    const int part = blockIdx.x % p.P, kslice = blockIdx.x / p.P, nK = gridDim.x / p.P;
+    // Row part and column slice of this block.  The grid need not be a multiple of P: the first gridDim mod P
+    // parts then have one column slice more than the others.
+    const int part = blockIdx.x % p.P, kslice = blockIdx.x / p.P;
+    const bool long_part = part < (int)(gridDim.x % p.P);
+    const int nK = gridDim.x / p.P + (long_part ? 1 : 0);
     const int g = team / p.Sc, sl = team - g * p.Sc;
     const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
 
@@ -418,8 +423,9 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     if (streams) {
         // group u of nK * G owns n / units ranks, the first n mod units groups one more.  n / units without a
         // division: units_inv = floor(2^32 / units) gives a quotient that is at most one too small
-        uint32_t share = __umulhi((uint32_t)n_surv, p.units_inv), extra = (uint32_t)n_surv - share * (uint32_t)p.units;
-        if (extra >= (uint32_t)p.units) { ++share; extra -= (uint32_t)p.units; }
+        const uint32_t units = (uint32_t)(nK * p.G), units_inv = long_part ? p.units_inv_long : p.units_inv;
+        uint32_t share = __umulhi((uint32_t)n_surv, units_inv), extra = (uint32_t)n_surv - share * units;
+        if (extra >= units) { ++share; extra -= units; }
         const int u = kslice * p.G + g;
         const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
         const int team_threads = 32 * p.W, bar_id = 1 + team;

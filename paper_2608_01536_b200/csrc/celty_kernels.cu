@@ -421,7 +421,7 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     pl.merge = (m->merge >= 0 ? m->merge : 1);
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
-    pl.grid = std::max(1, blocks / pl.P) * pl.P;
+    pl.grid = std::max(blocks, pl.P);           // any number of blocks >= P: parts may differ by one column slice
     if (pl.grid > di.sms) return CELTY_EINVAL;
     *out = pl;
     return CELTY_OK;
@@ -499,8 +499,9 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
-        fp.units = (plan.grid / plan.P) * plan.G;
-        fp.units_inv = fp.units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / (uint64_t)fp.units);
+        auto inverse = [](uint64_t units) { return units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / units); };
+        fp.units_inv = inverse((uint64_t)(plan.grid / plan.P) * plan.G);
+        fp.units_inv_long = inverse((uint64_t)(plan.grid / plan.P + 1) * plan.G);
         // the tickets count blocks of one launch shape: start them over when the shape changes
         if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
             CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
