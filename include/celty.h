@@ -258,7 +258,7 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
 
 /*
  * celty_set_launch -- tuning knobs for experiments and tests; 0 = the library's choice.
- *   grid     thread blocks per launch (rounded down to what fits the device at once)
+ *   grid     thread blocks per launch (at most what fits the device at once, at least one per row part)
  *   variant  LANE_TILE only, a sum of: 1 = two launches (compaction kernel, then a kernel that loads
  *            straight from global memory) instead of the single fused launch; for the fused launch
  *            2 = merge the blocks' results through per-block partial vectors summed in a fixed
