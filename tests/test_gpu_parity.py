@@ -4,6 +4,8 @@ Bit-exact for the compacted list and the decoded indices; |y_gpu - y_ref| <= 2e-
 + 1e-6 per element for FP16-in / FP32-accumulate values; bit-exact too where the data make the FP32
 sum order-independent (small integers).
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -164,6 +166,37 @@ def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows, spb
         m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth, team=team)
         y = _run(m, x, tau)
         _check_y(y, W, mask, x, tau, exact=True)
+
+
+@pytest.mark.parametrize("case", range(int(os.environ.get("CELTY_RANDOM_CASES", "40"))))
+def test_random_shapes_and_options(case):
+    """Seeded draws (forty unless CELTY_RANDOM_CASES says otherwise) of shape, densities, tile rows, slabs per
+    block and launch knobs on the fused path."""
+    rng = np.random.default_rng(5000 + case)
+    M = int(rng.choice([1, 7, 31, 32, 33, 100, 255, 777, 2048, 5000, 9001]))
+    K = int(rng.choice([1, 5, 8, 31, 32, 33, 64, 200, 513, 1500]))
+    d_w = float(rng.choice([0.02, 0.2, 0.5, 0.8, 1.0]))
+    d_a = float(rng.choice([0.05, 0.3, 0.5, 0.9, 1.0]))
+    tile_rows = int(rng.choice([0, 0, 0, 1, 3, 8, 17, 48, 100, 240]))
+    spb = int(rng.choice([0, 0, 1, 2, 5]))
+    W = synth.weights(6000 + case, M, K)
+    mask = synth.mask_bernoulli(6000 + case, M, K, d_w)
+    x = synth.activations(6000 + case, K, "laplace")
+    tau = synth.threshold_for_density(x, d_a)
+    try:
+        m = celty.Matrix(W, mask, tile_rows=tile_rows, slabs_per_block=spb, device="cuda")
+    except celty.CeltyError as e:                       # more than 32 slabs: a refused option, not a failure
+        assert e.status == -1 and tile_rows > 0 and (M + 31) // 32 > 32 * tile_rows
+        return
+    grid, groups, depth, team = (int(rng.choice([0, 0, 1, 5, 40, 148])), int(rng.choice([0, 0, 1, 3])),
+                                 int(rng.choice([0, 0, 1, 3])), int(rng.choice([0, 1, 2, 4])))
+    variant = int(rng.choice([0, 0, 2, 8]))
+    m.set_launch(grid=grid, variant=variant, groups=groups, depth=depth, team=team)
+    _check_y(_run(m, x, tau), W, mask, x, tau)
+    idx, val = m.last_compaction()
+    oi, ov, _ = orc.compact(x, tau)
+    assert np.array_equal(idx.cpu().numpy(), oi)
+    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
