@@ -57,6 +57,34 @@ def test_encoder_matches_oracle(M, K, d_w, layout, tile_rows):
         assert np.array_equal(pad, opad)
 
 
+@pytest.mark.parametrize("case", range(60))
+def test_encoder_matches_oracle_on_random_draws(case):
+    """Seeded draws of shape, density and tile rows: the packed image decodes to exactly what the oracle's
+    encoder produces for the row-permuted matrix."""
+    rng = np.random.default_rng(7000 + case)
+    M = int(rng.choice([1, 5, 31, 32, 33, 63, 100, 257, 1000, 3001]))
+    K = int(rng.choice([1, 2, 7, 16]))
+    d_w = float(rng.choice([0.0, 0.03, 0.3, 0.7, 1.0]))
+    tile_rows = int(rng.choice([0, 1, 2, 5, 16, 33, 96, 240]))
+    spb = int(rng.choice([0, 1, 3]))
+    if tile_rows and (M + 31) // 32 > 32 * tile_rows:
+        tile_rows = 0
+    W = synth.weights(8000 + case, M, K)
+    mask = synth.mask_bernoulli(8000 + case, M, K, d_w)
+    m = celty.Matrix(W, mask, tile_rows=tile_rows, slabs_per_block=spb)
+    S, R, C = m.row_map()
+    assert 32 * S * R >= M and R % C == 0 and (tile_rows == 0 or R == tile_rows)
+    Wp, mp, rowmap = permute_for_lane_tiles(W, mask, S, R, C)
+    enc = orc.rlc_encode(Wp, mp, 4, tile_rows=R)
+    info = m.info()
+    assert info.nnz == int(mask.sum()) and info.n_pad == int(enc.is_pad.sum())
+    for j in range(K):
+        rows, vals, runs, pad = m.decode_host(j)
+        orows, ovals, opad, oruns = orc.column_entries(enc, j)
+        assert np.array_equal(rows, rowmap[orows])
+        assert np.array_equal(vals, ovals) and np.array_equal(runs, oruns) and np.array_equal(pad, opad)
+
+
 def test_null_mask_keeps_nonzero_weights():
     W = synth.weights(3, 100, 11)
     W[::3] = 0
