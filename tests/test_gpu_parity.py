@@ -117,6 +117,27 @@ def test_device_decode_bit_exact(layout, M, K, d_w, tile_rows):
         assert np.array_equal(vals, ovals), j
 
 
+@pytest.mark.parametrize("case", range(24))
+def test_device_decode_random_draws(case):
+    rng = np.random.default_rng(9000 + case)
+    M = int(rng.choice([1, 31, 33, 100, 777, 3001, 9001]))
+    K = int(rng.choice([1, 3, 6]))
+    d_w = float(rng.choice([0.03, 0.3, 0.7, 1.0]))
+    tile_rows = int(rng.choice([0, 0, 1, 5, 16, 96, 240]))
+    if tile_rows and (M + 31) // 32 > 32 * tile_rows:
+        tile_rows = 0
+    W = synth.weights(9500 + case, M, K)
+    mask = synth.mask_bernoulli(9500 + case, M, K, d_w)
+    m = celty.Matrix(W, mask, tile_rows=tile_rows, device="cuda")
+    S, R, C = m.row_map()
+    Wp, mp, rowmap = permute_for_lane_tiles(W, mask, S, R, C)
+    enc = orc.rlc_encode(Wp, mp, 4, tile_rows=R)
+    for j in range(K):
+        rows, vals = m.decode_device(j)
+        orows, ovals, _, _ = orc.column_entries(enc, j)
+        assert np.array_equal(rows, rowmap[orows]) and np.array_equal(vals, ovals)
+
+
 # ----------------------------------------------------------------------------- product
 SHAPES = [
     # M, K, d_w, d_a
