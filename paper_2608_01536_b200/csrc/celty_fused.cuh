@@ -342,8 +342,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             y_ticket = atomicInc(&p.tickets[0], 2u * gridDim.x - 1u);
         }
     }
-    // ---- a1: threshold all of x.  A thread takes 8 activations (one 128-bit load) and makes one keep byte,
-    // four neighbouring lanes assemble a keep word, and the warp scans the survivor counts of its 8 words:
+    // ---- a1: threshold all of x.  A thread takes 32 activations (four 128-bit loads) and makes one keep word,
+    // and eight neighbouring lanes scan the survivor counts of their block of 8 words:
     //   kbw[w]  keep bits of activations 32w .. 32w+31,
     //   wrel[w] survivors in the words before w of the same block of 8 words,
     //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
@@ -351,47 +351,49 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 7) >> 3;
     {
         const __half2 tau2 = __half2half2(__float2half_rd(p.tau));
-        for (int q0 = 0; q0 < nwords * 4; q0 += nthreads) {       // the same trip count for every thread
-            const int q = q0 + tid;
-            uint32_t keep = 0;
-            if (q < ngroups) {
-                uint32_t h[4];
-                if (8 * q + 8 <= p.K) {
-                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p.x + 8 * q));
-                    h[0] = v.x; h[1] = v.y; h[2] = v.z; h[3] = v.w;
-                } else {
+        for (int w0 = 0; w0 < nwords; w0 += nthreads) {             // the same trip count for every thread
+            const int w = w0 + tid;
+            uint32_t word = 0;
+            if (w < nwords) {
+                uint32_t h[4][4];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint32_t lo = (8 * q + 2 * k < p.K) ? p.x[8 * q + 2 * k] : 0u;
-                        const uint32_t hi = (8 * q + 2 * k + 1 < p.K) ? p.x[8 * q + 2 * k + 1] : 0u;
-                        h[k] = lo | (hi << 16);
+                for (int c = 0; c < 4; ++c) {                          // four independent 128-bit loads per thread
+                    const int q = 4 * w + c;
+                    h[c][0] = h[c][1] = h[c][2] = h[c][3] = 0u;        // zero past the end of x: never kept (tau >= 0)
+                    if (8 * q + 8 <= p.K) {
+                        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p.x + 8 * q));
+                        h[c][0] = v.x; h[c][1] = v.y; h[c][2] = v.z; h[c][3] = v.w;
+                    } else if (q < ngroups) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const uint32_t lo = (8 * q + 2 * k < p.K) ? p.x[8 * q + 2 * k] : 0u;
+                            const uint32_t hi = (8 * q + 2 * k + 1 < p.K) ? p.x[8 * q + 2 * k + 1] : 0u;
+                            h[c][k] = lo | (hi << 16);
+                        }
                     }
                 }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const __half2 a = __habs2(*reinterpret_cast<const __half2 *>(&h[k]));
-                    const __half2 le = __hle2(a, tau2);            // 1.0 where |x| <= tau (false for NaN)
-                    const uint32_t bits = *reinterpret_cast<const uint32_t *>(&le);
-                    if ((bits & 0xFFFFu) == 0 && 8 * q + 2 * k < p.K) keep |= 1u << (2 * k);
-                    if ((bits >> 16) == 0 && 8 * q + 2 * k + 1 < p.K) keep |= 2u << (2 * k);
-                }
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        // 0xFFFF in a half where |x| <= tau (false for NaN); the keep bits are the complement
+                        const uint32_t le = __hle2_mask(__habs2(*reinterpret_cast<const __half2 *>(&h[c][k])), tau2);
+                        word |= ((~le & 1u) | ((~le >> 15) & 2u)) << (8 * c + 2 * k);
+                    }
+                if (32 * w + 32 > p.K) word &= (32 * w < p.K) ? (0xFFFFFFFFu >> (32 * w + 32 - p.K)) : 0u;
             }
-            uint32_t word = keep << (8 * (lane & 3));
-            word |= __shfl_xor_sync(kFull, word, 1);
-            word |= __shfl_xor_sync(kFull, word, 2);
-            const int cnt = (lane & 3) == 0 ? __popc(word) : 0;
+            const int cnt = __popc(word);
             int incl = cnt;
 #pragma unroll
-            for (int d = 4; d < 32; d <<= 1) {
-                const int up = __shfl_up_sync(kFull, incl, d);
-                if (lane >= d) incl += up;
+            for (int d = 1; d < 8; d <<= 1) {                          // scan within the block of 8 words
+                const int up = __shfl_up_sync(kFull, incl, d, 8);
+                if ((lane & 7) >= d) incl += up;
             }
-            const int w = q >> 2;
-            if ((lane & 3) == 0 && w < nwords) {
+            if (w < nwords) {
                 kbw[w] = word;
                 wrel[w] = incl - cnt;
             }
-            if (lane == 28 && (w >> 3) < nblk) const_cast<int *>(blk)[w >> 3] = incl;
+            if ((lane & 7) == 7 && (w >> 3) < nblk) const_cast<int *>(blk)[w >> 3] = incl;
         }
     }
     CELTY_MARK(10);
