@@ -268,9 +268,9 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
     l.zero = off;      off += 16;                                          // the all-zero group that idle lanes fetch
     l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
-    l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 8
-    l.blk = off;       off += ((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16; // survivors in each block of 8 keep words
-    l.blkw = off;      off += 16 * (((size_t)((K + 255) / 256) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
+    l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 32
+    l.blk = off;       off += ((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16; // survivors in each block of 32 keep words
+    l.blkw = off;      off += 16 * (((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
     l.total = off;
     return l;
 }
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
     int *zero_group = reinterpret_cast<int *>(smem + lay.zero);                           // 16 bytes of zeros
     int *wrel = reinterpret_cast<int *>(smem + lay.wrel);                                 // [nwords]
-    const int *blk = reinterpret_cast<const int *>(smem + lay.blk);                       // [nwords / 8] counts
+    const int *blk = reinterpret_cast<const int *>(smem + lay.blk);                       // [nwords / 32] counts
     int *myblk = reinterpret_cast<int *>(smem + lay.blkw) + (size_t)warp * ((lay.blkw - lay.blk) / 4);   // this warp's prefix
     uint32_t *kbw = reinterpret_cast<uint32_t *>(smem + lay.keep);
 
@@ -343,12 +343,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         }
     }
     // ---- a1: threshold all of x.  A thread takes 32 activations (four 128-bit loads) and makes one keep word,
-    // and eight neighbouring lanes scan the survivor counts of their block of 8 words:
+    // and the warp scans the survivor counts of its block of 32 words:
     //   kbw[w]  keep bits of activations 32w .. 32w+31,
-    //   wrel[w] survivors in the words before w of the same block of 8 words,
+    //   wrel[w] survivors in the words before w of the same block of 32 words,
     //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
-    const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 7) >> 3;
+    const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 31) >> 5;
     {
         const __half2 tau2 = __half2half2(__float2half_rd(p.tau));
         for (int w0 = 0; w0 < nwords; w0 += nthreads) {             // the same trip count for every thread
@@ -385,15 +385,15 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             const int cnt = __popc(word);
             int incl = cnt;
 #pragma unroll
-            for (int d = 1; d < 8; d <<= 1) {                          // scan within the block of 8 words
-                const int up = __shfl_up_sync(kFull, incl, d, 8);
-                if ((lane & 7) >= d) incl += up;
+            for (int d = 1; d < 32; d <<= 1) {                         // scan within the block of 32 words
+                const int up = __shfl_up_sync(kFull, incl, d);
+                if (lane >= d) incl += up;
             }
             if (w < nwords) {
                 kbw[w] = word;
                 wrel[w] = incl - cnt;
             }
-            if ((lane & 7) == 7 && (w >> 3) < nblk) const_cast<int *>(blk)[w >> 3] = incl;
+            if (lane == 31 && (w >> 5) < nblk) const_cast<int *>(blk)[w >> 5] = incl;
         }
     }
     CELTY_MARK(10);
@@ -451,14 +451,14 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             // ---- column of rank r: the lane whose words hold it, then the word, then the bit
             for (int i = member * 32 + lane; i < cnt; i += team_threads) {
                 const int r = rb + i;
-                // the block of 8 keep words that holds rank r (the last one with blk[e] <= r), the word in it
+                // the block of 32 keep words that holds rank r (the last one with blk[e] <= r), the word in it
                 // (the last one with wrel[w] <= what is left) ...
                 int e = 0;
                 for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
                     if (e + step < nblk && myblk[e + step] <= r) e += step;
-                int k = r - myblk[e], w = 8 * e;
+                int k = r - myblk[e], w = 32 * e;
 #pragma unroll
-                for (int step = 4; step; step >>= 1)
+                for (int step = 16; step; step >>= 1)
                     if (w + step < nwords && wrel[w + step] <= k) w += step;
                 k -= wrel[w];
                 // ... and the bit in it: halve the word, keep the half that holds the wanted set bit
