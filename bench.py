@@ -52,7 +52,7 @@ DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"
 # summarised under profiles/ (small-case captures of the same kernel and workload).
 NCU_DRAM_BYTES_PER_LAUNCH = {
     "llama7b_attn_4096x4096_s50_a50": 11.57e6,
-    "llama70b_mlp_28672x8192_s50_a50": 166.4e6,
+    "llama70b_mlp_28672x8192_s50_a50": 165.3e6,
 }
 
 
