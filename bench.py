@@ -352,6 +352,113 @@ def run_sweep(args):
                       "CUDA graph, CUDA events around the replays", "peak_GBps": peak, "points": points, **extra}))
 
 
+def run_format_study(args):
+    """Compression efficiency against weight sparsity (the paper's Figure 3 question, on synthetic Bernoulli
+    masks): bytes of the 4-bit run-length format as the library's host encoder writes it, for the whole-column
+    layout and for the lane-tile device image, beside the closed form 1.25 * d * (1 + rho) (rho = pads per
+    nonzero = s^16 / (1 - s^16)) and a bitmap format's d + 1/16.  Host only: no GPU is needed."""
+    from paper_2608_01536_b200 import build as lib_build, celty
+    lib_build.build()
+    celty.load()
+    M, K = 4096, 1024
+    rows = []
+    for s in (0.1, 0.2, 0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9, 0.95):
+        seed = synth.point_seed(2, 900 + int(round(s * 100)))
+        W = synth.weights(seed, M, K)
+        mask = synth.mask_bernoulli(seed, M, K, 1.0 - s)
+        dense_bytes = 2.0 * M * K
+        out = {"weight_sparsity": s}
+        for name, layout in (("column", celty.LAYOUT_COLUMN), ("lane_tile", celty.LAYOUT_LANE_TILE)):
+            m = celty.Matrix(W, mask, layout=layout)
+            info = m.info()
+            out[name] = {"image_over_dense": m.device_bytes()[0] / dense_bytes,
+                         "entries_over_dense": 2.5 * (info.nnz + info.n_pad) / dense_bytes,
+                         "pads_per_nonzero": info.n_pad / max(1, info.nnz)}
+            out["realised_density"] = info.nnz / (M * K)
+        d = 1.0 - s
+        rho = s ** 16 / (1.0 - s ** 16)
+        out["closed_form_rlc4"] = 1.25 * d * (1.0 + rho)
+        out["closed_form_bitmap"] = d + 1.0 / 16.0
+        rows.append(out)
+        print(json.dumps(out), file=sys.stderr, flush=True)
+    print(json.dumps({"sweep": "format", "M": M, "K": K, "mask": "bernoulli", "points": rows}))
+
+
+def run_knob_study(args):
+    """Launch-parameter study (the paper's Figure 11 question -- how far to split the columns -- asked of this
+    kernel): time of one workload against the number of thread blocks (column slices = blocks / row parts),
+    warp teams per block, ring depth and warps per team, everything else the library's choice.  Same protocol as
+    the sweeps: rotation over device copies beyond 2x L2, one CUDA graph, CUDA events."""
+    import torch
+    from paper_2608_01536_b200 import build as lib_build, celty
+    lib_build.build()
+    celty.load()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    name = args.workload
+    W, mask = make_layer(name, 0)
+    first = celty.Matrix(W, mask, device=dev)
+    copies = int(np.ceil(2.5 * l2 / first.device_bytes()[0])) + 1
+    mats = [first] + [celty.Matrix(W, mask, device=dev) for _ in range(copies - 1)]
+    xs, taus = [], []
+    for c in range(copies):
+        x, tau = make_x(name, c)
+        xs.append(torch.from_numpy(x).to(dev))
+        taus.append(tau)
+    ys = [torch.empty(W.shape[0], dtype=torch.float32, device=dev) for _ in range(copies)]
+    S = first.row_map()[0]
+
+    def timed(**kn):
+        for m in mats:
+            m.set_launch(**kn)
+        calls = [(lambda c=c: mats[c].spmspv(xs[c], taus[c], ys[c])) for c in range(copies)]
+        for f in calls:
+            f()
+        torch.cuda.synchronize()
+        if any(m.last_status() != 0 for m in mats):
+            return None
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for f in calls:
+                f()
+        g.replay()
+        torch.cuda.synchronize()
+        reps = max(3, -(-args.sweep_calls // copies))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / (reps * copies)
+
+    points = []
+    def add(knob, value, **kn):
+        try:
+            us = timed(**kn)
+        except celty.CeltyError as e:                       # a setting that does not fit the device is refused
+            us = None
+            print(f"{knob}={value}: {e}", file=sys.stderr)
+        points.append({"knob": knob, "value": value, "us_per_call": us})
+        print(json.dumps(points[-1]), file=sys.stderr, flush=True)
+
+    add("default", 0)
+    for grid in sorted({max(S, sms // 8), max(S, sms // 4), max(S, sms // 2), max(S, 3 * sms // 4), sms}):
+        add("grid", grid, grid=grid)
+    for groups in (1, 2, 4, 6, 8):
+        add("groups", groups, groups=groups)
+    for depth in (2, 3, 4):
+        add("depth", depth, depth=depth)
+    for team in (1, 2, 4):
+        add("team", team, team=team)
+    for m in mats:
+        m.set_launch()
+    print(json.dumps({"sweep": "knobs", "workload": name, "row_parts": int(S), "device_copies": copies,
+                      "points": points}))
+
+
 def run_celty(args):
     import torch
     import torch.distributed as dist
@@ -584,10 +691,16 @@ def main():
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
-    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS), help="time every point of a configured sweep")
+    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS) + ["format", "knobs"],
+                    help="time every point of a configured sweep; format = compression study on the host; "
+                         "knobs = launch-parameter study of --workload")
     ap.add_argument("--sweep-calls", type=int, default=600, help="calls timed per sweep point (at least)")
     args = ap.parse_args()
-    if args.sweep:
+    if args.sweep == "format":
+        run_format_study(args)
+    elif args.sweep == "knobs":
+        run_knob_study(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -22,3 +22,22 @@ def test_reference_arm_prints_one_json_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     assert d["cpu_baseline"]["value"] == d["value"] == d["e2e"]["value"] > 0
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_format_study_matches_the_closed_form():
+    """Section 3.2: a stored entry costs 2.5 bytes against 2 dense, and a gap of more than 15 rows costs one
+    padding entry per 16 rows.  On Bernoulli masks of density d = 1 - s that is 1.25 * d * (1 + rho) of the dense
+    size with rho = s^16 / (1 - s^16); the host encoder's entry counts must land on it (sampling noise only)."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--sweep", "format"], capture_output=True,
+                         text=True, timeout=600, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
+    assert d["sweep"] == "format" and len(d["points"]) >= 9
+    for pt in d["points"]:
+        s = pt["weight_sparsity"]
+        want = 1.25 * pt["realised_density"] * (1.0 + s ** 16 / (1.0 - s ** 16))
+        assert abs(pt["column"]["entries_over_dense"] - want) < 0.004 * max(want, 0.25), pt
+        # the lane-tile image pays for headers and for filling each lane's last group of 8
+        assert pt["lane_tile"]["image_over_dense"] > pt["lane_tile"]["entries_over_dense"]
+    half = [pt for pt in d["points"] if pt["weight_sparsity"] == 0.5][0]
+    assert abs(half["column"]["entries_over_dense"] - 0.625) < 0.002          # "about 63 %" at 50 % sparsity
