@@ -299,6 +299,29 @@ def test_llama7b_attention_shape_in_bench_configuration(layout):
     _check_y(_run(m, x, tau), W, mask, x, tau)
 
 
+def test_llama70b_mlp_shape_in_bench_configuration():
+    """28672 x 8192, Bernoulli mask at 50%, Laplace activations kept at 50%: the large workload bench.py times, at
+    full size in the launch configuration it is timed in, every row compared and the list bit for bit.  (The weights
+    repeat a 28672 x 1024 block eight times along K to keep the generator's time down; the mask does not repeat,
+    so no two columns hold the same entries.)"""
+    M, K = 28672, 8192
+    seed = synth.point_seed(5, 3)
+    W = np.tile(synth.weights(seed, M, K // 8), (1, 8))
+    mask = synth.mask_bernoulli(seed, M, K, 0.5)
+    x = synth.activations(seed, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.5)
+    m = _matrix(W, mask, (celty.LAYOUT_LANE_TILE, 0))
+    assert m.row_map() == (8, 112, 16)
+    y = _run(m, x, tau)
+    _check_y(y, W, mask, x, tau)
+    idx, val = m.last_compaction()
+    oi, ov, _ = orc.compact(x, tau)
+    assert np.array_equal(idx.cpu().numpy(), oi)
+    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+    # a second call on the same handle (tickets wrap around) gives the same rows within the bound
+    _check_y(_run(m, x, tau), W, mask, x, tau)
+
+
 @pytest.mark.parametrize("layout", LAYOUTS)
 def test_tallest_layer_the_library_takes(layout):
     """M = 49152 rows (the documented limit): 12 slabs of 128 local rows."""
