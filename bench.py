@@ -356,7 +356,8 @@ def run_format_study(args):
     """Compression efficiency against weight sparsity (the paper's Figure 3 question, on synthetic Bernoulli
     masks): bytes of the 4-bit run-length format as the library's host encoder writes it, for the whole-column
     layout and for the lane-tile device image, beside the closed form 1.25 * d * (1 + rho) (rho = pads per
-    nonzero = s^16 / (1 - s^16)) and a bitmap format's d + 1/16.  Host only: no GPU is needed."""
+    nonzero = s^16 / (1 - s^16)) and a bitmap format's d + 1/16; and the entry counts at run widths of 2 to 8 bits
+    (celty_count_entries), which show where the paper's 4 bits sit.  Host only: no GPU is needed."""
     from paper_2608_01536_b200 import build as lib_build, celty
     lib_build.build()
     celty.load()
@@ -378,6 +379,16 @@ def run_format_study(args):
         d = 1.0 - s
         rho = s ** 16 / (1.0 - s ** 16)
         out["closed_form_rlc4"] = 1.25 * d * (1.0 + rho)
+        # the same question for other run widths n (why 4 bits?): entries counted by the library at width n,
+        # (2 + n / 8) bytes each, beside the closed form d * (1 + s^L / (1 - s^L)) * (2 + n / 8) / 2, L = 2^n
+        out["run_width"] = {}
+        for n in (2, 3, 4, 5, 6, 8):
+            nnz, pads = celty.count_entries(mask, n)
+            L = 2 ** n
+            out["run_width"][str(n)] = {"entries_over_dense": (2.0 + n / 8.0) * (nnz + pads) / dense_bytes,
+                                        "pads_per_nonzero": pads / max(1, nnz),
+                                        "closed_form": d * (1.0 + s ** L / (1.0 - s ** L)) * (2.0 + n / 8.0) / 2.0}
+        out["best_run_width"] = min(out["run_width"], key=lambda k: out["run_width"][k]["entries_over_dense"])
         out["closed_form_bitmap"] = d + 1.0 / 16.0
         rows.append(out)
         print(json.dumps(out), file=sys.stderr, flush=True)

@@ -251,6 +251,19 @@ int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx_host, int64_t 
                         int64_t *total_bytes);
 
 /*
+ * celty_count_entries -- how many entries the format of Section 3.2 would store for a mask if its
+ * runs were `run_bits` wide (1..8), whole columns, without building anything: the kept positions
+ * (nnz) and the padding entries the rule inserts (a gap of g dropped rows costs floor(g / 2^run_bits)
+ * of them; rows after a column's last kept row cost nothing).  An entry then takes 2 + run_bits / 8
+ * bytes.  This is the quantity behind the paper's choice of 4-bit runs (Section 3.2, Figure 3); the
+ * encoder itself takes 4 bits only.  mask_host: M x K row-major, `ldm` bytes from row to row,
+ * nonzero = kept.  Host-only.  Errors: CELTY_EINVAL (null mask, M or K <= 0, ldm < K, run_bits
+ * outside 1..8), CELTY_ENOMEM.
+ */
+int celty_count_entries(const uint8_t *mask_host, int64_t ldm, int64_t M, int64_t K, int run_bits, int64_t *nnz,
+                        int64_t *n_pad);
+
+/*
  * celty_last_status -- synchronises `stream`, reads the workspace status word and clears it.
  * Returns CELTY_OK, CELTY_ETIMEOUT or CELTY_EBOUNDS (or CELTY_ECUDA / CELTY_ESTATE).
  */

@@ -39,6 +39,8 @@ SIGNATURES = {
     "celty_last_compaction": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
     "celty_decode_device": (ctypes.c_int, [_vp, _i64, _vp, _vp, _i64, _vp, _vp]),
     "celty_fetched_bytes": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "celty_count_entries": (ctypes.c_int, [_vp, _i64, _i64, _i64, ctypes.c_int, ctypes.POINTER(_i64),
+                                           ctypes.POINTER(_i64)]),
     "celty_last_status": (ctypes.c_int, [_vp, _vp]),
     "celty_set_launch": (ctypes.c_int, [_vp, _i32, _i32, _i32, _i32, _i32]),
     "celty_last_cuda_error": (ctypes.c_int, []),
@@ -257,3 +259,14 @@ def compact(x, tau: float, stream=None):
                                 _stream_ptr(stream)), "celty_compact")
     n = int(cnt.item())
     return idx[:n], val[:n]
+
+
+def count_entries(mask, run_bits: int = 4):
+    """(kept positions, padding entries) the whole-column format would store for `mask` (M x K, nonzero =
+    kept) with runs of `run_bits` bits; an entry then takes 2 + run_bits / 8 bytes.  Host only."""
+    mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+    M, K = mask.shape
+    nnz, pad = _i64(), _i64()
+    _check(load().celty_count_entries(_np_ptr(mask), K, M, K, int(run_bits), ctypes.byref(nnz), ctypes.byref(pad)),
+           "celty_count_entries")
+    return nnz.value, pad.value

@@ -413,6 +413,35 @@ extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, in
     return CELTY_OK;
 }
 
+extern "C" int celty_count_entries(const uint8_t *mask, int64_t ldm, int64_t M, int64_t K, int run_bits,
+                                   int64_t *nnz, int64_t *n_pad)
+{
+    if (!mask || M <= 0 || K <= 0 || ldm < K || run_bits < 1 || run_bits > 8) return CELTY_EINVAL;
+    // rows outermost (the mask is row-major); gap[j] = dropped rows of column j since its last kept row
+    std::vector<int64_t> gap;
+    try {
+        gap.assign((size_t)K, 0);
+    } catch (const std::bad_alloc &) {
+        return CELTY_ENOMEM;
+    }
+    int64_t kept = 0, pads = 0;
+    for (int64_t i = 0; i < M; ++i) {
+        const uint8_t *row = mask + i * ldm;
+        for (int64_t j = 0; j < K; ++j) {
+            if (!row[j]) {
+                ++gap[(size_t)j];
+                continue;
+            }
+            ++kept;
+            pads += gap[(size_t)j] >> run_bits;      // a padding entry covers 2^run_bits rows: its run and itself
+            gap[(size_t)j] = 0;
+        }
+    }
+    if (nnz) *nnz = kept;
+    if (n_pad) *n_pad = pads;
+    return CELTY_OK;
+}
+
 extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth,
                                 int32_t team)
 {

@@ -41,3 +41,13 @@ def test_format_study_matches_the_closed_form():
         assert pt["lane_tile"]["image_over_dense"] > pt["lane_tile"]["entries_over_dense"]
     half = [pt for pt in d["points"] if pt["weight_sparsity"] == 0.5][0]
     assert abs(half["column"]["entries_over_dense"] - 0.625) < 0.002          # "about 63 %" at 50 % sparsity
+    # other run widths: the library's entry counts sit on the closed form, width 4 is the encoder's own count, and
+    # 4 bits are the smallest format in the range the paper prunes to (70 - 80 %), 3 bits at 50 - 60 %
+    for pt in d["points"]:
+        for n, v in pt["run_width"].items():
+            # (the rows after a column's last kept row store nothing, which the closed form ignores: up to half a
+            # per cent fewer padding entries at 2 bits and 95 % sparsity with 4096 rows)
+            assert abs(v["entries_over_dense"] - v["closed_form"]) < 0.008 * max(v["closed_form"], 0.25), (pt, n)
+        assert abs(pt["run_width"]["4"]["entries_over_dense"] - pt["column"]["entries_over_dense"]) < 1e-12
+    best = {pt["weight_sparsity"]: pt["best_run_width"] for pt in d["points"]}
+    assert best[0.7] == "4" and best[0.8] == "4" and best[0.5] == "3" and best[0.3] == "2" and best[0.95] == "6"

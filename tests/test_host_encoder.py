@@ -145,3 +145,37 @@ def test_fetched_bytes_accounting():
     assert abs(sb - 2.5 * n_j.sum()) <= 2.5 * 8 * idx.size + 16 * idx.size
     assert tb == sb + 8 * idx.size + 2 * K + 6 * idx.size + 4 * M
     assert m.fetched_bytes(np.zeros(0, np.int32)) == (0, 2 * K + 4 * M)
+
+
+@pytest.mark.parametrize("run_bits", [1, 2, 3, 4, 5, 6, 8])
+def test_entry_count_per_run_width_matches_oracle_encoder(run_bits):
+    """celty_count_entries against the number of entries the oracle's encoder really emits at that run width,
+    on Bernoulli and row-clustered masks, an empty matrix, a dense one and single-entry columns."""
+    masks = []
+    for M, K, d in ((257, 19, 0.5), (1000, 37, 0.1), (4097, 5, 0.02), (64, 7, 1.0), (300, 9, 0.0)):
+        masks.append(synth.mask_bernoulli(M * 3 + K, M, K, d))
+    masks.append(synth.mask_powerlaw(11, 2000, 13, 0.3))
+    last = np.zeros((777, 3), dtype=np.uint8)
+    last[776, 0] = last[255, 1] = last[256, 2] = 1                 # gaps of 776, 255 and 256 rows
+    masks.append(last)
+    for mask in masks:
+        M, K = mask.shape
+        enc = orc.rlc_encode(np.ones((M, K), dtype=np.float16), mask, run_bits=run_bits)
+        nnz = int(np.count_nonzero(mask))
+        assert celty.count_entries(mask, run_bits) == (nnz, len(enc.runs) - nnz)
+    # by hand: a column whose only kept row is 776 needs floor(776 / 2^n) padding entries
+    assert celty.count_entries(last[:, :1], run_bits) == (1, 776 >> run_bits)
+
+
+def test_entry_count_rejects_bad_arguments():
+    import ctypes
+    lib = celty.load()
+    mask = np.ones((4, 4), dtype=np.uint8)
+    p = mask.ctypes.data_as(ctypes.c_void_p)
+    n = ctypes.c_int64()
+    assert lib.celty_count_entries(None, 4, 4, 4, 4, ctypes.byref(n), None) == -1
+    assert lib.celty_count_entries(p, 4, 4, 4, 0, ctypes.byref(n), None) == -1
+    assert lib.celty_count_entries(p, 4, 4, 4, 9, ctypes.byref(n), None) == -1
+    assert lib.celty_count_entries(p, 3, 4, 4, 4, ctypes.byref(n), None) == -1
+    assert lib.celty_count_entries(p, 4, 0, 4, 4, ctypes.byref(n), None) == -1
+    assert lib.celty_count_entries(p, 4, 4, 4, 4, ctypes.byref(n), None) == 0 and n.value == 16
