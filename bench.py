@@ -51,8 +51,8 @@ DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_spmspv_fused launch, from the ncu captures
 # summarised under profiles/ (small-case captures of the same kernel and workload).
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "llama7b_attn_4096x4096_s50_a50": 11.57e6,
-    "llama70b_mlp_28672x8192_s50_a50": 165.3e6,
+    "llama7b_attn_4096x4096_s50_a50": 11.58e6,
+    "llama70b_mlp_28672x8192_s50_a50": 166.0e6,
 }
 
 
