@@ -3,14 +3,18 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl celty|reference] [--workload NAME]
 
-A step is one celty_spmspv call (activation compaction, column fetch, run-length decode,
-shared-memory accumulation, reduction to y) on the Llama-2-7B attention shape (4096 x 4096, W
-magnitude-pruned 50% per column, x ~ Laplace thresholded to 50% density).  Calls rotate over
-device copies of the layer whose total size exceeds twice the L2, so every call reads HBM.
+A step is one celty_spmspv call (activation compaction, column fetch, run-length decode, shared-memory
+accumulation, reduction to y).  The default workload is the largest single-GPU configuration, the
+Llama-70B-shaped MLP layer 28672 x 8192 (Bernoulli mask, 50% of the weights kept, x ~ Laplace thresholded to
+50% density); the Llama-2-7B attention shape 4096 x 4096 is timed beside it as a second, labelled figure.
+Calls rotate over device copies of the layer whose total size exceeds twice the L2, so every call reads HBM.
+The K steps are whole replays of one CUDA graph between two CUDA events; that region is taken at least ten
+times and the median is reported, so a short run gives the same microseconds per call as a long one.
 Prints ONE JSON line: the metric (achieved GB/s on the bytes a call must fetch) with microseconds per call, the
-roofline object (achieved against the measured HBM copy bandwidth, DRAM traffic from the profiler), the
-end-to-end figure through host buffers, the SM clocks sampled while timing, context (stream-enqueued, L2-warm and
-isolated timings, dense cuBLAS GEMV in both weight layouts) and the CPU oracle on the host cores.
+roofline object (achieved against the measured HBM copy bandwidth, DRAM traffic from the profiler, the dense
+cuBLAS GEMV under the same rotation and the speed-up over it, the second workload), the end-to-end figure
+through host buffers, the SM clocks sampled while timing, context (stream-enqueued, L2-warm and isolated
+timings) and the CPU oracle on the host cores.
 `--impl reference` times the CPU oracle alone; `--sweep cfgN` times every point of a configured sweep.
 """
 from __future__ import annotations
@@ -46,20 +50,15 @@ WORKLOADS = {
     "llama70b_mlp_28672x8192_s70_a50": (28672, 8192, 0.7, "bernoulli", "laplace", 0.5, 5),
     "small_1024x1024_s50_a50": (1024, 1024, 0.5, "bernoulli", "normal", 0.5, 1),
 }
-DEFAULT_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"
-
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_spmspv_fused launch, from the ncu captures
-# summarised under profiles/ (small-case captures of the same kernel and workload).
-NCU_DRAM_BYTES_PER_LAUNCH = {
-    "llama7b_attn_4096x4096_s50_a50": 11.58e6,
-    "llama70b_mlp_28672x8192_s50_a50": 166.0e6,
-}
-
+DEFAULT_WORKLOAD = "llama70b_mlp_28672x8192_s50_a50"     # the largest single-GPU configuration: the headline
+SECONDARY_WORKLOAD = "llama7b_attn_4096x4096_s50_a50"    # a second, labelled figure (latency-bound)
 
 def make_layer(name: str, variant: int):
     M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
     seed = synth.point_seed(cfg, variant)
-    W = synth.weights(seed, M, K)
+    # the largest layers repeat a block of K/8 columns of weights along K (drawing 235 M normals takes minutes);
+    # their masks are drawn in full, so no two columns hold the same entries
+    W = synth.weights_tiled(seed, M, K, K // 8) if M * K > (1 << 26) else synth.weights(seed, M, K)
     if family == "magnitude":
         mask = synth.mask_magnitude(W, s)
     elif family == "bernoulli":
@@ -73,6 +72,19 @@ def make_x(name: str, variant: int):
     M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
     x = synth.activations(synth.point_seed(cfg, 50 + variant), K, dist)
     return x, synth.threshold_for_density(x, d_a)
+
+
+L2_POLICY = ("inputs larger than L2: on the GPU, calls rotate over enough device copies of the layer (each with its own "
+             "activation vector) to exceed 2x the L2 capacity, so every call reads HBM")
+
+
+def workload_config(name):
+    """The `config` object of the JSON line: what defines the workload, identical for both --impl arms."""
+    M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
+    return {"workload": name, "M": M, "K": K, "weight_sparsity": s, "mask": family, "activations": dist,
+            "activation_density": d_a,
+            "weights": "N(0, 0.02^2) block of K/8 columns repeated along K, mask not repeated" if M * K > (1 << 26)
+            else "N(0, 0.02^2)", "l2": L2_POLICY}
 
 
 class ClockSampler:
@@ -152,11 +164,9 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-def oracle_seconds_per_call(name: str, budget_s: float, threads: int):
+def oracle_seconds_per_call(W, mask, x, tau, budget_s: float, threads: int):
     """The oracle's plain definition on the bench workload, repeated for about budget_s seconds."""
     from oracle import celty_oracle as orc
-    W, mask = make_layer(name, 0)
-    x, tau = make_x(name, 0)
     orc.masked_gemv(W[:64], mask[:64], x, tau, threads=threads)          # load the library
     t0 = time.perf_counter()
     calls = 0
@@ -169,11 +179,12 @@ def oracle_seconds_per_call(name: str, budget_s: float, threads: int):
 
 
 def run_reference(args):
-    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only).  Nothing of the CUDA
+    library is loaded: the byte numerator is the format's own count (2.5 bytes per stored entry of the surviving
+    columns from the oracle encoder's block pointers, two pointer words per surviving column, x, the list, y)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle import celty_oracle as orc
-    from paper_2608_01536_b200 import build as lib_build, celty
     name = args.workload
     M, K, s, family, dist, d_a, cfg = WORKLOADS[name]
     W, mask = make_layer(name, 0)
@@ -193,10 +204,9 @@ def run_reference(args):
         orc.masked_gemv(Ws, ms, x, tau, threads=threads)
     dt = (time.perf_counter() - t0) / args.steps
     sec_per_call = dt * (M / rows)
-    # bytes the GPU path would fetch for this call: host-side table arithmetic of the library
-    lib_build.build()
     idx = orc.compact(x, tau)[0]
-    total_bytes = celty.Matrix(W, mask).fetched_bytes(idx)[1]
+    ptr = orc.rlc_count(np.ascontiguousarray(mask[:, idx]), 4, 0)
+    total_bytes = 2.5 * float(ptr[-1]) + 8.0 * idx.size + 2.0 * K + 6.0 * idx.size + 4.0 * M
     gbs = total_bytes / sec_per_call / 1e9
     sample = f"rows 0..{rows - 1} of {M} per step, scaled to a full call"
     print(json.dumps({
@@ -204,7 +214,8 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_per_call * 1e3,
         "us_per_call": sec_per_call * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": name, "M": M, "K": K, "weight_sparsity": s, "activation_density": d_a},
+        "config": workload_config(name),
+        "bytes_per_call": {"bare_format": total_bytes},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -270,14 +281,14 @@ def run_sweep(args):
             key = (M, K, s, fam)
             mats, dense, dense_t = [], [], []
             seed = synth.point_seed(pt["cfg"], 0)
-            W = synth.weights(seed, M, K)
+            W = synth.weights_tiled(seed, M, K, K // 8) if M * K > (1 << 26) else synth.weights(seed, M, K)
             mask = (synth.mask_magnitude(W, s) if fam == "magnitude" else
                     synth.mask_bernoulli(seed, M, K, 1.0 - s) if fam == "bernoulli" else
                     synth.mask_powerlaw(seed, M, K, 1.0 - s))
             mats.append(celty.Matrix(W, mask, device=dev))
             copies = int(np.ceil(2.5 * l2 / mats[0].device_bytes()[0])) + 1
             while len(mats) < copies:
-                mats.append(celty.Matrix(W, mask, device=dev))
+                mats.append(mats[0].clone(device=dev))
             Wm = torch.from_numpy(np.where(mask != 0, W, np.float16(0)))
             dense = [Wm.to(dev) for _ in range(min(copies, int(np.ceil(2.5 * l2 / (2 * M * K))) + 1))]
             dense_t = [w.t().contiguous() for w in dense]
@@ -412,7 +423,7 @@ def run_knob_study(args):
     W, mask = make_layer(name, 0)
     first = celty.Matrix(W, mask, device=dev)
     copies = int(np.ceil(2.5 * l2 / first.device_bytes()[0])) + 1
-    mats = [first] + [celty.Matrix(W, mask, device=dev) for _ in range(copies - 1)]
+    mats = [first] + [first.clone(device=dev) for _ in range(copies - 1)]
     xs, taus = [], []
     for c in range(copies):
         x, tau = make_x(name, c)
@@ -470,6 +481,148 @@ def run_knob_study(args):
                       "points": points}))
 
 
+def pick_copies(needed: int, steps: int) -> int:
+    """Device copies in the rotation: the smallest count >= needed that divides `steps` (so that every timed
+    region of `steps` calls walks the rotation a whole number of times and a copy is never reused early);
+    `needed` itself when no divisor is close."""
+    for c in range(needed, 2 * needed + 5):
+        if steps % c == 0:
+            return c
+    return needed
+
+
+def graph_unit(copies: int, steps: int, cap: int = 256) -> int:
+    """Calls held by the CUDA graph: a whole number of rotations, at most `cap` calls, dividing `steps` when
+    the rotation does (the timed region is then whole replays and nothing else)."""
+    if steps % copies:
+        return steps if steps <= 4 * cap else copies
+    rotations = steps // copies
+    k = max(1, min(rotations, cap // copies))
+    while rotations % k:
+        k -= 1
+    return copies * k
+
+
+class Workload:
+    """One configured layer resident `copies` times on the device (every copy its own activation vector), the
+    CUDA graph that walks the rotation, and the byte accounting of a call."""
+
+    def __init__(self, name, dev, args, steps, celty, torch):
+        self.name = name
+        M, K, s, family, dist_name, d_a, cfg = WORKLOADS[name]
+        self.M, self.K = M, K
+        layout = celty.LAYOUT_COLUMN if args.layout == "column" else celty.LAYOUT_LANE_TILE
+        self.l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+        distinct_n = max(1, min(args.distinct, 1 if M * K > (1 << 26) else args.distinct))
+        self.distinct = [make_layer(name, v) for v in range(distinct_n)]
+        base = [celty.Matrix(W, mask, layout=layout, tile_rows=args.tile_rows) for W, mask in self.distinct]
+        self.image_bytes = base[0].device_bytes()[0]
+        needed = max(distinct_n, int(np.ceil(2.5 * self.l2 / self.image_bytes)) + 1)
+        self.copies = args.copies if args.copies else pick_copies(needed, steps)
+        self.mats, self.xs, self.taus = [], [], []
+        for c in range(self.copies):
+            m = base[c % distinct_n] if c < distinct_n else base[c % distinct_n].clone()
+            m.to(dev)
+            if args.grid or args.variant or args.groups or args.depth:
+                m.set_launch(args.grid, args.variant, args.groups, args.depth)
+            x, tau = make_x(name, c)
+            self.mats.append(m)
+            self.xs.append(torch.from_numpy(x).to(dev))
+            self.taus.append(tau)
+        self.ys = [torch.empty(M, dtype=torch.float32, device=dev) for _ in range(self.copies)]
+        torch.cuda.synchronize()
+        # bytes per call: host arithmetic on the library's tables, from the list the call itself produced
+        fetched, entries, self.survivors = [], [], []
+        for c in range(self.copies):
+            self.call(c)
+            idx, _ = self.mats[c].last_compaction()
+            assert self.mats[c].last_status() == 0
+            idx = idx.cpu().numpy()
+            fetched.append(self.mats[c].fetched_bytes(idx))
+            entries.append(self.mats[c].stored_entries(idx))
+            self.survivors.append(int(idx.size))
+        self.stream_bytes = float(np.mean([f[0] for f in fetched]))
+        self.total_bytes = float(np.mean([f[1] for f in fetched]))
+        n = float(np.mean(self.survivors))
+        # the format's own bytes: 2.5 per stored entry of the surviving columns, two offset words per column,
+        # x read, the list written, y written -- no alignment padding, no per-block headers
+        self.bare_bytes = 2.5 * float(np.mean(entries)) + 8 * n + 2 * K + 6 * n + 4 * M
+        self.info = self.mats[0].info()
+        self.graph = None
+        self.unit = None
+
+    def call(self, c):
+        self.mats[c].spmspv(self.xs[c], self.taus[c], self.ys[c])
+
+    def capture(self, torch, steps):
+        self.unit = graph_unit(self.copies, steps)
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            for i in range(self.unit):
+                self.call(i % self.copies)
+        for _ in range(2):
+            self.graph.replay()
+        torch.cuda.synchronize()
+
+
+def timed_regions(torch, replay, replays_per_region, min_regions=10, min_total_s=0.25, max_regions=400):
+    """CUDA-event time (ms) of regions of `replays_per_region` graph replays each.  An untimed replay is queued
+    directly ahead of every region, so the opening event is taken while the device is busy and the first timed
+    kernel starts behind it without a launch gap; the regions are independent samples of the same K steps."""
+    times = []
+    t0 = time.perf_counter()
+    while len(times) < min_regions or (time.perf_counter() - t0 < min_total_s and len(times) < max_regions):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        replay()
+        a.record()
+        for _ in range(replays_per_region):
+            replay()
+        b.record()
+        b.synchronize()
+        times.append(a.elapsed_time(b))
+    return times
+
+
+def dense_gemv_us(torch, wl, dev, steps):
+    """Dense cuBLAS FP16 GEMV on the same masked weights under the same rotation: W row-major (M x K) and its
+    transpose stored row-major (K x M); microseconds per call of each."""
+    out = {}
+    n_dense = max(2, int(np.ceil(2.5 * wl.l2 / (2.0 * wl.M * wl.K))) + 1)
+    Wm = [torch.from_numpy(np.where(mask != 0, W, np.float16(0))) for W, mask in wl.distinct]
+    base = [w.to(dev) for w in Wm]
+    for transposed in (False, True):
+        Wd = [base[c % len(base)].clone() for c in range(n_dense)]
+        if transposed:
+            Wd = [w.t().contiguous() for w in Wd]
+        op = (lambda w, x, o: torch.mv(w.t(), x, out=o)) if transposed else (lambda w, x, o: torch.mv(w, x, out=o))
+        yd = torch.empty(wl.M, dtype=torch.float16, device=dev)
+        op(Wd[0], wl.xs[0], yd)
+        torch.cuda.synchronize()
+        unit = n_dense * max(1, min(64, steps) // n_dense)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(unit):
+                op(Wd[i % n_dense], wl.xs[i % wl.copies], yd)
+        g.replay()
+        torch.cuda.synchronize()
+        reps = max(1, steps // unit)
+        out["transposed_KxM" if transposed else "row_major_MxK"] = \
+            float(np.median(timed_regions(torch, g.replay, reps, min_total_s=0.1))) * 1e3 / (reps * unit)
+        del Wd, g
+    return out
+
+
+def dram_traffic_per_launch(name):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused kernel on this workload, from the
+    profiler capture summarised under profiles/ (kept as data next to the summaries); None when there is none."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(name, {}).get("dram_bytes_per_launch")
+    except OSError:
+        return None
+
+
 def run_celty(args):
     import torch
     import torch.distributed as dist
@@ -487,81 +640,39 @@ def run_celty(args):
     dev = torch.device("cuda", local)
     name = args.workload
     M, K, s, family, dist_name, d_a, cfg = WORKLOADS[name]
-    layout = celty.LAYOUT_COLUMN if args.layout == "column" else celty.LAYOUT_LANE_TILE
-
-    # ---- workload: a few distinct matrices, replicated on the device until the copies exceed 2x L2
-    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
-    distinct = [make_layer(name, v) for v in range(args.distinct)]
-    probe = celty.Matrix(*distinct[0], layout=layout, tile_rows=args.tile_rows)
-    image_bytes = probe.device_bytes()[0]
-    copies = max(args.distinct, int(np.ceil(2.5 * l2 / image_bytes)) + 1)
-    if args.copies:
-        copies = args.copies
-    mats, xs, taus, fetched, survivors = [], [], [], [], []
-    for c in range(copies):
-        W, mask = distinct[c % args.distinct]
-        m = celty.Matrix(W, mask, layout=layout, tile_rows=args.tile_rows, device=dev)
-        if args.grid or args.variant or args.groups or args.depth or args.team:
-            m.set_launch(args.grid, args.variant, args.groups, args.depth, args.team)
-        x, tau = make_x(name, c)
-        mats.append(m)
-        xs.append(torch.from_numpy(x).to(dev))
-        taus.append(tau)
-    ys = [torch.empty(M, dtype=torch.float32, device=dev) for _ in range(copies)]
-    torch.cuda.synchronize()
-
-    def call(c):
-        mats[c].spmspv(xs[c], taus[c], ys[c])
-
-    # bytes per call (host arithmetic on the library's tables, from the oracle-free compacted list)
-    for c in range(copies):
-        call(c)
-        idx, _ = mats[c].last_compaction()
-        fetched.append(mats[c].fetched_bytes(idx.cpu().numpy()))
-        survivors.append(int(idx.numel()))
-        assert mats[c].last_status() == 0
-    stream_bytes = float(np.mean([f[0] for f in fetched]))
-    total_bytes = float(np.mean([f[1] for f in fetched]))
-    info = mats[0].info()
+    steps = args.steps
+    warmup = max(3, args.warmup)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- warm-up, then one CUDA graph holding one rotation over all copies
-    for i in range(max(3, args.warmup)):
-        call(i % copies)
+    wl = Workload(name, dev, args, steps, celty, torch)
+    for i in range(warmup):
+        wl.call(i % wl.copies)
     torch.cuda.synchronize()
-    graph = None
-    if not args.no_graph:
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            for c in range(copies):
-                call(c)
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-    reps, rem = (args.steps // copies, args.steps % copies) if graph is not None else (0, args.steps)
+    if args.no_graph:
+        def replay():
+            for i in range(steps):
+                wl.call(i % wl.copies)
+        per_region = 1
+    else:
+        wl.capture(torch, steps)
+        replay, per_region = wl.graph.replay, max(1, steps // wl.unit)
+    calls_per_region = steps if args.no_graph else per_region * wl.unit
 
-    def timed_region():
-        for _ in range(reps):
-            graph.replay()
-        for i in range(rem):
-            call(i % copies)
-
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- the timed region: K steps as whole graph replays between two CUDA events, taken several times over;
+    # the median region is the figure, the fastest and the count are reported beside it
     with ClockSampler(local) as clocks:
         barrier()
-        e0.record()
-        timed_region()
-        e1.record()
+        regions = timed_regions(torch, replay, per_region)
         barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1), dev)
-    sec_per_call = ms / 1e3 / args.steps
-    gbs = aggregate_throughput(total_bytes, world, sec_per_call)
+    ms = max_over_ranks(float(np.median(regions)), dev)
+    sec_per_call = ms / 1e3 / calls_per_region
+    gbs = aggregate_throughput(wl.total_bytes, world, sec_per_call)
 
-    # ---- stream-enqueued (no graph) and L2-warm numbers, for context
+    # ---- context: stream-enqueued calls (no graph) and the L2-warm figure
     def time_calls(fn, n):
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -571,109 +682,116 @@ def run_celty(args):
         b.record()
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n * 1e3
-    n_ctx = min(args.steps, 2000)
-    us_enqueued = time_calls(lambda i: call(i % copies), n_ctx)
-    us_warm = None
-    if graph is not None:
-        gw = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gw):
-            for _ in range(copies):
-                call(0)
-        gw.replay()
-        us_warm = time_calls(lambda i: gw.replay(), max(1, n_ctx // copies)) / copies
+    n_ctx = int(min(max(steps, 200), 2000))
+    us_enqueued = time_calls(lambda i: wl.call(i % wl.copies), n_ctx)
+    gw = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gw):
+        for _ in range(16):
+            wl.call(0)
+    gw.replay()
+    us_warm = float(np.median(timed_regions(torch, gw.replay, 4, min_total_s=0.05))) * 1e3 / 64
 
     # ---- end to end through the host-buffer entry point: pinned x in, y out, every step
-    xh = [torch.from_numpy(make_x(name, c)[0]).pin_memory() for c in range(copies)]
+    xh = [torch.from_numpy(make_x(name, c)[0]).pin_memory() for c in range(wl.copies)]
     yh = torch.empty(M, dtype=torch.float32).pin_memory()
     xstage = torch.empty(K, dtype=torch.float16, device=dev)
-    n_e2e = min(args.steps, 2000)
+    n_e2e = int(min(max(steps, 200), 2000))
     for i in range(5):
-        mats[i % copies].spmspv_host(xh[i % copies], taus[i % copies], yh, xstage, ys[0])
+        wl.mats[i % wl.copies].spmspv_host(xh[i % wl.copies], wl.taus[i % wl.copies], yh, xstage, wl.ys[0])
     barrier()
     t0 = time.perf_counter()
     for i in range(n_e2e):
-        c = i % copies
-        mats[c].spmspv_host(xh[c], taus[c], yh, xstage, ys[0])
+        c = i % wl.copies
+        wl.mats[c].spmspv_host(xh[c], wl.taus[c], yh, xstage, wl.ys[0])
     barrier()
     e2e_sec = max_over_ranks((time.perf_counter() - t0) / n_e2e, dev)
 
     # ---- one isolated call, host timer around call + synchronize (launch and sync latency included)
     iso = []
     for i in range(50):
-        c = i % copies
+        c = i % wl.copies
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        call(c)
+        wl.call(c)
         torch.cuda.synchronize()
         iso.append((time.perf_counter() - t0) * 1e6)
     us_isolated = float(np.median(iso))
 
-    # ---- dense cuBLAS GEMV on the same GPU, same rotation (context, not the target): W row-major (M x K)
-    # and its transpose stored row-major (K x M), the better of the two is quoted
-    dense_us, dense_both = None, None
-    if not args.no_dense:
-        def dense_rotation(transposed):
-            Wd = [torch.from_numpy(distinct[c % args.distinct][0]).to(dev) for c in range(min(copies, 12))]
-            if transposed:
-                Wd = [w.t().contiguous() for w in Wd]
-            if len(Wd) * Wd[0].numel() * 2 < 2 * l2:
-                Wd = Wd + [w.clone() for w in Wd]
-            op = (lambda w, x, out: torch.mv(w.t(), x, out=out)) if transposed else (lambda w, x, out: torch.mv(w, x, out=out))
-            yd = torch.empty(M, dtype=torch.float16, device=dev)
-            gd = torch.cuda.CUDAGraph()
-            op(Wd[0], xs[0], yd)
-            torch.cuda.synchronize()
-            with torch.cuda.graph(gd):
-                for c in range(len(Wd)):
-                    op(Wd[c], xs[c % copies], yd)
-            gd.replay()
-            return time_calls(lambda i: gd.replay(), max(3, n_ctx // len(Wd))) / len(Wd)
-        dense_both = {"row_major_MxK": dense_rotation(False), "transposed_KxM": dense_rotation(True)}
-        dense_us = min(dense_both.values())
+    # ---- dense cuBLAS GEMV on the same GPU under the same rotation: the better weight layout is quoted
+    dense_both = None if args.no_dense else dense_gemv_us(torch, wl, dev, steps)
+    dense_us = min(dense_both.values()) if dense_both else None
+
+    # ---- a second, labelled figure: the Llama-2-7B attention shape (latency-bound), same protocol
+    secondary = None
+    if not args.no_secondary and name != SECONDARY_WORKLOAD and world == 1:
+        w2 = Workload(SECONDARY_WORKLOAD, dev, args, 240, celty, torch)
+        w2.capture(torch, 240)
+        us2 = float(np.median(timed_regions(torch, w2.graph.replay, max(1, 240 // w2.unit), min_total_s=0.1))) \
+            * 1e3 / (max(1, 240 // w2.unit) * w2.unit)
+        d2 = None if args.no_dense else min(dense_gemv_us(torch, w2, dev, 240).values())
+        secondary = {"workload": SECONDARY_WORKLOAD, "us_per_call": us2, "bytes_per_call": w2.total_bytes,
+                     "achieved": w2.total_bytes / us2 / 1e3, "device_copies": w2.copies,
+                     "dense_gemv_us": d2, "speedup_vs_dense_gemv": (d2 / us2) if d2 else None}
+        del w2
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
     peak, peak_src = measured_peaks()
-    launches_per_step = 1 if (layout == celty.LAYOUT_LANE_TILE and args.variant == 0) else 2
+    if secondary:
+        secondary["frac"] = secondary["achieved"] / peak
+    launches_per_step = 1 if (args.layout != "column" and (args.variant & 1) == 0) else 2
+    us_per_call = sec_per_call * 1e6
+    info = wl.info
     out = {
-        "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": sec_per_call * 1e3, "us_per_call": sec_per_call * 1e6,
+        "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": sec_per_call * 1e3, "us_per_call": us_per_call,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {
-            "workload": name, "M": M, "K": K, "weight_sparsity": s, "mask": family, "activations": dist_name,
-            "activation_density": d_a, "layout": "column" if layout == celty.LAYOUT_COLUMN else "lane_tile",
-            "tile_rows": info.tile_rows, "l2": f"rotation over {copies} device copies ({args.distinct} distinct "
-            f"matrices, {copies} distinct x), {copies * image_bytes / 1e6:.0f} MB > 2x L2 ({l2 / 1e6:.0f} MB)",
-            "launch": "cuda graph of one rotation" if graph is not None else "stream enqueue",
+        "config": workload_config(name),
+        "run": {
+            "layout": args.layout, "tile_rows": info.tile_rows,
+            "l2": f"rotation over {wl.copies} device copies ({len(wl.distinct)} distinct matrices, {wl.copies} distinct "
+                  f"x), {wl.copies * wl.image_bytes / 1e6:.0f} MB > 2x L2 ({wl.l2 / 1e6:.0f} MB)",
+            "launch": "stream enqueue" if args.no_graph else f"cuda graph of {wl.unit} calls",
+            "timing": f"median of {len(regions)} regions of {calls_per_region} calls (whole graph replays between two "
+                      "CUDA events, an untimed replay queued ahead of each region)",
             "multi_gpu": "replicas only" if world > 1 else "single",
         },
-        "bytes_per_call": {"entry_stream": stream_bytes, "total": total_bytes, "dense_fp16": 2.0 * M * K,
+        "bytes_per_call": {"entry_stream": wl.stream_bytes, "total": wl.total_bytes, "bare_format": wl.bare_bytes,
+                           "total_over_bare": wl.total_bytes / wl.bare_bytes, "dense_fp16": 2.0 * M * K,
                            "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad},
-        "roofline": {"bound": "hbm", "achieved": total_bytes / sec_per_call / 1e9, "peak": peak, "unit": "GB/s",
-                     "frac": total_bytes / sec_per_call / 1e9 / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(name),
-                     "frac_of_nominal_8000": total_bytes / sec_per_call / 1e9 / 8000.0,
-                     "peak_source": peak_src, "kernel": "k_spmspv_fused" if launches_per_step == 1 else "all kernels of the call",
-                     "note": "one launch per call: algorithmic bytes per call / CUDA-event time per call"},
-        "e2e": {"value": aggregate_throughput(total_bytes, world, e2e_sec), "unit": "GB/s", "us_per_call": e2e_sec * 1e6,
-                "h2d_bytes_per_step": 2 * K, "d2h_bytes_per_step": 4 * M},
-        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": wl.total_bytes / sec_per_call / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": wl.total_bytes / sec_per_call / 1e9 / peak, "traffic": dram_traffic_per_launch(name),
+                     "frac_on_bare_format_bytes": wl.bare_bytes / sec_per_call / 1e9 / peak,
+                     "frac_of_nominal_8000": wl.total_bytes / sec_per_call / 1e9 / 8000.0,
+                     "peak_source": peak_src,
+                     "kernel": "k_spmspv_fused" if launches_per_step == 1 else "all kernels of the call",
+                     "note": "one launch per call: algorithmic bytes per call / CUDA-event time per call",
+                     "us_per_call": us_per_call, "us_per_call_fastest_region": min(regions) * 1e3 / calls_per_region,
+                     "dense_gemv_us": dense_us, "dense_gemv_us_by_layout": dense_both,
+                     "speedup_vs_dense_gemv": (dense_us / us_per_call) if dense_us else None,
+                     "combined_sparsity": 1.0 - (1.0 - s) * d_a,
+                     "secondary": secondary},
+        "e2e": {"value": aggregate_throughput(wl.total_bytes, world, e2e_sec), "unit": "GB/s",
+                "us_per_call": e2e_sec * 1e6, "h2d_bytes_per_step": 2 * K, "d2h_bytes_per_step": 4 * M},
+        "gpu_launches": launches_per_step * calls_per_region,
         "clocks": clocks.summary(),
         "context": {"us_per_call_stream_enqueued": us_enqueued, "us_per_call_l2_warm": us_warm,
                     "us_per_call_isolated_host_timer": us_isolated,
                     "dense_equivalent_GBps": 2.0 * M * K / sec_per_call / 1e9,
-                    "survivors": float(np.mean(survivors)), "realised_activation_density": float(np.mean(survivors)) / K,
-                    "realised_weight_density": info.nnz / (M * K),
-                    "cublas_gemv_fp16_us": dense_us, "cublas_gemv_fp16_us_by_layout": dense_both,
-                    "speedup_vs_cublas_gemv": (dense_us / (sec_per_call * 1e6)) if dense_us else None},
+                    "survivors": float(np.mean(wl.survivors)),
+                    "realised_activation_density": float(np.mean(wl.survivors)) / K,
+                    "realised_weight_density": info.nnz / (M * K), "regions_ms": [round(r, 5) for r in regions[:40]]},
     }
     if world == 1 and not args.no_cpu:
         from oracle import celty_oracle as orc
         threads = orc.max_threads()
-        sec, calls = oracle_seconds_per_call(name, args.cpu_seconds, threads)
-        sec1, calls1 = oracle_seconds_per_call(name, args.cpu_seconds / 4, 1)
-        out["cpu_baseline"] = {"value": total_bytes / sec / 1e9, "unit": "GB/s", "us_per_call": sec * 1e6,
+        W0, mask0 = wl.distinct[0]
+        x0, tau0 = make_x(name, 0)
+        sec, calls = oracle_seconds_per_call(W0, mask0, x0, tau0, args.cpu_seconds, threads)
+        sec1, calls1 = oracle_seconds_per_call(W0, mask0, x0, tau0, args.cpu_seconds / 4, 1)
+        out["cpu_baseline"] = {"value": wl.total_bytes / sec / 1e9, "unit": "GB/s", "us_per_call": sec * 1e6,
                                "cores": threads, "kind": "oracle",
                                "sample": f"{calls} full calls of the fp64 masked product on this workload",
                                "one_thread": {"us_per_call": sec1 * 1e6, "sample": f"{calls1} full calls"}}
@@ -696,11 +814,11 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--groups", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
-    ap.add_argument("--team", type=int, default=0)
     ap.add_argument("--tile-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the second, labelled workload")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS) + ["format", "knobs"],
                     help="time every point of a configured sweep; format = compression study on the host; "

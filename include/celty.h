@@ -65,7 +65,7 @@ typedef enum {
 enum { CELTY_LAYOUT_COLUMN = 0, CELTY_LAYOUT_LANE_TILE = 1 };
 
 typedef struct {
-    int32_t run_bits;    /* must be 4 (Section 3.2: "Celty uses 4-bit RLC-CSC")                      */
+    int32_t run_bits;    /* must be 4, the run width Section 3.2 settles on (Figure 3)               */
     int32_t layout;      /* CELTY_LAYOUT_COLUMN or CELTY_LAYOUT_LANE_TILE                             */
     int32_t tile_rows;   /* COLUMN: must be 0.  LANE_TILE: local rows per tile, 1..240, or 0 = choose */
     int32_t slabs_per_block; /* LANE_TILE: slabs of rows one thread block works on, 1..15; 0 = choose (1);
@@ -92,6 +92,14 @@ int celty_encode(const uint16_t *W_host, int64_t ldw, const uint8_t *mask_host, 
 
 /* Frees the handle and its host memory.  Device buffers stay with the caller.  NULL is allowed. */
 void celty_destroy(celty_matrix *m);
+
+/*
+ * celty_clone -- a second handle holding a copy of the encoded matrix (host memory only; the copy is not
+ * bound to device memory and has the library's default launch settings), for callers that want the same
+ * layer resident several times (one binding per handle) without packing it again.
+ * Errors: CELTY_EINVAL, CELTY_ENOMEM.
+ */
+int celty_clone(const celty_matrix *m, celty_matrix **out);
 
 /*
  * celty_info -- sizes of the encoded matrix.  Any output pointer may be NULL.
@@ -249,6 +257,14 @@ int celty_decode_device(celty_matrix *m, int64_t col, int32_t *rows_dev, uint16_
  */
 int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx_host, int64_t n, int64_t *stream_bytes,
                         int64_t *total_bytes);
+
+/*
+ * celty_stored_entries -- stored entries (kept weights + padding entries, Section 3.2) of the n listed
+ * columns (host array of indices): times 2.5 bytes this is what the format itself makes a call fetch for
+ * those columns, before any alignment padding or per-block header of the device image.  Host-only.
+ * Errors: CELTY_EINVAL.
+ */
+int celty_stored_entries(const celty_matrix *m, const int32_t *idx_host, int64_t n, int64_t *entries);
 
 /*
  * celty_count_entries -- how many entries the format of Section 3.2 would store for a mask if its

@@ -155,6 +155,17 @@ def rlc_encode(W, mask, run_bits: int = 4, tile_rows: int = 0):
     return enc
 
 
+def rlc_count(mask, run_bits: int = 4, tile_rows: int = 0) -> np.ndarray:
+    """block_ptr alone (stored entries before each block, Section 3.2's rule), without building the arrays:
+    the counting pass of rlc_encode, for byte accounting on large masks."""
+    mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+    M, K = mask.shape
+    T = (M + tile_rows - 1) // tile_rows if tile_rows > 0 else 1
+    block_ptr = np.zeros(K * T + 1, np.int64)
+    _load().orc_rlc_count(_p(mask), K, M, K, run_bits, tile_rows, _p(block_ptr))
+    return block_ptr
+
+
 def rlc_decode_rows(enc) -> np.ndarray:
     rows = np.zeros(enc.vals.size, np.int32)
     _load().orc_rlc_decode_rows(_p(enc.runs), _p(enc.block_ptr), enc.K, enc.M, enc.tile_rows,

@@ -26,6 +26,7 @@ _sz = ctypes.c_size_t
 SIGNATURES = {
     "celty_encode": (ctypes.c_int, [_vp, _i64, _vp, _i64, _i64, _vp, ctypes.POINTER(_vp)]),
     "celty_destroy": (None, [_vp]),
+    "celty_clone": (ctypes.c_int, [_vp, ctypes.POINTER(_vp)]),
     "celty_info": (ctypes.c_int, [_vp] + [ctypes.POINTER(_i64)] * 5 + [ctypes.POINTER(_i32)] * 2),
     "celty_row_map": (ctypes.c_int, [_vp] + [ctypes.POINTER(_i32)] * 3),
     "celty_decode_host": (ctypes.c_int, [_vp, _i64, _vp, _vp, _vp, _vp, _i64, ctypes.POINTER(_i64)]),
@@ -39,6 +40,7 @@ SIGNATURES = {
     "celty_last_compaction": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
     "celty_decode_device": (ctypes.c_int, [_vp, _i64, _vp, _vp, _i64, _vp, _vp]),
     "celty_fetched_bytes": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "celty_stored_entries": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64)]),
     "celty_count_entries": (ctypes.c_int, [_vp, _i64, _i64, _i64, ctypes.c_int, ctypes.POINTER(_i64),
                                            ctypes.POINTER(_i64)]),
     "celty_last_status": (ctypes.c_int, [_vp, _vp]),
@@ -121,6 +123,17 @@ class Matrix:
         if device is not None:
             self.to(device)
 
+    def clone(self, device=None):
+        """A second handle on a copy of the encoded matrix (not packed again), optionally bound to `device`."""
+        h = _vp()
+        _check(load().celty_clone(self._h, ctypes.byref(h)), "celty_clone")
+        other = object.__new__(Matrix)
+        other._h, other.M, other.K = h, self.M, self.K
+        other._image = other._ws = None
+        if device is not None:
+            other.to(device)
+        return other
+
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
         if h and _lib is not None:
@@ -172,6 +185,13 @@ class Matrix:
         _check(load().celty_fetched_bytes(self._h, _np_ptr(idx), idx.size, ctypes.byref(s), ctypes.byref(t)),
                "celty_fetched_bytes")
         return s.value, t.value
+
+    def stored_entries(self, idx) -> int:
+        """Stored entries (kept weights + padding entries) of the listed columns."""
+        idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
+        e = _i64()
+        _check(load().celty_stored_entries(self._h, _np_ptr(idx), idx.size, ctypes.byref(e)), "celty_stored_entries")
+        return e.value
 
     def set_launch(self, grid: int = 0, variant: int = 0, groups: int = 0, depth: int = 0, team: int = 0):
         _check(load().celty_set_launch(self._h, grid, variant, groups, depth, team), "celty_set_launch")

@@ -283,6 +283,23 @@ extern "C" int celty_encode(const uint16_t *W, int64_t ldw, const uint8_t *mask,
 
 extern "C" void celty_destroy(celty_matrix *m) { delete m; }
 
+extern "C" int celty_clone(const celty_matrix *m, celty_matrix **out)
+{
+    if (!m || !out) return CELTY_EINVAL;
+    *out = nullptr;
+    try {
+        std::unique_ptr<celty_matrix> copy(new celty_matrix(*m));
+        copy->d_image = nullptr;                  // the copy starts unbound, with the library's launch choices
+        copy->d_ws = nullptr;
+        copy->last_grid = 0;
+        copy->last_merge = -1;
+        *out = copy.release();
+        return CELTY_OK;
+    } catch (const std::bad_alloc &) {
+        return CELTY_ENOMEM;
+    }
+}
+
 extern "C" int celty_info(const celty_matrix *m, int64_t *M, int64_t *K, int64_t *nnz, int64_t *n_pad,
                           int64_t *compressed_bytes, int32_t *layout, int32_t *tile_rows)
 {
@@ -410,6 +427,19 @@ extern "C" int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx, in
     // x read once, the list written (4-byte index + 2-byte value), y written once.  Scratch traffic of
     // the split-K merge (per-block partial sums) is not counted: it is overhead, not work.
     if (total_bytes) *total_bytes = sb + mb + 2 * m->K + 6 * n + 4 * m->M;
+    return CELTY_OK;
+}
+
+extern "C" int celty_stored_entries(const celty_matrix *m, const int32_t *idx, int64_t n, int64_t *entries)
+{
+    if (!m || (!idx && n > 0) || n < 0 || !entries) return CELTY_EINVAL;
+    int64_t e = 0;
+    for (int64_t p = 0; p < n; ++p) {
+        const int64_t j = idx[p];
+        if (j < 0 || j >= m->K) return CELTY_EINVAL;
+        e += (int64_t)m->block_ptr[(j + 1) * m->T] - (int64_t)m->block_ptr[j * m->T];
+    }
+    *entries = e;
     return CELTY_OK;
 }
 

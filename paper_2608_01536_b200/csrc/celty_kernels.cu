@@ -359,7 +359,11 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
 }
 
 // Raise a kernel's dynamic shared-memory limit once per device (and again only if a larger size is
-// asked for), so that steady-state calls make no attribute calls.
+// asked for), so that steady-state calls make no attribute calls.  The attribute belongs to the kernel,
+// so every entry point that launches a kernel shares that kernel's cache (g_granted_*): two caches for
+// one kernel could disagree about what the runtime currently allows.
+int g_granted_fused[64], g_granted_column[64], g_granted_lane[64];
+
 template <typename Kernel>
 int ensure_smem(Kernel kernel, size_t bytes, int *granted /* [64], per device */)
 {
@@ -483,8 +487,7 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         FusedPlan plan;
         rc = plan_fused(m, di, &plan);
         if (rc) return rc;
-        static int granted[64];
-        rc = ensure_smem(k_spmspv_fused, plan.smem, granted);
+        rc = ensure_smem(k_spmspv_fused, plan.smem, g_granted_fused);
         if (rc) return rc;
         FusedParams fp;
         fp.meta = reinterpret_cast<const uint32_t *>(m->d_image);
@@ -523,13 +526,14 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused, fp));
         return CELTY_OK;
     }
-    rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);
-    if (rc) return rc;
+    // two launches: compaction (which also clears y), then the product.  Sizes are checked and the
+    // shared-memory limit is raised before the first launch, so that an error return leaves y untouched.
     if (m->layout == CELTY_LAYOUT_COLUMN) {
         const size_t smem = (size_t)m->M * 4;
         if (smem > (size_t)di.max_smem_optin) return CELTY_EINVAL;
-        static int granted[64];
-        rc = ensure_smem(k_spmspv_column, smem, granted);
+        rc = ensure_smem(k_spmspv_column, smem, g_granted_column);
+        if (rc) return rc;
+        rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);
         if (rc) return rc;
         const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (size_t)(di.max_smem_optin) / (smem + 1024)));
         const int grid = m->grid > 0 ? m->grid : di.sms * per_sm;
@@ -541,8 +545,9 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         int G = (int)std::min<size_t>((size_t)di.max_smem_optin / group_bytes, (size_t)(32 / m->S));
         G = std::max(1, std::min(G, m->groups > 0 ? m->groups : (int)std::max<int64_t>(1, 8 / m->S)));
         const size_t smem = group_bytes * G;
-        static int granted[64];
-        rc = ensure_smem(k_spmspv_lane, smem, granted);
+        rc = ensure_smem(k_spmspv_lane, smem, g_granted_lane);
+        if (rc) return rc;
+        rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);
         if (rc) return rc;
         const int grid = m->grid > 0 ? m->grid : di.sms;
         k_spmspv_lane<<<grid, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(m->d_image),
@@ -601,19 +606,19 @@ extern "C" int celty_spmspv_static(const celty_matrix *m, const void *image_dev,
     uint8_t *scratch = nullptr;
     rc = static_scratch_address(&scratch);
     if (rc) return rc;
-    int32_t *count = reinterpret_cast<int32_t *>(scratch) + 1;
-    int32_t *idx = reinterpret_cast<int32_t *>(scratch + 256);
-    uint16_t *val = reinterpret_cast<uint16_t *>(scratch + 256 + (size_t)kStaticMaxK * 4);
-    float *y = static_cast<float *>(y_dev);
-    rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);     // also clears y
-    if (rc) return rc;
+    // every check comes before the first launch: an error return leaves y untouched
     const size_t group_bytes = (size_t)m->S * (m->R + kTileSlack) * 32 * 4;
     if (group_bytes > (size_t)di.max_smem_optin || m->S > 32) return CELTY_ELIMIT;
     const int G = (int)std::max<size_t>(1, std::min<size_t>((size_t)di.max_smem_optin / group_bytes,
                                                              (size_t)std::max<int64_t>(1, 8 / m->S)));
     const size_t smem = group_bytes * G;
-    static int granted[64];
-    rc = ensure_smem(k_spmspv_lane, smem, granted);
+    rc = ensure_smem(k_spmspv_lane, smem, g_granted_lane);
+    if (rc) return rc;
+    int32_t *count = reinterpret_cast<int32_t *>(scratch) + 1;
+    int32_t *idx = reinterpret_cast<int32_t *>(scratch + 256);
+    uint16_t *val = reinterpret_cast<uint16_t *>(scratch + 256 + (size_t)kStaticMaxK * 4);
+    float *y = static_cast<float *>(y_dev);
+    rc = launch_compact(x_dev, m->K, tau, idx, val, count, y, m->M, st);     // also clears y
     if (rc) return rc;
     const uint8_t *image = static_cast<const uint8_t *>(image_dev);
     k_spmspv_lane<<<di.sms, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(image),

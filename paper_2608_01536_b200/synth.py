@@ -12,6 +12,8 @@ with mix64 the SplitMix64 output function.
 """
 from __future__ import annotations
 
+import os
+
 import numpy as np
 
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
@@ -36,15 +38,29 @@ def _key(seed: int, tag: int) -> np.uint64:
 
 
 def uniform(seed: int, tag: int, n: int, start: int = 0) -> np.ndarray:
-    """n doubles in [0, 1), elements start .. start+n-1 of stream (seed, tag)."""
+    """n doubles in [0, 1), elements start .. start+n-1 of stream (seed, tag).  Every element depends only on
+    its own counter, so large requests are filled chunk by chunk on a few threads (same values either way)."""
     out = np.empty(n, np.float64)
     key = _key(seed, tag)
-    with np.errstate(over="ignore"):
-        for a in range(0, n, _CHUNK):
-            b = min(n, a + _CHUNK)
+
+    def fill(a):
+        b = min(n, a + _CHUNK)
+        with np.errstate(over="ignore"):
             ctr = np.arange(start + a + 1, start + b + 1, dtype=np.uint64)
-            z = _mix64(key + ctr * _GOLDEN)
-            out[a:b] = (z >> np.uint64(11)).astype(np.float64) * (1.0 / 9007199254740992.0)
+            ctr *= _GOLDEN
+            ctr += key
+            z = _mix64(ctr)
+            z >>= np.uint64(11)
+        np.multiply(z, 1.0 / 9007199254740992.0, out=out[a:b])
+
+    starts = range(0, n, _CHUNK)
+    if n <= 4 * _CHUNK:
+        for a in starts:
+            fill(a)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(min(16, os.cpu_count() or 1)) as pool:
+            list(pool.map(fill, starts))
     return out
 
 
@@ -52,19 +68,28 @@ def normal(seed: int, tag: int, n: int) -> np.ndarray:
     """Standard normal by Box-Muller on streams tag and tag+1."""
     u1 = uniform(seed, tag, n)
     u2 = uniform(seed, tag + 1, n)
-    return np.sqrt(-2.0 * np.log1p(-u1)) * np.cos(2.0 * np.pi * u2)
+    return np.sqrt(-2.0 * np.log(1.0 - u1)) * np.cos(2.0 * np.pi * u2)     # 1 - u1 is exact
 
 
 def laplace(seed: int, tag: int, n: int) -> np.ndarray:
     """Laplace(0, 1) by inverse CDF."""
     u = uniform(seed, tag, n) - 0.5
-    return -np.sign(u) * np.log1p(-2.0 * np.abs(u))
+    return -np.sign(u) * np.log(1.0 - 2.0 * np.abs(u))
 
 
 # ----------------------------------------------------------------------------- weights / masks
 def weights(seed: int, M: int, K: int, std: float = 0.02) -> np.ndarray:
     """FP16 M x K row-major weights ~ N(0, std^2)."""
     return (normal(seed, 1, M * K) * std).astype(np.float16).reshape(M, K)
+
+
+def weights_tiled(seed: int, M: int, K: int, block_cols: int, std: float = 0.02) -> np.ndarray:
+    """FP16 M x K weights whose columns repeat a block of `block_cols` columns ~ N(0, std^2) along K.  For the
+    largest layers, where drawing every weight would take minutes: which weights are kept comes from the mask,
+    which is never repeated, so no two columns hold the same entries."""
+    block = weights(seed, M, min(K, block_cols), std)
+    reps = -(-K // block.shape[1])
+    return np.ascontiguousarray(np.tile(block, (1, reps))[:, :K])
 
 
 def integer_weights(seed: int, M: int, K: int, amp: int = 3) -> np.ndarray:

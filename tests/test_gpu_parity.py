@@ -81,6 +81,38 @@ def test_compaction_bit_exact(K):
         assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
 
 
+SPECIAL_X = np.array([0x0000, 0x8000, 0x7E00, 0xFE00, 0x7C00, 0xFC00, 0x0001, 0x8001, 0x03FF, 0x83FF, 0x0400, 0x8400,
+                      0x7BFF, 0xFBFF, 0x3C00, 0xBC00, 0x3C01, 0x3BFF, 0x3800, 0xB800], np.uint16)
+
+
+@pytest.mark.parametrize("K", [20, 64, 1000, 4099])
+@pytest.mark.parametrize("tau", [0.0, 1e-8, 5.9604645e-08, 0.99975586, 1.0, 1.0004883, 0.7, 65504.0, 65519.9, 1e5])
+def test_fused_kernel_thresholding_bit_exact_on_special_values(K, tau):
+    """The fused kernel has its own thresholding code (it compares in FP16 against tau rounded down to FP16, which
+    is the same decision as |x| > tau in FP32): +-0, NaNs, +-infinity, the smallest and largest subnormals, the
+    smallest normal, the largest finite value and the neighbours of 1, against thresholds that are 0, below the
+    smallest subnormal, exactly on FP16 values, strictly between two FP16 neighbours, the largest finite FP16
+    value and beyond it.  The list the call leaves behind must be the oracle's, bit for bit."""
+    x = synth.activations(K + 3, K, "laplace").view(np.uint16).copy()
+    pos = (np.arange(SPECIAL_X.size) * 37) % K if K > SPECIAL_X.size else np.arange(SPECIAL_X.size)
+    x[pos[:K]] = SPECIAL_X[:K]
+    x = x.view(np.float16)
+    M = 64
+    W = synth.weights(K, M, K)
+    m = celty.Matrix(W, None, device="cuda")
+    m.spmspv(_dev(x), tau)
+    torch.cuda.synchronize()
+    assert m.last_status() == 0
+    idx, val = m.last_compaction()
+    oi, ov, n = orc.compact(x, tau)
+    assert idx.numel() == n
+    assert np.array_equal(idx.cpu().numpy(), oi)
+    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+    # the stand-alone compaction kernel takes the same decisions
+    i2, v2 = celty.compact(_dev(x), tau)
+    assert np.array_equal(i2.cpu().numpy(), oi) and np.array_equal(v2.cpu().numpy().view(np.uint16), ov)
+
+
 def test_compaction_ties_are_dropped():
     x = np.array([0.5, -0.5] * 20, np.float16)
     assert celty.compact(_dev(x), 0.5)[0].numel() == 0
@@ -286,40 +318,58 @@ def test_longest_column_and_power_law_rows(layout):
     _check_y(_run(m, x, tau), W, mask, x, tau)
 
 
-@pytest.mark.parametrize("layout", LAYOUTS)
-def test_llama7b_attention_shape_in_bench_configuration(layout):
-    """4096 x 4096, magnitude-pruned 50% per column, Laplace activations kept at 50%: the workload
-    and launch configuration bench.py times, compared in full."""
-    M = K = 4096
-    W = synth.weights(synth.point_seed(2, 4), M, K)
-    mask = synth.mask_magnitude(W, 0.5)
-    x = synth.activations(synth.point_seed(2, 4), K, "laplace")
-    tau = synth.threshold_for_density(x, 0.5)
-    m = _matrix(W, mask, layout)
-    _check_y(_run(m, x, tau), W, mask, x, tau)
-
-
-def test_llama70b_mlp_shape_in_bench_configuration():
-    """28672 x 8192, Bernoulli mask at 50%, Laplace activations kept at 50%: the large workload bench.py times, at
-    full size in the launch configuration it is timed in, every row compared and the list bit for bit.  (The weights
-    repeat a 28672 x 1024 block eight times along K to keep the generator's time down; the mask does not repeat,
-    so no two columns hold the same entries.)"""
-    M, K = 28672, 8192
-    seed = synth.point_seed(5, 3)
-    W = np.tile(synth.weights(seed, M, K // 8), (1, 8))
-    mask = synth.mask_bernoulli(seed, M, K, 0.5)
-    x = synth.activations(seed, K, "laplace")
-    tau = synth.threshold_for_density(x, 0.5)
-    m = _matrix(W, mask, (celty.LAYOUT_LANE_TILE, 0))
-    assert m.row_map() == (8, 112, 16)
-    y = _run(m, x, tau)
-    _check_y(y, W, mask, x, tau)
-    idx, val = m.last_compaction()
+def _full_size_case(W, mask, x, tau):
+    """Every row within the bound, the list bit for bit, and a second call on the same handle (the tickets wrap
+    around), in the launch configuration the library picks by default -- the one bench.py times."""
+    m = celty.Matrix(W, mask, device="cuda")
+    y_ref, a_ref = orc.masked_gemv(W, mask, x, tau, threads=orc.max_threads())
     oi, ov, _ = orc.compact(x, tau)
-    assert np.array_equal(idx.cpu().numpy(), oi)
-    assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
-    # a second call on the same handle (tickets wrap around) gives the same rows within the bound
-    _check_y(_run(m, x, tau), W, mask, x, tau)
+    xd = _dev(x)
+    for call in range(2):
+        y = m.spmspv(xd, tau, y=torch.full((W.shape[0],), float(call + 5), device="cuda"))
+        torch.cuda.synchronize()
+        assert m.last_status() == 0
+        err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+        bound = 2e-3 * a_ref + 1e-6
+        worst = int(np.argmax(err - bound))
+        assert np.all(err <= bound), (call, worst, err[worst], bound[worst])
+        idx, val = m.last_compaction()
+        assert np.array_equal(idx.cpu().numpy(), oi)
+        assert np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+
+
+def _bench_module():
+    import importlib
+    return importlib.import_module("bench")
+
+
+BENCH_WORKLOADS = ["llama7b_attn_4096x4096_s50_a50", "llama7b_gateup_11008x4096_s50_a50",
+                   "llama7b_down_4096x11008_s50_a50", "llama13b_attn_5120x5120_s50_a40",
+                   "llama13b_gateup_13824x5120_s50_a40", "llama13b_down_5120x13824_s50_a40",
+                   "llama70b_mlp_28672x8192_s50_a50", "llama70b_down_8192x28672_s50_a50",
+                   "llama70b_mlp_28672x8192_s30_a50", "llama70b_mlp_28672x8192_s70_a50", "small_1024x1024_s50_a50"]
+
+
+@pytest.mark.parametrize("name", BENCH_WORKLOADS)
+def test_every_bench_workload_at_full_size(name):
+    """Each workload bench.py can time, at its full size, drawn by bench.py's own recipe (same seeds)."""
+    bench = _bench_module()
+    assert sorted(bench.WORKLOADS) == sorted(BENCH_WORKLOADS)          # none is left out of this test
+    W, mask = bench.make_layer(name, 0)
+    x, tau = bench.make_x(name, 0)
+    _full_size_case(W, mask, x, tau)
+
+
+@pytest.mark.parametrize("M,K,s,d_a", [(28672, 8192, 0.7, 0.3), (8192, 28672, 0.3, 0.7)])
+def test_power_law_masks_of_the_large_sweep_at_full_size(M, K, s, d_a):
+    """Row-clustered power-law masks of the 28672 x 8192 / 8192 x 28672 sweep (dense top rows, a long sparse tail
+    with many gaps beyond 15 rows), at full size."""
+    seed = synth.point_seed(5, 0)
+    W = synth.weights_tiled(seed, M, K, K // 8)
+    mask = synth.mask_powerlaw(seed, M, K, 1.0 - s)
+    x = synth.activations(synth.point_seed(5, 50), K, "laplace")
+    tau = synth.threshold_for_density(x, d_a)
+    _full_size_case(W, mask, x, tau)
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)

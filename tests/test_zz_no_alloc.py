@@ -33,10 +33,62 @@ def test_static_scratch_entry_point_matches_the_workspace_entry_point_twice():
         y_ws = m.spmspv(xd, tau)                              # existing entry point
         y_st = m.spmspv_static(xd, tau, y=torch.full((M,), 3.0, device="cuda"))
         torch.cuda.synchronize()
-        _, a_ref = orc.masked_gemv(W, mask, x, tau, threads=8)
-        err = np.abs(y_st.cpu().numpy().astype(np.float64) - y_ws.cpu().numpy().astype(np.float64))
-        assert np.all(err <= 2e-3 * a_ref + 1e-6), (call, float(err.max()))
+        y_ref, a_ref = orc.masked_gemv(W, mask, x, tau, threads=8)
+        bound = 2e-3 * a_ref + 1e-6
+        got = y_st.cpu().numpy().astype(np.float64)
+        # against the existing entry point ...
+        assert np.all(np.abs(got - y_ws.cpu().numpy().astype(np.float64)) <= bound), call
+        # ... and against the definition itself
+        assert np.all(np.abs(got - y_ref) <= bound), call
         assert torch.count_nonzero(y_st).item() > 0
+
+
+def test_static_scratch_entry_point_leaves_device_memory_alone():
+    """The point of the entry point: a call takes no device memory.  The free-memory figure of the
+    driver must be the same before and after a call (the first call on the device has already looked
+    up the array's address; outputs are allocated beforehand)."""
+    build.build()
+    M, K = 2048, 1024
+    W = synth.weights(78, M, K)
+    mask = synth.mask_bernoulli(78, M, K, 0.5)
+    m = celty.Matrix(W, mask, device="cuda")
+    x = synth.activations(3, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.5)
+    xd = torch.from_numpy(x).cuda()
+    y = torch.empty(M, dtype=torch.float32, device="cuda")
+    m.spmspv_static(xd, tau, y=y)                             # set-up call
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    m.spmspv_static(xd, tau, y=y)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    y_ref, a_ref = orc.masked_gemv(W, mask, x, tau, threads=8)
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= 2e-3 * a_ref + 1e-6)
+
+
+def test_static_and_two_launch_entry_points_share_one_kernel_attribute():
+    """Both entry points launch the same lane-tile kernel with different amounts of dynamic shared memory
+    (a 4096-row handle asks for more than a 12288-row one).  Interleaving them must not leave either with
+    a stale idea of what the runtime currently allows."""
+    build.build()
+    K = 256
+    mats = []
+    for M in (4096, 12288):
+        W = synth.weights(80 + M, M, K)
+        mask = synth.mask_bernoulli(80 + M, M, K, 0.5)
+        m = celty.Matrix(W, mask, device="cuda")
+        m.set_launch(variant=1)
+        mats.append((m, W, mask))
+    x = synth.activations(5, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.5)
+    xd = torch.from_numpy(x).cuda()
+    small, big = 0, 1
+    for which, static in ((small, False), (big, True), (small, False), (small, True), (big, False)):
+        m, W, mask = mats[which]
+        y = m.spmspv_static(xd, tau) if static else m.spmspv(xd, tau)
+        torch.cuda.synchronize()
+        y_ref, a_ref = orc.masked_gemv(W, mask, x, tau, threads=8)
+        assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= 2e-3 * a_ref + 1e-6), (W.shape, static)
 
 
 def test_static_scratch_entry_point_rejects_what_it_cannot_hold():
