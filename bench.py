@@ -409,7 +409,7 @@ def run_format_study(args):
 def run_knob_study(args):
     """Launch-parameter study (the paper's Figure 11 question -- how far to split the columns -- asked of this
     kernel): time of one workload against the number of thread blocks (column slices = blocks / row parts),
-    warp teams per block, ring depth and warps per team, everything else the library's choice.  Same protocol as
+    warp teams per block, ring depth and thread blocks per cluster, everything else the library's choice.  Same protocol as
     the sweeps: rotation over device copies beyond 2x L2, one CUDA graph, CUDA events."""
     import torch
     from paper_2608_01536_b200 import build as lib_build, celty
@@ -473,8 +473,8 @@ def run_knob_study(args):
         add("groups", groups, groups=groups)
     for depth in (2, 3, 4):
         add("depth", depth, depth=depth)
-    for team in (1, 2, 4):
-        add("team", team, team=team)
+    for cluster in (1, 2, 4):
+        add("cluster", cluster, cluster=cluster)
     for m in mats:
         m.set_launch()
     print(json.dumps({"sweep": "knobs", "workload": name, "row_parts": int(S), "device_copies": copies,
@@ -523,8 +523,8 @@ class Workload:
         for c in range(self.copies):
             m = base[c % distinct_n] if c < distinct_n else base[c % distinct_n].clone()
             m.to(dev)
-            if args.grid or args.variant or args.groups or args.depth:
-                m.set_launch(args.grid, args.variant, args.groups, args.depth)
+            if args.grid or args.variant or args.groups or args.depth or args.cluster:
+                m.set_launch(args.grid, args.variant, args.groups, args.depth, args.cluster)
             x, tau = make_x(name, c)
             self.mats.append(m)
             self.xs.append(torch.from_numpy(x).to(dev))
@@ -751,6 +751,7 @@ def run_celty(args):
         "config": workload_config(name),
         "run": {
             "layout": args.layout, "tile_rows": info.tile_rows,
+            "fused_launch": wl.mats[0].launch_plan() if args.layout != "column" else None,
             "l2": f"rotation over {wl.copies} device copies ({len(wl.distinct)} distinct matrices, {wl.copies} distinct "
                   f"x), {wl.copies * wl.image_bytes / 1e6:.0f} MB > 2x L2 ({wl.l2 / 1e6:.0f} MB)",
             "launch": "stream enqueue" if args.no_graph else f"cuda graph of {wl.unit} calls",
@@ -814,6 +815,7 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--groups", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
+    ap.add_argument("--cluster", type=int, default=0)
     ap.add_argument("--tile-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-dense", action="store_true")

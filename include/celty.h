@@ -185,8 +185,10 @@ int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *idx_dev, uin
  * independent), so results may differ in the last bits between calls.  Activations must be finite
  * for the result to equal the definition in every row: a zero-valued stored slot (a padding entry,
  * or a slot that fills a lane's last group of 8) times an infinite or NaN x_j is NaN.
- * Errors: CELTY_EINVAL, CELTY_ESTATE, CELTY_ECUDA.  Device-side problems (a bounded wait that ran
- * out, an out-of-range index) do not fault: they set the status word, see celty_last_status.
+ * Errors: CELTY_EINVAL, CELTY_ESTATE, CELTY_ECUDA.  A bounded wait that runs out inside the kernel does
+ * not hang or fault: it sets the status word (CELTY_ETIMEOUT from celty_last_status).  Decoded row indices
+ * are range-checked by the COLUMN kernel only (CELTY_EBOUNDS); the LANE_TILE kernels trust the image that
+ * celty_encode built.
  */
 int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, celty_stream_t stream);
 
@@ -296,10 +298,33 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            launch (with which the kernel's set-up overlaps the tail of the previous kernel of the stream)
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
- *   team     fused kernel: warps that share one sub-block and one accumulator (1, 2 or 4)
+ *   cluster  fused kernel, bulk reduce-add merge: thread blocks per cluster (1, 2 or 4); the blocks of a
+ *            cluster add their accumulators through distributed shared memory before anything goes to y
+ *            (the split-K trade-off of Sections 3.1 and 6.4 with an on-chip stage).  A size the grid or the
+ *            device cannot take is halved until it fits.
  * Errors: CELTY_EINVAL.
  */
-int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth, int32_t team);
+int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth, int32_t cluster);
+
+/*
+ * celty_launch_plan -- the shape the fused kernel would be launched with for this handle on the current
+ * device, with the knobs of celty_set_launch applied (LANE_TILE handles; needs a CUDA device):
+ *   out[0..9] = thread blocks, threads per block, dynamic shared memory (bytes), warp teams per slab,
+ *   ring slots per team, thread blocks per cluster, row parts, slabs per block, ring slot size (bytes),
+ *   merge (0 ordered two-stage sum, 1 bulk reduce-add).   n = capacity of out (at least 10).
+ * Errors: CELTY_EINVAL, CELTY_ECUDA.
+ */
+int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n);
+
+/*
+ * celty_set_wait_limit -- how many polls a bounded wait inside the kernels (for a bulk copy, for the other
+ * thread blocks' tickets) makes before it gives up, sets the status word and lets the kernel finish; 0 = the
+ * library's limit (about two million polls, far beyond any real wait).  The kernels never spin without a
+ * limit: a wait that runs out shows up as CELTY_ETIMEOUT from celty_last_status, the call's y is then
+ * undefined, and the handle is usable again after that call to celty_last_status.
+ * Errors: CELTY_EINVAL.
+ */
+int celty_set_wait_limit(celty_matrix *m, uint32_t polls);
 
 /* The cudaError_t of the last failing CUDA call made through this library (0 if none). */
 int celty_last_cuda_error(void);

@@ -45,6 +45,8 @@ SIGNATURES = {
                                            ctypes.POINTER(_i64)]),
     "celty_last_status": (ctypes.c_int, [_vp, _vp]),
     "celty_set_launch": (ctypes.c_int, [_vp, _i32, _i32, _i32, _i32, _i32]),
+    "celty_launch_plan": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), _i32]),
+    "celty_set_wait_limit": (ctypes.c_int, [_vp, ctypes.c_uint32]),
     "celty_last_cuda_error": (ctypes.c_int, []),
     "celty_strerror": (ctypes.c_char_p, [ctypes.c_int]),
 }
@@ -193,8 +195,20 @@ class Matrix:
         _check(load().celty_stored_entries(self._h, _np_ptr(idx), idx.size, ctypes.byref(e)), "celty_stored_entries")
         return e.value
 
-    def set_launch(self, grid: int = 0, variant: int = 0, groups: int = 0, depth: int = 0, team: int = 0):
-        _check(load().celty_set_launch(self._h, grid, variant, groups, depth, team), "celty_set_launch")
+    def set_launch(self, grid: int = 0, variant: int = 0, groups: int = 0, depth: int = 0, cluster: int = 0):
+        _check(load().celty_set_launch(self._h, grid, variant, groups, depth, cluster), "celty_set_launch")
+
+    def launch_plan(self) -> dict:
+        """Shape of the fused kernel's launch for this handle on the current device."""
+        out = (_i32 * 10)()
+        _check(load().celty_launch_plan(self._h, out, 10), "celty_launch_plan")
+        keys = ("grid", "threads", "smem_bytes", "teams_per_slab", "ring_depth", "cluster", "row_parts",
+                "slabs_per_block", "slot_bytes", "merge")
+        return dict(zip(keys, [int(v) for v in out]))
+
+    def set_wait_limit(self, polls: int = 0):
+        """Polls a bounded wait inside the kernels makes before it gives up (0 = the library's limit)."""
+        _check(load().celty_set_wait_limit(self._h, polls), "celty_set_wait_limit")
 
     # ---------------------------------------------------------------- device side
     def to(self, device="cuda", stream=None):

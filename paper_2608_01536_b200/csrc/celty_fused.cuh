@@ -4,24 +4,27 @@
 // One launch does the whole call (Sections 3.1-3.3):
 //   a0  the last warp of every block clears its share of y and takes a ticket (the merge at the end adds into y);
 //   a1  every block thresholds all of x (K <= a few 10k values, served by L2) into one keep bit per
-//       activation and ranks the survivors (popcounts + warp scans); each warp team then looks up the
-//       columns whose ranks belong to it -- the list is balanced over all teams by count.  The team
-//       that owns a rank on slab 0 also writes it to the global list (index, value, count) for the API;
-//   a2  each team streams the sub-blocks (column j, slab s) of its columns from HBM into its ring of
-//       shared-memory slots with bulk asynchronous copies (cp.async.bulk + mbarrier complete_tx), D deep;
-//   a3  each lane decodes its own tile's runs on packed bytes and keeps a running row; the W warps of a
-//       team split the steps of a sub-block at the split points its header carries;
+//       activation and ranks the survivors (popcounts + warp scans).  The survivor list is cut into equal
+//       runs of ranks, one per thread block; the threads that made the keep words write the columns of
+//       the block's run straight into its work list in shared memory, and the streaming warps fetch each
+//       listed column's activation and sub-block offset in one round trip.  The blocks of row part 0
+//       also write the list (index, value, count) for the API;
+//   a2  the block's warp teams take columns from that list one at a time (a shared-memory counter) and
+//       stream their sub-blocks (column j, slab s) from HBM into per-team rings of shared-memory slots
+//       with bulk asynchronous copies (cp.async.bulk + mbarrier complete_tx), D deep;
+//   a3  each lane decodes its own tile's runs on packed bytes and keeps a running row;
 //   a4  value * x_j is accumulated (FP16 x FP16 + FP32 fused multiply-add) into the lane's private bank of
 //       the team's accumulator;
-//   a5  the block adds its G accumulators; the row map makes a slab's accumulator a sequence of 32*C-row
+//   a5  the thread blocks of a cluster add their accumulators through distributed shared memory, each
+//       block the row segments it owns; the row map makes a slab's accumulator a sequence of 32*C-row
 //       segments of y, and each goes out as one bulk reduce-add copy (FP32 add in L2) once the tickets show
 //       that every block has cleared its share of y.  Option: per-block partial vectors, a bounded
 //       grid-wide ticket barrier and a sum in a fixed order (bit-reproducible, no clearing of y).
 //
-// Rows are split over P parts (blockIdx % P) of Sc slabs each, columns over gridDim/P slices; inside a
-// block G groups take different columns, a team = (group, slab) owns one accumulator slab.  Every block
-// must be resident at once (grid <= SM count) because of the tickets.  All waits are bounded:
-// when one runs out the kernel sets kStatusTimeout in the status word and carries on to a clean exit.
+// Rows are split over P parts of Sc slabs each, columns over the blocks of a part; a team = one warp with
+// its own accumulator slab, G teams per slab.  Every block must be resident at once (grid <= SM count)
+// because of the tickets.  All waits are bounded: when one runs out the kernel sets kStatusTimeout in the
+// status word and carries on to a clean exit.
 
 struct FusedParams {
     const uint32_t *meta;      // [K*S + 1] offset/16 of sub-block (j, s) in the stream
@@ -33,20 +36,24 @@ struct FusedParams {
     uint16_t *val;
     int32_t *count;
     uint32_t *status;
-    uint32_t *tickets;         // [0] partial stored, [1] departed
+    uint32_t *tickets;         // [0] y cleared / partial stored, [1] departed
     float *partials;           // gridDim.x vectors of Sc * R * 32 floats (accumulator layout)
     int M, K, R, S, C;         // rows, columns, local rows per tile, slabs, chunk of the row map (tile_row)
-    int G, Sc, P, D, W;        // groups, slabs per block, row parts, ring depth, warps per team (1, 2 or 4)
+    int G, Sc, P, D;           // teams per slab, slabs per block, row parts, ring depth
+    int cl;                    // thread blocks per cluster (1, 2 or 4); blocks of a cluster share a row part
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
-    int cap;                   // items a team looks up per batch
-    // groups that share the survivor list of a row part: units = (column slices of the part) * G;
-    // units_inv = floor(2^32 / units) for parts with grid / P slices, units_inv_long for those with one more
-    uint32_t units_inv, units_inv_long;
-    int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row tiles into y
+    int cap;                   // columns the block's work list holds at a time
+    int win_cols;              // columns of the offset table a block copies into shared memory at its start
+    int fixed_deal;            // 1: a team takes every G-th column of the list instead of the next free one
+    // column slices of a row part = blocks that share its survivor list: slices_inv = floor(2^32 / slices)
+    // for parts with gridDim / cl / P clusters, slices_inv_long for those with one cluster more
+    uint32_t slices_inv, slices_inv_long;
+    int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row segments into y
+    uint32_t spin_limit;       // polls a bounded wait makes before it gives up
 };
 
-constexpr uint32_t kSpinLimit = 1u << 21;
+constexpr uint32_t kSpinLimit = 1u << 21;   // default for FusedParams::spin_limit
 
 // Development builds only (compiled out of the product):
 //   -DCELTY_TRACE  thread 0 of every block stores clock64() at phase k into trace[blockIdx.x * 16 + k];
@@ -102,28 +109,82 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 
 // Wait for a phase of an mbarrier with an iteration limit; false = gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 256) __nanosleep(128);
     }
     return false;
 }
 
-// Bulk asynchronous copy global -> shared (1-D, no tensor map, no multicast); src, dst and bytes are
-// multiples of 16.  Every lane of a converged warp calls this; one elected lane announces the bytes on the
-// mbarrier and issues the copy, both under a predicate (no branch), and completion is signalled on the
-// mbarrier as transferred bytes.
-__device__ __forceinline__ void bulk_load_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+// Bulk asynchronous copy global -> shared (1-D, no tensor map; every sub-block has exactly one consumer,
+// the team that asked for it); src, dst and bytes are multiples of 16.  Every lane of a converged warp calls
+// this; one elected lane notes the column's activation beside the slot, announces the bytes on the mbarrier
+// and issues the copy, all under a predicate (no branch); completion is signalled on the mbarrier as
+// transferred bytes.
+__device__ __forceinline__ void bulk_load_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
+                                                  uint32_t note_addr, uint32_t note)
 {
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "elect.sync _|P, 0xffffffff;\n\t"
+        "@P st.shared.u32 [%4], %5;\n\t"
         "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t"
         "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%2], [%3], %1, [%0];\n\t}" ::"r"(bar),
-        "r"(bytes), "r"(dst), "l"(src)
+        "r"(bytes), "r"(dst), "l"(src), "r"(note_addr), "r"(note)
         : "memory");
+}
+
+// The same with one more step for the elected lane: it takes the next position of the block's work list
+// (shared-memory counter at `next_addr`) for the refill after this one.  `taken` is meaningful in lane `leader`
+// only; the caller broadcasts it when it needs it, a whole sub-block later, so nobody waits for the atomic.
+__device__ __forceinline__ void bulk_load_elected_take(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
+                                                       uint32_t note_addr, uint32_t note, uint32_t next_addr,
+                                                       uint32_t &taken, uint32_t &leader)
+{
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync %1|P, 0xffffffff;\n\t"
+        "@P st.shared.u32 [%6], %7;\n\t"
+        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%2], %3;\n\t"
+        "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%4], [%5], %3, [%2];\n\t"
+        "@P atom.shared.add.u32 %0, [%8], 1;\n\t}"
+        : "+r"(taken), "=r"(leader)
+        : "r"(bar), "r"(bytes), "r"(dst), "l"(src), "r"(note_addr), "r"(note), "r"(next_addr)
+        : "memory");
+}
+
+// The take alone (after a team's first copies).
+__device__ __forceinline__ void take_elected(uint32_t next_addr, uint32_t &taken, uint32_t &leader)
+{
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync %1|P, 0xffffffff;\n\t"
+        "@P atom.shared.add.u32 %0, [%2], 1;\n\t}"
+        : "+r"(taken), "=r"(leader)
+        : "r"(next_addr)
+        : "memory");
+}
+
+// Barrier across the thread blocks of the cluster (release / acquire: shared-memory writes made before it
+// are visible to the other blocks' distributed-shared-memory reads after it).
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// 128-bit load from the shared memory of block `rank` of the cluster, at this block's address `local`.
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local, uint32_t rank)
+{
+    uint32_t remote;
+    float4 v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(remote)
+                 : "memory");
+    return v;
 }
 
 // Polling load that goes to L2 every time but carries no ordering (and so leaves the L1 of the other
@@ -142,14 +203,7 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
     return v;
 }
 
-// Barrier among the 32 * nwarps threads of one team (hardware named barrier `id`, 1..15).
-__device__ __forceinline__ void team_sync(int id, int nthreads)
-{
-    if (nthreads == 32) __syncwarp();
-    else asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-
-// One lane's work on a range of steps of a sub-block, as a three-stage software pipeline (a step =
+// One lane's work on the steps of a sub-block, as a three-stage software pipeline (a step =
 // one group of 8 entries of every lane that still has one):
 //   fetch(q+2)   128-bit value vector + 32-bit run word from the ring slot
 //   decode(q)    run-length decode on packed bytes, cell addresses; the 8 accumulator loads are
@@ -254,24 +308,27 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, items, imeta, zero, keep, wrel, blk, blkw, total;
+    size_t acc, ring, bars, note, items, imeta, next, zero, keep, wrel, blk, blkx, total;
 };
 
-__host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
+__host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int Sc, int D, int slot_bytes, int cap)
 {
     FusedSmem l;
     size_t off = 0;
+    const size_t words = ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16, blocks = ((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16;
     l.acc = off;       off += (size_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
     l.ring = off;      off += (size_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
-    l.bars = off;      off += (size_t)teams * D * 8;                       // one "full" mbarrier per slot
+    l.bars = off;      off += (size_t)teams * D * 8 + 8;                   // one "full" mbarrier per slot, one for the offset window
+    l.note = off;      off += (size_t)teams * D * 4;                       // the activation of the column in each slot
     off = (off + 15) / 16 * 16;
-    l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
-    l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
+    l.items = off;     off += (size_t)cap * 8;                             // work list: {column, x bits}
+    l.imeta = off;     off += (size_t)Sc * cap * 8;                        // per slab of the block: {offset/16, bytes}
+    l.next = off;      off += 64;                                          // per slab: next list position to hand out
     l.zero = off;      off += 16;                                          // the all-zero group that idle lanes fetch
-    l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
-    l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 32
-    l.blk = off;       off += ((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16; // survivors in each block of 32 keep words
-    l.blkw = off;      off += 16 * (((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
+    l.keep = off;      off += words;                                       // one keep bit per activation
+    l.wrel = off;      off += words;                                       // survivors before each keep word, in its block of 32
+    l.blk = off;       off += blocks;                                      // survivors in each block of 32 keep words
+    l.blkx = off;      off += blocks;                                      // survivors before each block
     l.total = off;
     return l;
 }
@@ -284,28 +341,31 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     // derived from it) is the same for all lanes, and keeps the streaming loop free of divergence handling
     const int warp = __shfl_sync(kFull, tid >> 5, 0);
     const int slab_words = (p.R + kTileSlack) * 32;
-    // Warps [0, teams * W) stream columns, W warps per team; the others only help with the phases that
-    // are plain data-parallel work (thresholding, clearing, storing and summing partial vectors).
+    // Warps [0, teams) stream columns, one warp per team; the others only help with the phases that are plain
+    // data-parallel work (thresholding, the work list, clearing, the merge).
     const int teams = p.G * p.Sc;
-    const bool streams = warp < teams * p.W;
-    const int team = streams ? warp / p.W : 0, member = streams ? warp - team * p.W : 0;
-    const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.D, p.slot_bytes, p.cap);
+    const bool streams = warp < teams;
+    const int team = streams ? warp : 0;
+    const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.Sc, p.D, p.slot_bytes, p.cap);
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
-    int2 *items = reinterpret_cast<int2 *>(smem + lay.items) + (size_t)team * p.cap;      // [cap] {column, x bits}
-    uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
+    int2 *items = reinterpret_cast<int2 *>(smem + lay.items);                             // [cap] {column, x bits}
+    int *next = reinterpret_cast<int *>(smem + lay.next);                                 // [Sc]
     int *zero_group = reinterpret_cast<int *>(smem + lay.zero);                           // 16 bytes of zeros
     int *wrel = reinterpret_cast<int *>(smem + lay.wrel);                                 // [nwords]
-    const int *blk = reinterpret_cast<const int *>(smem + lay.blk);                       // [nwords / 32] counts
-    int *myblk = reinterpret_cast<int *>(smem + lay.blkw) + (size_t)warp * ((lay.blkw - lay.blk) / 4);   // this warp's prefix
+    int *blk = reinterpret_cast<int *>(smem + lay.blk);                                   // [nwords / 32] counts
+    int *blkx = reinterpret_cast<int *>(smem + lay.blkx);                                 // [nwords / 32] exclusive prefix
     uint32_t *kbw = reinterpret_cast<uint32_t *>(smem + lay.keep);
 
-    // Row part and column slice of this block.  The grid need not be a multiple of P: the first gridDim mod P
-    // parts then have one column slice more than the others.
-    const int part = blockIdx.x % p.P, kslice = blockIdx.x / p.P;
-    const bool long_part = part < (int)(gridDim.x % p.P);
-    const int nK = gridDim.x / p.P + (long_part ? 1 : 0);
+    // Row part and column slice of this block.  The blocks of a cluster work on the same row part (they add
+    // their accumulators before anything goes to y).  The number of clusters need not be a multiple of P: the
+    // first (clusters mod P) parts then have one cluster more than the others.
+    const int crank = blockIdx.x % p.cl, cid = blockIdx.x / p.cl, nclusters = gridDim.x / p.cl;
+    const int part = cid % p.P;
+    const bool long_part = part < nclusters % p.P;
+    const int nK = p.cl * (nclusters / p.P + (long_part ? 1 : 0));
+    const int kslice = (cid / p.P) * p.cl + crank;
     const int g = team / p.Sc, sl = team - g * p.Sc;
     const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
 
@@ -314,16 +374,31 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     // and do everything that touches neither the caller's vectors nor the workspace (warming L2 with the offset
     // table, setting up shared memory) before waiting for the previous kernel of the stream to be complete.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // The sub-block offsets are needed right after the ranks are known: start pulling the table into L2
-    // now, each block its own share of the lines (L2 is shared by all blocks).
-    {
-        const size_t lines = (((size_t)p.K * p.S + 1) * 4 + 127) / 128;
-        const size_t per = (lines + gridDim.x - 1) / gridDim.x, l0 = (size_t)blockIdx.x * per;
-        for (size_t l = l0 + tid; l < min(lines, l0 + per); l += nthreads)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(p.meta) + l * 128));
+    // The sub-block offsets are needed right after the ranks are known.  A block's columns lie around the same
+    // fraction of K as its position among the blocks of its row part, so it copies that window of the offset
+    // table into shared memory now -- into the accumulator area, which is not in use until the first copies of
+    // the entry stream are under way -- and looks there first (columns outside the window: global memory).
+    const uint32_t win_bar = smem_u32(&bars[teams * p.D]);
+    const uint32_t *win = reinterpret_cast<const uint32_t *>(smem + lay.acc);
+    int win_w0 = 0, win_n = 0;                                     // first table word in the window, words in it
+    if (p.win_cols > 0) {
+        const int mid = (int)(((int64_t)(2 * kslice + 1) * p.K) / (2 * nK));
+        const int c0 = max(0, min(p.K - p.win_cols, mid - p.win_cols / 2));
+        win_w0 = (c0 * p.S) & ~3;
+        win_n = min(((c0 + p.win_cols) * p.S + 1 - win_w0 + 3) & ~3, ((p.K * p.S + 1 + 3) & ~3) - win_w0);
+        if (tid == 0) {
+            mbar_init(win_bar, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(win_bar), "r"((uint32_t)win_n * 4u) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                             smem_u32(win)),
+                         "l"(p.meta + win_w0), "r"((uint32_t)win_n * 4u), "r"(win_bar)
+                         : "memory");
+        }
     }
     if (tid < 4) zero_group[tid] = 0;
-    if (streams && member == 0 && lane == 0) {
+    if (streams && lane == 0) {
         for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -347,7 +422,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     // and the warp scans the survivor counts of its block of 32 words:
     //   kbw[w]  keep bits of activations 32w .. 32w+31,
     //   wrel[w] survivors in the words before w of the same block of 32 words,
-    //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
+    //   blk[e]  survivors in block e.
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
     const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 31) >> 5;
     {
@@ -394,17 +469,23 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 kbw[w] = word;
                 wrel[w] = incl - cnt;
             }
-            if (lane == 31 && (w >> 5) < nblk) const_cast<int *>(blk)[w >> 5] = incl;
+            if (lane == 31 && (w >> 5) < nblk) blk[w >> 5] = incl;
         }
     }
     CELTY_MARK(10);
     __syncthreads();
     CELTY_MARK(1);
-    // ---- ranks: every streaming warp turns the block counts into survivors before each block for itself, 32
-    // blocks at a time (a copy per warp costs a few hundred bytes and saves a block-wide barrier behind a single
-    // warp); the list is then cut into equal shares for the groups that work on different columns.
+    bool failed = false;
+    // the window has had the whole thresholding pass to arrive; nobody may clear an accumulator before it has
+    if (p.win_cols > 0 && !mbar_wait_bounded(win_bar, 0, p.spin_limit)) {
+        failed = true;
+        win_n = 0;
+    }
+    // ---- ranks: every warp turns the block counts into survivors before each block for itself, 32 blocks at a
+    // time.  All warps store the same numbers into the one table and each reads only what it has stored itself,
+    // which saves a block-wide barrier behind a single scanning warp.
     int n_surv = 0;
-    if (streams) {
+    {
         int carry = 0;
         for (int e0 = 0; e0 < nblk; e0 += 32) {
             const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
@@ -414,219 +495,221 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 const int up = __shfl_up_sync(kFull, incl, d);
                 if (lane >= d) incl += up;
             }
-            if (e < nblk) myblk[e] = carry + incl - cnt;
+            if (e < nblk) blkx[e] = carry + incl - cnt;
             carry += __shfl_sync(kFull, incl, 31);
         }
         __syncwarp();
         n_surv = carry;
-        if (blockIdx.x == 0 && warp == 0 && lane == 0) *p.count = carry;
+        if (blockIdx.x == 0 && tid == 0) *p.count = carry;
+    }
+    // The survivor list is cut into nK runs of ranks, one per block of this row part: n / nK each, the first
+    // n mod nK blocks one more.  n / nK without a division: slices_inv = floor(2^32 / nK) gives a quotient that is
+    // at most one too small.
+    int rb0, rb1;
+    {
+        const uint32_t inv = long_part ? p.slices_inv_long : p.slices_inv;
+        uint32_t share = __umulhi((uint32_t)n_surv, inv), extra = (uint32_t)n_surv - share * (uint32_t)nK;
+        if (extra >= (uint32_t)nK) { ++share; extra -= (uint32_t)nK; }
+        rb0 = kslice * (int)share + min(kslice, (int)extra);
+        rb1 = rb0 + (int)share + (kslice < (int)extra ? 1 : 0);
     }
     CELTY_MARK(2);
 
-    if (streams) {
-        // group u of nK * G owns n / units ranks, the first n mod units groups one more.  n / units without a
-        // division: units_inv = floor(2^32 / units) gives a quotient that is at most one too small
-        const uint32_t units = (uint32_t)(nK * p.G), units_inv = long_part ? p.units_inv_long : p.units_inv;
-        uint32_t share = __umulhi((uint32_t)n_surv, units_inv), extra = (uint32_t)n_surv - share * units;
-        if (extra >= units) { ++share; extra -= units; }
-        const int u = kslice * p.G + g;
-        const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
-        const int team_threads = 32 * p.W, bar_id = 1 + team;
-        const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
-        const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
-        const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
-        const uint32_t bar0 = smem_u32(&bars[team * p.D]);
-        bool zeroed = false;
-        const uint32_t lt_mask = (1u << lane) - 1u;
-        const uint32_t items0 = smem_u32(items);
-        uint32_t issued = 0, consumed = 0;                            // ring positions of this team
-        uint32_t slot = 0, parity = 0, islot = 0;                     // consumed % D, (consumed / D) & 1, issued % D
-        bool failed = false;
-        long long dbg_wait = 0, dbg_head = 0, dbg_loop = 0, dbg_tail = 0, dbg_steps = 0;   // development builds
-        (void)dbg_wait; (void)dbg_head; (void)dbg_loop; (void)dbg_tail; (void)dbg_steps;
-        StepBuf b0, b1;                                               // pipeline registers, live across items
-        const uint32_t zeros = smem_u32(zero_group);
+    // ---- a2-a4, in passes of at most `cap` columns (one pass on every configured shape)
+    const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
+    const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
+    const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
+    const uint32_t bar0 = smem_u32(&bars[team * p.D]);
+    const uint32_t note0 = smem_u32(smem + lay.note) + 4u * (uint32_t)(team * p.D);
+    uint2 *imeta_all = reinterpret_cast<uint2 *>(smem + lay.imeta);           // [Sc][cap] {offset/16, bytes}
+    const uint2 *imeta = imeta_all + (size_t)sl * p.cap;                      // this team's slab
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const uint32_t zeros = smem_u32(zero_group);
+    bool zeroed = false;
+    uint32_t slot = 0, parity = 0, islot = 0;                      // ring position: consumed % D, its phase, issued % D
+    StepBuf b0, b1;                                                // pipeline registers, live across columns
 
-        for (int rb = r_begin; rb < r_end; rb += p.cap) {
-            const int cnt = min(p.cap, r_end - rb);
-            // ---- column of rank r: the lane whose words hold it, then the word, then the bit
-            for (int i = member * 32 + lane; i < cnt; i += team_threads) {
-                const int r = rb + i;
-                // the block of 32 keep words that holds rank r (the last one with blk[e] <= r), the word in it
-                // (the last one with wrel[w] <= what is left) ...
-                int e = 0;
-                for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
-                    if (e + step < nblk && myblk[e + step] <= r) e += step;
-                int k = r - myblk[e], w = 32 * e;
-#pragma unroll
-                for (int step = 16; step; step >>= 1)
-                    if (w + step < nwords && wrel[w + step] <= k) w += step;
-                k -= wrel[w];
-                // ... and the bit in it: halve the word, keep the half that holds the wanted set bit
-                const uint32_t word = kbw[w];
-                int pos = 0;
-#pragma unroll
-                for (int sh = 16; sh; sh >>= 1) {
-                    const int c = __popc((word >> pos) & ((1u << sh) - 1u));
-                    if (k >= c) { k -= c; pos += sh; }
-                }
-                if (!CELTY_CHECK(((word >> pos) & 1u) != 0 && k == 0, 8, w)) pos = 0;
-                int j = 32 * w + pos;
-                if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
-                const uint16_t xb = p.x[j];
-                items[i] = make_int2(j, (int)xb);
-                if (part == 0 && sl == 0 && CELTY_CHECK(r >= 0 && r < p.K, 10, r)) {
-                    p.idx[r] = j;
-                    p.val[r] = xb;
-                }
-                if (s < p.S) {
-                    const uint32_t o0 = p.meta[(size_t)j * p.S + s], o1 = p.meta[(size_t)j * p.S + s + 1];
-                    imeta[i] = make_uint2(o0, (o1 - o0) * 16u);
-                    if (!CELTY_CHECK(o1 > o0 && (o1 - o0) * 16u <= (uint32_t)p.slot_bytes &&
-                                         (long long)o1 * 16 <= p.stream_bytes, 4, o1 - o0))
-                        imeta[i] = make_uint2(0u, (uint32_t)kSubHeader);
-                }
+    for (int w0 = rb0; w0 < rb1; w0 += p.cap) {
+        const int w1 = min(rb1, w0 + p.cap), n = w1 - w0;
+        if (w0 > rb0) __syncthreads();                             // everybody is done with the previous pass's list
+        // every team starts with D columns of its own (positions g, g + G, ...); the rest are handed out one at a time
+        if (tid < p.Sc) next[tid] = p.D * p.G;
+        // ---- the threads write the columns of ranks [w0, w1) into the list: a keep word knows the rank of its
+        // first survivor (survivors before its block + before it within the block)
+        for (int w = tid; w < nwords; w += nthreads) {
+            const int base = blkx[w >> 5] + wrel[w];
+            uint32_t word = kbw[w];
+            if (base >= w1 || base + __popc(word) <= w0) continue;
+            for (int r = base; word; ++r) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+                if (r >= w0 && r < w1) items[r - w0].x = 32 * w + b;
             }
-
-            team_sync(bar_id, team_threads);
-            if (s >= p.S) continue;
-            // ---- a2: keep D copies in flight.  The team's first warp issues the first D of a batch and refills a
-            // slot whenever the team has finished with it.  (A dedicated producer warp that polled per-slot
-            // "empty" barriers was measured and was no faster at any configured shape.)  Every lane of that warp
-            // calls issue(), converged, and keeps the ring position; one elected lane (elect.sync) runs the two
-            // instructions under a predicate -- 3 % faster at 28672 x 8192 than a branch on lane 0, around which
-            // the warp diverges and reconverges for every sub-block.
-            auto issue_im = [&](const uint2 im) {
-                bulk_load_elected(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y,
-                                  bar0 + 8u * islot);
-                ++issued;
-                if (++islot == (uint32_t)p.D) islot = 0;
-            };
-            auto issue = [&](int i) { issue_im(imeta[i]); };
-            if (member == 0 && !failed)
-                for (int i = 0; i < min(cnt, p.D); ++i) issue(i);
-            CELTY_MARK(3);
-            if (!zeroed) {                                          // clear the slab while the first copies fly
-                float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
-                for (int i = member * 32 + lane; i < slab_words / 4; i += team_threads) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                zeroed = true;
-                team_sync(bar_id, team_threads);
-            }
-            for (int i = 0; i < cnt; ++i) {
-                const long long t_a = CELTY_CLOCK();
-                uint32_t xbits;                                       // the column's activation: asked for before the wait
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(items0 + 8u * (uint32_t)i + 4u));
-                // A warp that gave up on a copy keeps walking the items (and the team barriers) without
-                // touching them, so that the warps of a team never wait for one another in vain.
-                if (!failed && !mbar_wait_bounded(bar0 + 8u * slot, parity)) failed = true;
-                failed = __any_sync(kFull, failed);
-                if (i == 0) CELTY_MARK(4);
-                const long long t_b = CELTY_CLOCK();
-                ++consumed;
-                if (failed) {
-                    team_sync(bar_id, team_threads);
-                    if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
-                    continue;
-                }
-                const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
-                // what the refill at the end of this sub-block will need, read now so that it does not wait then
-                const bool refill = member == 0 && i + p.D < cnt;
-                const uint2 next_im = refill ? imeta[i + p.D] : make_uint2(0u, 0u);
-                const uint16_t xj = (uint16_t)xbits;
-                // ---- a3 + a4.  Header: groups per lane, split points, totals (see kSubHeader).
-                uint32_t gl, hw;
-                asm volatile("ld.shared.u8 %0, [%1];" : "=r"(gl) : "r"(sub + lane));
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw) : "r"(sub + 136));      // vectors | steps << 16
-                const uint32_t steps = hw >> 16, Gs = hw & 0xFFFFu;
-                const uint32_t vbase = sub + kSubHeader, rbase = vbase + 16 * Gs;
-                const uint32_t slot_end = sub + (uint32_t)p.slot_bytes;
-                // this warp's range of steps [q_lo, q_hi), its first vector and its lanes' first rows
-                uint32_t q_lo = 0, q_hi = steps, cum = 0, row0 = 0;
-                if (p.W > 1) {
-                    const uint32_t k_lo = (uint32_t)member * (4u / (uint32_t)p.W);       // split index 0..3
-                    const uint32_t k_hi = k_lo + 4u / (uint32_t)p.W;
-                    q_lo = (k_lo * steps + 3) >> 2;
-                    q_hi = k_hi >= 4 ? steps : (k_hi * steps + 3) >> 2;
-                    if (k_lo) {
-                        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(cum) : "r"(sub + 126 + 2 * k_lo));
-                        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(row0) : "r"(sub + 32 * k_lo + lane));
-                    }
-                }
-                uint32_t cell = cell0 + row0 * 128u;
-                const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
-                const long long t_c = CELTY_CLOCK();
-                step_fetch(b0, gl, q_lo, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                step_fetch(b1, gl, q_lo + 1, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                step_decode(b0, cell, spare, slab0, slab_end);                                    // step q_lo
-                step_fetch(b0, gl, q_lo + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                uint32_t q = q_lo + 1;
-#pragma unroll 2
-                for (; q + 1 < q_hi; q += 2) {                                             // two real steps per pass
-                    step_decode(b1, cell, spare, slab0, slab_end);                                // step q
-                    step_finish(b0, xj);                                                   // step q-1
-                    step_fetch(b1, gl, q + 2, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                    step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
-                    step_finish(b1, xj);                                                   // step q
-                    step_fetch(b0, gl, q + 3, q_hi, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                }
-                if (q < q_hi) {                                                            // one real step left
-                    step_decode(b1, cell, spare, slab0, slab_end);
-                    step_finish(b0, xj);
-                    step_finish(b1, xj);
-                } else {                                                                   // only the last one to finish
-                    step_finish(b0, xj);
-                }
-                const long long t_d = CELTY_CLOCK();
-                // every warp of the team is done with this sub-block (and with its rows) before the
-                // slot is refilled and before anybody touches the accumulator for the next column
-                team_sync(bar_id, team_threads);
-                // The slot's contents were consumed by loads whose values have been used, and the barrier
-                // above orders every team member's reads before this point: the copy may overwrite it.
-                if (refill) issue_im(next_im);
-                if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
-                dbg_wait += t_b - t_a; dbg_head += t_c - t_b; dbg_loop += t_d - t_c; dbg_tail += CELTY_CLOCK() - t_d;
-                dbg_steps += q_hi - q_lo;
-            }
-            CELTY_STORE(11, dbg_wait); CELTY_STORE(12, dbg_head); CELTY_STORE(13, dbg_loop); CELTY_STORE(14, dbg_tail);
-            CELTY_STORE(15, dbg_steps);
-            issued = __shfl_sync(kFull, issued, 0);
-            islot = __shfl_sync(kFull, islot, 0);
-            team_sync(bar_id, team_threads);                      // items / imeta are rewritten by the next batch
         }
-        if (!zeroed && s < p.S) {                                     // a team without columns still owns a slab
+        __syncthreads();
+        CELTY_MARK(11);
+        if (!streams) continue;
+        // ---- the streaming warps fetch, for every listed column, its activation and the offsets of its sub-blocks
+        // (one round trip to L2 for the lot); row part 0 also writes the list for the API
+        for (int i = warp * 32 + lane; i < n; i += teams * 32) {
+            int j = items[i].x;
+            if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
+            const uint16_t xb = __ldg(p.x + j);                      // x went through L1 in the thresholding pass
+            for (int f = 0; f < p.Sc; ++f) {
+                const int sf = part * p.Sc + f;
+                if (sf >= p.S) break;
+                const int wq = j * p.S + sf - win_w0;                  // the window is there in the first pass only
+                uint32_t o0, o1;
+                if (w0 == rb0 && wq >= 0 && wq + 1 < win_n) {
+                    o0 = win[wq];
+                    o1 = win[wq + 1];
+                } else {
+                    o0 = p.meta[(size_t)j * p.S + sf];
+                    o1 = p.meta[(size_t)j * p.S + sf + 1];
+                }
+                uint2 im = make_uint2(o0, (o1 - o0) * 16u);
+                if (!CELTY_CHECK(o1 > o0 && (o1 - o0) * 16u <= (uint32_t)p.slot_bytes &&
+                                     (long long)o1 * 16 <= p.stream_bytes, 4, o1 - o0))
+                    im = make_uint2(0u, (uint32_t)kSubHeader);
+                imeta_all[(size_t)f * p.cap + i] = im;
+            }
+            items[i].y = (int)xb;
+            if (part == 0) {
+                p.idx[w0 + i] = j;
+                p.val[w0 + i] = xb;
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"r"(teams * 32) : "memory");      // the streaming warps only
+        if (s >= p.S) continue;
+        // ---- a2: keep D copies in flight.  Every lane calls issue(), converged, and keeps the ring position; one
+        // elected lane (elect.sync) runs the instructions under a predicate -- measured 3 % faster at 28672 x 8192
+        // than a branch on lane 0, around which the warp diverges and reconverges for every sub-block.
+        uint32_t issued = 0, consumed = 0;
+        auto issue = [&](const uint2 im, uint32_t xbits) {
+            bulk_load_elected(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y,
+                              bar0 + 8u * islot, note0 + 4u * islot, xbits);
+            ++issued;
+            if (++islot == (uint32_t)p.D) islot = 0;
+        };
+        const uint32_t next_addr = smem_u32(&next[sl]);
+        uint32_t taken = (uint32_t)n, leader = 0;                  // the list position for the refill after next
+        if (!failed)
+            for (int d = 0, i = g; d < p.D && i < n; ++d, i += p.G) issue(imeta[i], (uint32_t)items[i].y);
+        if (issued == (uint32_t)p.D) {
+            if (p.fixed_deal) taken = (uint32_t)(g + p.D * p.G);
+            else take_elected(next_addr, taken, leader);
+        }
+        CELTY_MARK(3);
+        if (!zeroed) {                                              // clear the slab while the first copies fly
             float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
-            for (int i = member * 32 + lane; i < slab_words / 4; i += team_threads) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            zeroed = true;
+        }
+        __syncwarp();
+        while (consumed < issued) {
+            uint32_t xbits;                                           // the column's activation: asked for before the wait
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(note0 + 4u * slot));
+            if (!mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
+            failed = __any_sync(kFull, failed);
+            if (failed) break;                                        // the copies still in flight are awaited below
+            if (consumed == 0) CELTY_MARK(4);
+            const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
+            // what the refill at the end of this sub-block will need, read now so that it does not wait then
+            const int pend = (int)__shfl_sync(kFull, taken, leader);
+            const bool refill = pend < n;
+            const uint2 next_im = refill ? imeta[pend] : make_uint2(0u, 0u);
+            const uint32_t next_x = refill ? (uint32_t)items[pend].y : 0u;
+            const uint16_t xj = (uint16_t)xbits;
+            // ---- a3 + a4.  Header: groups per lane, vectors and steps (see kSubHeader).
+            uint32_t gl, hw;
+            asm volatile("ld.shared.u8 %0, [%1];" : "=r"(gl) : "r"(sub + lane));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw) : "r"(sub + 32));       // vectors | steps << 16
+            const uint32_t steps = hw >> 16, Gs = hw & 0xFFFFu;
+            const uint32_t vbase = sub + kSubHeader, rbase = vbase + 16 * Gs;
+            const uint32_t slot_end = sub + (uint32_t)p.slot_bytes;
+            uint32_t cum = 0, cell = cell0;
+            const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
+            step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+            step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+            step_decode(b0, cell, spare, slab0, slab_end);                                    // step 0
+            step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+            uint32_t q = 1;
+#pragma unroll 2
+            for (; q + 1 < steps; q += 2) {                                            // two real steps per pass
+                step_decode(b1, cell, spare, slab0, slab_end);                                // step q
+                step_finish(b0, xj);                                                   // step q-1
+                step_fetch(b1, gl, q + 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
+                step_finish(b1, xj);                                                   // step q
+                step_fetch(b0, gl, q + 3, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+            }
+            if (q < steps) {                                                           // one real step left
+                step_decode(b1, cell, spare, slab0, slab_end);
+                step_finish(b0, xj);
+                step_finish(b1, xj);
+            } else {                                                                   // only the last one to finish
+                step_finish(b0, xj);
+            }
+            // The slot's contents were consumed by loads whose values have been used, and the barrier orders
+            // every lane's reads before this point: the copy may overwrite it.
+            __syncwarp();
+            if (refill) {                                           // copy + the take for the refill after this one
+                if (p.fixed_deal) {
+                    issue(next_im, next_x);
+                    taken += (uint32_t)p.G;
+                } else {
+                    bulk_load_elected_take(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)next_im.x * 16,
+                                           next_im.y, bar0 + 8u * islot, note0 + 4u * islot, next_x, next_addr, taken, leader);
+                    ++issued;
+                    if (++islot == (uint32_t)p.D) islot = 0;
+                }
+            }
+            ++consumed;
+            if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
         }
         if (failed) {
-            // give copies that are still in flight a last (bounded) chance to land before the block exits
-            if (member == 0)
-                for (; consumed < issued; ++consumed)
-                    mbar_wait_bounded(bar0 + 8u * (consumed % (uint32_t)p.D), (consumed / (uint32_t)p.D) & 1u);
+            // give the copies that are still in flight a last (bounded) chance to land before the block goes on
+            for (; consumed < issued; ++consumed) {
+                mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit);
+                if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
+            }
             if (lane == 0) atomicOr(p.status, kStatusTimeout);
         }
+    }
+    if (failed && lane == 0) atomicOr(p.status, kStatusTimeout);
+    if (streams && !zeroed && s < p.S) {                              // a team without columns still owns a slab
+        float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
+        for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     __syncthreads();
     CELTY_MARK(5);
 
     if (p.merge == 1) {
-        // ---- a5 by bulk reduce-add: the block adds its G accumulators and the copy engine adds every 32*C-row
-        // segment into y (cp.reduce.async.bulk, FP32 add at L2).  y was cleared by all blocks at the start; the
-        // ticket makes sure of it.
+        // ---- a5 by bulk reduce-add.  The block adds its G accumulators; the row segments of its slabs (32*C rows
+        // of y each, see the row map) are then dealt to the blocks of the cluster, a block adds its peers' sums
+        // for its segments (through distributed shared memory), and the copy engine adds the result into y
+        // (cp.reduce.async.bulk, FP32 add at L2).  y was cleared by all blocks at the start; the ticket makes
+        // sure of it.
         if (warp == nwarps - 1 && lane == 0) {                      // every block's share of y is cleared by now
             const bool low_half = y_ticket < gridDim.x;
             bool ok = false;
-            for (uint32_t it = 0; it < kSpinLimit; ++it) {
+            for (uint32_t it = 0; it < p.spin_limit; ++it) {
                 const uint32_t cur = ld_relaxed_u32(&p.tickets[0]);
                 if (low_half ? (cur >= gridDim.x) : (cur < gridDim.x)) { ok = true; break; }
                 __nanosleep(64);
             }
             __threadfence();
+            // the clearing stores of the other blocks (generic proxy) come before this block's reduce-adds
+            // (asynchronous proxy) to the same addresses
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             if (!ok) atomicOr(p.status, kStatusTimeout);
         }
-        // add the G accumulators into the first one
+        __syncwarp();
+        // add the G accumulators of every slab into the first one
+        const int group_words = p.Sc * slab_words;
         if (p.G > 1) {
             float4 *acc4 = reinterpret_cast<float4 *>(acc);
-            const int group4 = p.Sc * slab_words / 4;
+            const int group4 = group_words / 4;
             for (int q4 = tid; q4 < group4; q4 += nthreads) {
                 float4 v = acc4[q4];
                 for (int gg = 1; gg < p.G; ++gg) {
@@ -636,14 +719,32 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 acc4[q4] = v;
             }
         }
+        const int seg = p.S == 1 ? 16 : p.C, nseg = (p.R + seg - 1) / seg, seg4 = seg * 8;
+        const int owned = (p.Sc * nseg - crank + p.cl - 1) / p.cl;   // segments crank, crank + cl, ...
+        if (p.cl > 1) {
+            cluster_sync();                                         // the peers' sums are complete
+            for (int t = tid; t < owned * seg4; t += nthreads) {
+                const int sg = crank + p.cl * (t / seg4), q4 = t % seg4;
+                const int fsl = sg / nseg, i0 = (sg - fsl * nseg) * seg;
+                if (i0 * 32 + q4 * 4 >= p.R * 32) continue;         // a slab's last segment may be short
+                float4 *cellp = reinterpret_cast<float4 *>(acc + (size_t)fsl * slab_words + (size_t)i0 * 32 + (size_t)q4 * 4);
+                float4 v = *cellp;
+                for (int b = 1; b < p.cl; ++b) {
+                    const float4 u = ld_cluster_f4(smem_u32(cellp), (uint32_t)((crank + b) % p.cl));
+                    v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+                }
+                // no other block reads this place: a block reads only the segments it owns, from everybody
+                *cellp = v;
+            }
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
         CELTY_MARK(6);
         // The row map makes local rows [kC, kC + C) of a slab 32*C consecutive rows of y, in accumulator
         // order (with one slab the whole accumulator is y itself): each such segment is one bulk reduce-add.
         {
-            const int seg = p.S == 1 ? 16 : p.C, nseg = (p.R + seg - 1) / seg;
-            for (int sg = tid; sg < p.Sc * nseg; sg += nthreads) {
+            for (int o = tid; o < owned; o += nthreads) {
+                const int sg = crank + p.cl * o;
                 const int fsl = sg / nseg, k = sg - fsl * nseg, sfull = part * p.Sc + fsl;
                 if (sfull >= p.S) continue;
                 const int i0 = k * seg, i1 = min(p.R, i0 + seg);
@@ -663,90 +764,92 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may go once it has been read
         }
         CELTY_MARK(7);
-    } else {
-        // ---- a5, stage 1: add the G accumulators, store the block's partial (accumulator layout, no slack rows)
-        const int tile_words = p.R * 32, part_words = p.Sc * tile_words;
-        {
-            float4 *mine4 = reinterpret_cast<float4 *>(p.partials + (size_t)blockIdx.x * part_words);
-            const float4 *acc4 = reinterpret_cast<const float4 *>(acc);
-            const int tile4 = tile_words >> 2, slab4 = slab_words >> 2, group4 = p.Sc * slab4;
-            for (int fsl = 0; fsl < p.Sc; ++fsl)
-                for (int q4 = tid; q4 < tile4; q4 += nthreads) {
-                    const float4 *src = acc4 + fsl * slab4 + q4;
-                    float4 v = src[0];
-                    for (int gg = 1; gg < p.G; ++gg) {
-                        const float4 t = src[gg * group4];
-                        v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
-                    }
-                    __stcg(mine4 + fsl * tile4 + q4, v);
-                }
-        }
-        __syncthreads();
-        CELTY_MARK(6);
-        if (tid == 0) {
-            __threadfence();                                          // the block's stores, ordered by the barrier above
-            atomicAdd(&p.tickets[0], 1u);
-            bool ok = false;
-            for (uint32_t it = 0; it < kSpinLimit; ++it) {
-                if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
-                __nanosleep(32);
-            }
-            if (!ok) atomicOr(p.status, kStatusTimeout);
-        }
-        __syncthreads();
-        CELTY_MARK(7);
+        if (p.cl > 1) cluster_sync();                               // no block leaves while a peer may still read it
+        return;
+    }
 
-        // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
-        // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
-        // every lane has up to 16 loads in flight, then the ranges are added in a fixed order.
-        {
-            float *red = reinterpret_cast<float *>(smem + lay.acc);   // the accumulators are no longer needed
-            const int wpc = (((part_words + nK - 1) / nK) + 31) & ~31;
-            const int wb = kslice * wpc, we = min(part_words, wb + wpc);
-            const int nchunks = max(0, (we - wb + 31) >> 5);
-            const size_t stride = (size_t)p.P * part_words;
-            for (int c0 = 0; c0 < nchunks; c0 += nwarps) {
-                const int pass_chunks = min(nwarps, nchunks - c0);
-                const int nsplit = nwarps / pass_chunks;              // warps per chunk in this pass
-                const int my_chunk = warp % pass_chunks, my_split = warp / pass_chunks;
-                const int word = wb + 32 * (c0 + my_chunk) + lane;
-                if (my_split < nsplit) {
-                    float sum = 0.f;
-                    if (word < we) {
-                        const int per = (nK + nsplit - 1) / nsplit;
-                        const int b_lo = my_split * per, b_hi = min(nK, b_lo + per);
-                        const float *src = p.partials + (size_t)part * part_words + word;
-                        for (int b0 = b_lo; b0 < b_hi; b0 += 16) {
-                            float t[16];
-    #pragma unroll
-                            for (int k = 0; k < 16; ++k)
-                                t[k] = (b0 + k < b_hi && CELTY_CHECK((size_t)(b0 + k) * stride + (size_t)part * part_words + word <
-                                                                         (size_t)gridDim.x * part_words, 13, b0 + k))
-                                           ? __ldcg(src + (size_t)(b0 + k) * stride) : 0.f;
-    #pragma unroll
-                            for (int k = 0; k < 16; ++k) sum += t[k];
-                        }
-                    }
-                    red[(my_split * pass_chunks + my_chunk) * 32 + lane] = sum;
+    // ---- a5, ordered: stage 1 adds the G accumulators and stores the block's partial (accumulator layout, no
+    // slack rows).  (Clusters are not used with this merge: cl == 1, so block b of part `part` is b * P + part.)
+    const int tile_words = p.R * 32, part_words = p.Sc * tile_words;
+    {
+        float4 *mine4 = reinterpret_cast<float4 *>(p.partials + (size_t)blockIdx.x * part_words);
+        const float4 *acc4 = reinterpret_cast<const float4 *>(acc);
+        const int tile4 = tile_words >> 2, slab4 = slab_words >> 2, group4 = p.Sc * slab4;
+        for (int fsl = 0; fsl < p.Sc; ++fsl)
+            for (int q4 = tid; q4 < tile4; q4 += nthreads) {
+                const float4 *src = acc4 + fsl * slab4 + q4;
+                float4 v = src[0];
+                for (int gg = 1; gg < p.G; ++gg) {
+                    const float4 t = src[gg * group4];
+                    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
                 }
-                __syncthreads();
-                if (warp < pass_chunks) {
-                    const int w2 = wb + 32 * (c0 + warp) + lane;
-                    if (w2 < we) {
-                        float total = 0.f;
-                        for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
-                        const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
-                        const int sfull = part * p.Sc + fsl;
-                        const int64_t row = tile_row(p.S, p.C, sfull, rem & 31, rem >> 5);
-                        if (sfull < p.S && row < p.M) p.y[row] = total;
-                    }
-                }
-                __syncthreads();
+                __stcg(mine4 + fsl * tile4 + q4, v);
             }
+    }
+    __syncthreads();
+    CELTY_MARK(6);
+    if (tid == 0) {
+        __threadfence();                                          // the block's stores, ordered by the barrier above
+        atomicAdd(&p.tickets[0], 1u);
+        bool ok = false;
+        for (uint32_t it = 0; it < p.spin_limit; ++it) {
+            if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
+            __nanosleep(32);
+        }
+        if (!ok) atomicOr(p.status, kStatusTimeout);
+    }
+    __syncthreads();
+    CELTY_MARK(7);
+
+    // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
+    // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
+    // every lane has up to 16 loads in flight, then the ranges are added in a fixed order.
+    {
+        float *red = reinterpret_cast<float *>(smem + lay.acc);   // the accumulators are no longer needed
+        const int wpc = (((part_words + nK - 1) / nK) + 31) & ~31;
+        const int wb = kslice * wpc, we = min(part_words, wb + wpc);
+        const int nchunks = max(0, (we - wb + 31) >> 5);
+        const size_t stride = (size_t)p.P * part_words;
+        for (int c0 = 0; c0 < nchunks; c0 += nwarps) {
+            const int pass_chunks = min(nwarps, nchunks - c0);
+            const int nsplit = nwarps / pass_chunks;              // warps per chunk in this pass
+            const int my_chunk = warp % pass_chunks, my_split = warp / pass_chunks;
+            const int word = wb + 32 * (c0 + my_chunk) + lane;
+            if (my_split < nsplit) {
+                float sum = 0.f;
+                if (word < we) {
+                    const int per = (nK + nsplit - 1) / nsplit;
+                    const int b_lo = my_split * per, b_hi = min(nK, b_lo + per);
+                    const float *src = p.partials + (size_t)part * part_words + word;
+                    for (int bb = b_lo; bb < b_hi; bb += 16) {
+                        float t[16];
+#pragma unroll
+                        for (int k = 0; k < 16; ++k)
+                            t[k] = (bb + k < b_hi && CELTY_CHECK((size_t)(bb + k) * stride + (size_t)part * part_words + word <
+                                                                     (size_t)gridDim.x * part_words, 13, bb + k))
+                                       ? __ldcg(src + (size_t)(bb + k) * stride) : 0.f;
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) sum += t[k];
+                    }
+                }
+                red[(my_split * pass_chunks + my_chunk) * 32 + lane] = sum;
+            }
+            __syncthreads();
+            if (warp < pass_chunks) {
+                const int w2 = wb + 32 * (c0 + warp) + lane;
+                if (w2 < we) {
+                    float total = 0.f;
+                    for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
+                    const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
+                    const int sfull = part * p.Sc + fsl;
+                    const int64_t row = tile_row(p.S, p.C, sfull, rem & 31, rem >> 5);
+                    if (sfull < p.S && row < p.M) p.y[row] = total;
+                }
+            }
+            __syncthreads();
         }
     }
     CELTY_MARK(8);
-    if (p.merge == 1) return;
     __syncthreads();
     if (tid == 0) {
         const uint32_t t = atomicAdd(&p.tickets[1], 1u);
@@ -759,11 +862,11 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 }
 
 struct FusedPlan {
-    int G, Sc, P, D, W, slot_bytes, cap, threads, grid, merge;
+    int G, Sc, P, D, cl, slot_bytes, cap, threads, grid, merge;
     size_t smem;
 };
 
 inline size_t fused_smem_bytes(int R, int K, int G, int Sc, int D, int slot_bytes, int cap)
 {
-    return fused_smem_layout(R, K, G * Sc, D, slot_bytes, cap).total;
+    return fused_smem_layout(R, K, G * Sc, Sc, D, slot_bytes, cap).total;
 }

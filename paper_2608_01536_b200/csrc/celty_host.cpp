@@ -106,7 +106,8 @@ void pack_column(celty_matrix *m, const Logical &lg)
 
 // Build the LANE_TILE image: meta uint32[K*S + 1] (offset/16 of each sub-block), then per
 // (column j, slab s) a sub-block
-//   [32 x u8: groups of lane L's tile 32s+L][G x 16 B values][G x 4 B runs], padded to 16 bytes,
+//   [48 B header: 32 x u8 groups of lane L's tile 32s+L, u32 vectors | steps << 16][G x 16 B values][G x 4 B runs],
+// padded to 16 bytes,
 // G = sum of the lanes' group counts.  Vectors are stored step-major: for step q = 0, 1, ... the
 // lanes that still have a q-th group, in lane order, so that a warp reads one contiguous span per step.
 void pack_lane_tile(celty_matrix *m, const Logical &lg)
@@ -149,24 +150,9 @@ void pack_lane_tile(celty_matrix *m, const Logical &lg)
                 G += g[L];
                 steps = std::max(steps, g[L]);
             }
-            // split points for up to four cooperating warps (see kSubHeader)
-            for (int k = 1; k <= 3; ++k) {
-                const uint64_t qk = (k * steps + 3) / 4;
-                uint64_t before = 0;
-                for (int L = 0; L < 32; ++L) {
-                    const uint64_t gq = std::min<uint64_t>(g[L], qk);        // groups of this lane before step q_k
-                    before += gq;
-                    uint64_t row = 0;                                          // rows those groups span
-                    for (uint64_t e = 0; e < std::min<uint64_t>(n[L], gq * kGroup); ++e) row += lg.runs[e0[L] + e] + 1;
-                    if (gq * kGroup > n[L]) row += gq * kGroup - n[L];         // zero-run slots that fill the last group
-                    sub[32 * k + L] = (uint8_t)row;
-                }
-                const uint16_t b16 = (uint16_t)before;
-                std::memcpy(sub + 128 + 2 * (k - 1), &b16, 2);
-            }
             {
                 const uint32_t gs = (uint32_t)G | ((uint32_t)steps << 16);
-                std::memcpy(sub + 136, &gs, 4);
+                std::memcpy(sub + 32, &gs, 4);
             }
             uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * G;
             uint64_t slot = 0;
@@ -473,19 +459,27 @@ extern "C" int celty_count_entries(const uint8_t *mask, int64_t ldm, int64_t M, 
 }
 
 extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth,
-                                int32_t team)
+                                int32_t cluster)
 {
-    if (!m || grid < 0 || variant < 0 || variant > 13 || groups < 0 || groups > 15 || depth < 0 || depth > 16 ||
-        !(team == 0 || team == 1 || team == 2 || team == 4))
+    if (!m || grid < 0 || variant < 0 || variant > 63 || groups < 0 || groups > 16 || depth < 0 || depth > 16 ||
+        !(cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4))
         return CELTY_EINVAL;
     m->grid = grid;
     // variant: bit 0 selects the two-launch path; 2 / 4 force the ordered two-stage / the bulk reduce-add merge
     m->merge = (variant & 2) ? 0 : (variant & 4) ? 1 : -1;
     m->no_overlap = (variant & 8) ? 1 : 0;
     m->variant = variant & 1;
+    m->exp_flags = (variant >> 4) & 3;
     m->groups = groups;
     m->depth = depth;
-    m->team = team;
+    m->cluster = cluster;
+    return CELTY_OK;
+}
+
+extern "C" int celty_set_wait_limit(celty_matrix *m, uint32_t polls)
+{
+    if (!m) return CELTY_EINVAL;
+    m->spin_limit = polls;
     return CELTY_OK;
 }
 

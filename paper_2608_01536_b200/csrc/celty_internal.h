@@ -12,13 +12,9 @@ constexpr int kGroup = 8;            // entries per 16-byte value vector / 32-bi
 constexpr int kChunkGroups = 32;     // COLUMN layout: groups per warp-wide chunk (256 entries)
 constexpr int kTileSlack = 8;        // LANE_TILE: spare accumulator rows per slab for group-tail slots
 // LANE_TILE sub-block header (bytes), ahead of the value vectors and run words:
-//   [0,32)    groups of 8 entries that lane L's tile holds (u8)
-//   [32,128)  for k = 1,2,3: the lane's local row after its first q_k groups (u8 each), where
-//             q_k = ceil(k * steps / 4) and steps = the largest group count -- lets up to four warps
-//             start decoding the same sub-block at those steps without reading the runs before them
-//   [128,134) for k = 1,2,3: vectors stored before step q_k (u16)
-//   [136,140) vectors in the sub-block | steps << 16 (u32);  rest zero
-constexpr int kSubHeader = 144;
+//   [0,32)   groups of 8 entries that lane L's tile holds (u8)
+//   [32,36)  vectors in the sub-block | steps << 16 (u32), steps = the largest group count;  rest zero
+constexpr int kSubHeader = 48;
 constexpr int kMaxTileRows = 240;    // keeps local rows (and the spare rows after them) in a byte
 constexpr int64_t kMaxM = 49152;     // accumulators of one thread block must fit shared memory
 constexpr size_t kAlign = 256;
@@ -99,7 +95,9 @@ struct celty_matrix {
     uint8_t *d_image = nullptr;
     uint8_t *d_ws = nullptr;
     celty::WorkspaceLayout ws{};
-    int32_t grid = 0, variant = 0, groups = 0, depth = 0, team = 0;
+    int32_t grid = 0, variant = 0, groups = 0, depth = 0, cluster = 0;
+    int32_t exp_flags = 0;                    // experiments: 1 = no offset window, 2 = columns dealt to teams in a fixed order
+    uint32_t spin_limit = 0;                  // bounded waits inside the kernels: 0 = the library's limit
     int32_t last_grid = 0, last_merge = -1;   // what the tickets in the workspace were last used with
     int32_t no_overlap = 0; // fused kernel: 1 = plain launch (no programmatic dependent launch)
     int32_t merge = -1;     // fused kernel: -1 = library's choice, 0 = ordered two-stage sum, 1 = bulk reduce-add

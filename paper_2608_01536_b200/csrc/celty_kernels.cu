@@ -386,24 +386,20 @@ int launch_compact(const void *x, int64_t K, float tau, int32_t *idx, uint16_t *
     return CELTY_OK;
 }
 
-// Shape of the fused launch: P row parts of Sc slabs, G groups (teams = G * Sc, one accumulator slab and one
-// ring of D slots each), W warps per team.
+// Shape of the fused launch: P row parts of Sc slabs, G teams per slab (teams = G * Sc warps, one accumulator
+// slab and one ring of D slots each), clusters of cl thread blocks that add their accumulators on chip.
 int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
 {
     FusedPlan pl{};
     pl.P = m->P;
     pl.Sc = m->Sc;
-    if (pl.Sc > 15) return CELTY_EINVAL;      // one hardware named barrier per team
+    if (pl.Sc > 16) return CELTY_EINVAL;      // one warp per team, 16 warps per block
     pl.slot_bytes = (int)round_up((size_t)m->max_unit16 * 16, 128);
-    pl.cap = 64;
+    pl.cap = pl.Sc <= 2 ? 512 : pl.Sc <= 4 ? 256 : 128;
     const size_t budget = (size_t)di.max_smem_optin;
-    // Warps per team: measurements on B200 show no gain from sharing a sub-block between warps at the
-    // configured sizes, so one warp per team unless asked otherwise.  Groups first (each needs its own
-    // accumulator), then as many ring slots as still fit (at least two, to keep a copy in flight).
-    pl.W = m->team > 0 ? m->team : 1;
-    while (pl.W > 1 && pl.Sc * pl.W > 16) pl.W >>= 1;       // a requested team size that does not fit is reduced
-    if (pl.Sc * pl.W > 16) return CELTY_EINVAL;
-    const int g_cap = std::min(15 / pl.Sc, std::max(1, 16 / (pl.Sc * pl.W)));
+    // Teams first (each needs its own accumulator), then as many ring slots as still fit (at least two, to
+    // keep a copy in flight).
+    const int g_cap = std::max(1, 16 / pl.Sc);
     const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
     const int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 4;
     pl.G = 0;
@@ -419,21 +415,93 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
         pl.D = 1;
     }
     if (pl.G == 0) return CELTY_EINVAL;
-    pl.threads = std::max(512, 32 * pl.G * pl.Sc * pl.W);
-    if (pl.threads > 512) return CELTY_EINVAL;
+    pl.threads = 512;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
     pl.merge = (m->merge >= 0 ? m->merge : 1);
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
     if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
     pl.grid = std::max(blocks, pl.P);           // any number of blocks >= P: parts may differ by one column slice
     if (pl.grid > di.sms) return CELTY_EINVAL;
+    // Clusters (bulk reduce-add merge only): pairs unless asked otherwise, as long as the grid is made of whole
+    // clusters, every row part gets at least one, and the device can hold them all at once.
+    pl.cl = pl.merge == 1 ? (m->cluster > 0 ? m->cluster : 1) : 1;
+    while (pl.cl > 1 && (pl.grid % pl.cl != 0 || pl.grid / pl.cl < pl.P)) pl.cl >>= 1;
     *out = pl;
+    return CELTY_OK;
+}
+
+// How many clusters of `cl` blocks of the fused kernel (with `smem` bytes of dynamic shared memory each) the
+// current device holds at once; asked of the runtime once per (device, cluster size, shared-memory KB).
+int max_active_clusters(int cl, size_t smem, int threads, int *out)
+{
+    struct Entry { int dev, cl, kb, n; };
+    static std::mutex mu;
+    static Entry cache[64];
+    static int used = 0;
+    int dev = 0;
+    CELTY_CUDA(cudaGetDevice(&dev));
+    const int kb = (int)((smem + 1023) / 1024);
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i)
+        if (cache[i].dev == dev && cache[i].cl == cl && cache[i].kb == kb) {
+            *out = cache[i].n;
+            return CELTY_OK;
+        }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cl);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = (size_t)kb * 1024;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cl;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    CELTY_CUDA(cudaOccupancyMaxActiveClusters(&n, k_spmspv_fused, &cfg));
+    if (used < 64) cache[used++] = Entry{dev, cl, kb, n};
+    *out = n;
+    return CELTY_OK;
+}
+
+// fall back to smaller clusters while the device cannot hold the whole grid of them at once
+int fit_clusters(FusedPlan *plan)
+{
+    while (plan->cl > 1) {
+        int fit = 0;
+        const int rc = max_active_clusters(plan->cl, plan->smem, plan->threads, &fit);
+        if (rc) return rc;
+        if (fit * plan->cl >= plan->grid) break;
+        plan->cl >>= 1;
+        while (plan->cl > 1 && (plan->grid % plan->cl != 0 || plan->grid / plan->cl < plan->P)) plan->cl >>= 1;
+    }
     return CELTY_OK;
 }
 
 }  // namespace
 
 extern "C" int celty_last_cuda_error(void) { return g_last_cuda; }
+
+extern "C" int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n)
+{
+    if (!m || !out || n < 10) return CELTY_EINVAL;
+    if (m->layout != CELTY_LAYOUT_LANE_TILE) return CELTY_EINVAL;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    FusedPlan plan;
+    rc = plan_fused(m, di, &plan);
+    if (rc) return rc;
+    rc = ensure_smem(k_spmspv_fused, plan.smem, g_granted_fused);
+    if (rc) return rc;
+    rc = fit_clusters(&plan);
+    if (rc) return rc;
+    const int32_t v[10] = {plan.grid, plan.threads, (int32_t)plan.smem, plan.G, plan.D, plan.cl, plan.P, plan.Sc,
+                           plan.slot_bytes, plan.merge};
+    for (int i = 0; i < 10; ++i) out[i] = v[i];
+    return CELTY_OK;
+}
 
 #if defined(CELTY_TRACE) || defined(CELTY_GUARD)
 // Development builds only: where the fused kernel stores its phase timestamps (device pointer, 16 per block).
@@ -489,6 +557,8 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         if (rc) return rc;
         rc = ensure_smem(k_spmspv_fused, plan.smem, g_granted_fused);
         if (rc) return rc;
+        rc = fit_clusters(&plan);
+        if (rc) return rc;
         FusedParams fp;
         fp.meta = reinterpret_cast<const uint32_t *>(m->d_image);
         fp.stream = stream_base;
@@ -498,13 +568,23 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
         fp.partials = reinterpret_cast<float *>(m->d_ws + m->ws.partial_off);
         fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.C = m->C;
-        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.W = plan.W;
+        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.cl = plan.cl;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
+        {
+            // offset window: as many columns as 32 KB (or the accumulator area, or the table) hold
+            const size_t acc_bytes = (size_t)plan.G * plan.Sc * (m->R + kTileSlack) * 128;
+            const size_t words = std::min<size_t>(std::min<size_t>(acc_bytes, 32768) / 4, (size_t)m->K * m->S + 4);
+            fp.win_cols = (int)std::min<int64_t>(m->K, words >= 8 ? (int64_t)((words - 8) / m->S) : 0);
+        }
+        if (m->exp_flags & 1) fp.win_cols = 0;
+        fp.fixed_deal = (m->exp_flags & 2) ? 1 : 0;
         fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
+        fp.spin_limit = m->spin_limit ? m->spin_limit : kSpinLimit;
         auto inverse = [](uint64_t units) { return units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / units); };
-        fp.units_inv = inverse((uint64_t)(plan.grid / plan.P) * plan.G);
-        fp.units_inv_long = inverse((uint64_t)(plan.grid / plan.P + 1) * plan.G);
+        const int nclusters = plan.grid / plan.cl;
+        fp.slices_inv = inverse((uint64_t)plan.cl * std::max(1, nclusters / plan.P));
+        fp.slices_inv_long = inverse((uint64_t)plan.cl * (nclusters / plan.P + 1));
         // the tickets count blocks of one launch shape: start them over when the shape changes
         if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
             CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
@@ -518,11 +598,22 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         cfg.blockDim = dim3((unsigned)plan.threads);
         cfg.dynamicSmemBytes = plan.smem;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchAttribute attr[2];
+        int na = 0;
+        if (!m->no_overlap) {
+            attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[na].val.programmaticStreamSerializationAllowed = 1;
+            ++na;
+        }
+        if (plan.cl > 1) {
+            attr[na].id = cudaLaunchAttributeClusterDimension;
+            attr[na].val.clusterDim.x = (unsigned)plan.cl;
+            attr[na].val.clusterDim.y = 1;
+            attr[na].val.clusterDim.z = 1;
+            ++na;
+        }
         cfg.attrs = attr;
-        cfg.numAttrs = m->no_overlap ? 0 : 1;
+        cfg.numAttrs = na;
         CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused, fp));
         return CELTY_OK;
     }

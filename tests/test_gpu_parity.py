@@ -215,8 +215,9 @@ def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows, spb
     x = synth.integer_activations(M + K, K)
     tau = synth.threshold_for_density(x, d_a)
     m = _matrix(W, mask, layout, tile_rows, spb)
-    for grid, groups, depth, team in ((0, 0, 0, 0), (1, 0, 0, 1), (3, 1, 1, 4), (37, 3, 2, 2), (148, 2, 4, 1)):
-        m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth, team=team)
+    for grid, groups, depth, cluster in ((0, 0, 0, 0), (1, 0, 0, 1), (3, 1, 1, 4), (36, 3, 2, 2), (148, 2, 4, 1),
+                                        (148, 0, 0, 4), (7, 16, 0, 2)):
+        m.set_launch(grid=grid, variant=m.variant, groups=groups, depth=depth, cluster=cluster)
         y = _run(m, x, tau)
         _check_y(y, W, mask, x, tau, exact=True)
 
@@ -241,10 +242,10 @@ def test_random_shapes_and_options(case):
     except celty.CeltyError as e:                       # more than 32 slabs: a refused option, not a failure
         assert e.status == -1 and tile_rows > 0 and (M + 31) // 32 > 32 * tile_rows
         return
-    grid, groups, depth, team = (int(rng.choice([0, 0, 1, 5, 40, 148])), int(rng.choice([0, 0, 1, 3])),
-                                 int(rng.choice([0, 0, 1, 3])), int(rng.choice([0, 1, 2, 4])))
+    grid, groups, depth, cluster = (int(rng.choice([0, 0, 1, 5, 40, 148])), int(rng.choice([0, 0, 1, 3])),
+                                    int(rng.choice([0, 0, 1, 3])), int(rng.choice([0, 1, 2, 4])))
     variant = int(rng.choice([0, 0, 2, 8]))
-    m.set_launch(grid=grid, variant=variant, groups=groups, depth=depth, team=team)
+    m.set_launch(grid=grid, variant=variant, groups=groups, depth=depth, cluster=cluster)
     _check_y(_run(m, x, tau), W, mask, x, tau)
     idx, val = m.last_compaction()
     oi, ov, _ = orc.compact(x, tau)
