@@ -4,14 +4,13 @@
 // One launch does the whole call (Sections 3.1-3.3):
 //   a0  the last warp of every block clears its share of y and takes a ticket (the merge at the end adds into y);
 //   a1  every block thresholds all of x (K <= a few 10k values, served by L2) into one keep bit per
-//       activation and ranks the survivors (popcounts + warp scans).  The survivor list is cut into equal
-//       runs of ranks, one per thread block; the threads that made the keep words write the columns of
-//       the block's run straight into its work list in shared memory, and the streaming warps fetch each
-//       listed column's activation and sub-block offset in one round trip.  The blocks of row part 0
-//       also write the list (index, value, count) for the API;
-//   a2  the block's warp teams take columns from that list one at a time (a shared-memory counter) and
-//       stream their sub-blocks (column j, slab s) from HBM into per-team rings of shared-memory slots
-//       with bulk asynchronous copies (cp.async.bulk + mbarrier complete_tx), D deep;
+//       activation and ranks the survivors (popcounts + warp scans); each warp team then looks up the
+//       columns whose ranks belong to it -- the list is balanced over all teams by count -- and their
+//       sub-block offsets, which it finds in a window of the offset table that the block copied into
+//       shared memory when it started.  The team that owns a rank on slab 0 also writes it to the global
+//       list (index, value, count) for the API;
+//   a2  each team streams the sub-blocks (column j, slab s) of its columns from HBM into its ring of
+//       shared-memory slots with bulk asynchronous copies (cp.async.bulk + mbarrier complete_tx), D deep;
 //   a3  each lane decodes its own tile's runs on packed bytes and keeps a running row;
 //   a4  value * x_j is accumulated (FP16 x FP16 + FP32 fused multiply-add) into the lane's private bank of
 //       the team's accumulator;
@@ -21,8 +20,8 @@
 //       that every block has cleared its share of y.  Option: per-block partial vectors, a bounded
 //       grid-wide ticket barrier and a sum in a fixed order (bit-reproducible, no clearing of y).
 //
-// Rows are split over P parts of Sc slabs each, columns over the blocks of a part; a team = one warp with
-// its own accumulator slab, G teams per slab.  Every block must be resident at once (grid <= SM count)
+// Rows are split over P parts of Sc slabs each, columns over the blocks of a part and, inside a block, over
+// G teams per slab; a team = one warp with its own accumulator slab.  Every block must be resident at once (grid <= SM count)
 // because of the tickets.  All waits are bounded: when one runs out the kernel sets kStatusTimeout in the
 // status word and carries on to a clean exit.
 
@@ -43,12 +42,12 @@ struct FusedParams {
     int cl;                    // thread blocks per cluster (1, 2 or 4); blocks of a cluster share a row part
     long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
-    int cap;                   // columns the block's work list holds at a time
+    int cap;                   // columns a team looks up per batch
     int win_cols;              // columns of the offset table a block copies into shared memory at its start
-    int fixed_deal;            // 1: a team takes every G-th column of the list instead of the next free one
-    // column slices of a row part = blocks that share its survivor list: slices_inv = floor(2^32 / slices)
-    // for parts with gridDim / cl / P clusters, slices_inv_long for those with one cluster more
-    uint32_t slices_inv, slices_inv_long;
+    // teams that share the survivor list of a row part: units = (column slices of the part) * G;
+    // units_inv = floor(2^32 / units) for parts with gridDim / cl / P clusters, units_inv_long for those with
+    // one cluster more
+    uint32_t units_inv, units_inv_long;
     int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row segments into y
     uint32_t spin_limit;       // polls a bounded wait makes before it gives up
 };
@@ -68,15 +67,8 @@ __constant__ long long *g_celty_trace = nullptr;
     do {                                                                     \
         if (threadIdx.x == 0 && g_celty_trace) g_celty_trace[blockIdx.x * 16 + (k)] = clock64(); \
     } while (0)
-#define CELTY_CLOCK() clock64()
-#define CELTY_STORE(k, v)                                                     \
-    do {                                                                      \
-        if (threadIdx.x == 0 && g_celty_trace) g_celty_trace[blockIdx.x * 16 + (k)] = (long long)(v); \
-    } while (0)
 #else
 #define CELTY_MARK(k)
-#define CELTY_CLOCK() 0ll
-#define CELTY_STORE(k, v)
 #endif
 #ifdef CELTY_GUARD
 #define CELTY_CHECK(ok, code, value)                                                                   \
@@ -120,50 +112,16 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 
 // Bulk asynchronous copy global -> shared (1-D, no tensor map; every sub-block has exactly one consumer,
 // the team that asked for it); src, dst and bytes are multiples of 16.  Every lane of a converged warp calls
-// this; one elected lane notes the column's activation beside the slot, announces the bytes on the mbarrier
-// and issues the copy, all under a predicate (no branch); completion is signalled on the mbarrier as
-// transferred bytes.
-__device__ __forceinline__ void bulk_load_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
-                                                  uint32_t note_addr, uint32_t note)
+// this; one elected lane announces the bytes on the mbarrier and issues the copy, both under a predicate
+// (no branch); completion is signalled on the mbarrier as transferred bytes.
+__device__ __forceinline__ void bulk_load_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "elect.sync _|P, 0xffffffff;\n\t"
-        "@P st.shared.u32 [%4], %5;\n\t"
         "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t"
         "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%2], [%3], %1, [%0];\n\t}" ::"r"(bar),
-        "r"(bytes), "r"(dst), "l"(src), "r"(note_addr), "r"(note)
-        : "memory");
-}
-
-// The same with one more step for the elected lane: it takes the next position of the block's work list
-// (shared-memory counter at `next_addr`) for the refill after this one.  `taken` is meaningful in lane `leader`
-// only; the caller broadcasts it when it needs it, a whole sub-block later, so nobody waits for the atomic.
-__device__ __forceinline__ void bulk_load_elected_take(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
-                                                       uint32_t note_addr, uint32_t note, uint32_t next_addr,
-                                                       uint32_t &taken, uint32_t &leader)
-{
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "elect.sync %1|P, 0xffffffff;\n\t"
-        "@P st.shared.u32 [%6], %7;\n\t"
-        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%2], %3;\n\t"
-        "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%4], [%5], %3, [%2];\n\t"
-        "@P atom.shared.add.u32 %0, [%8], 1;\n\t}"
-        : "+r"(taken), "=r"(leader)
-        : "r"(bar), "r"(bytes), "r"(dst), "l"(src), "r"(note_addr), "r"(note), "r"(next_addr)
-        : "memory");
-}
-
-// The take alone (after a team's first copies).
-__device__ __forceinline__ void take_elected(uint32_t next_addr, uint32_t &taken, uint32_t &leader)
-{
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "elect.sync %1|P, 0xffffffff;\n\t"
-        "@P atom.shared.add.u32 %0, [%2], 1;\n\t}"
-        : "+r"(taken), "=r"(leader)
-        : "r"(next_addr)
+        "r"(bytes), "r"(dst), "l"(src)
         : "memory");
 }
 
@@ -308,27 +266,24 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, note, items, imeta, next, zero, keep, wrel, blk, blkx, total;
+    size_t acc, ring, bars, items, imeta, zero, keep, wrel, blk, blkw, total;
 };
 
-__host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int Sc, int D, int slot_bytes, int cap)
+__host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
 {
     FusedSmem l;
     size_t off = 0;
-    const size_t words = ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16, blocks = ((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16;
     l.acc = off;       off += (size_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
     l.ring = off;      off += (size_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
     l.bars = off;      off += (size_t)teams * D * 8 + 8;                   // one "full" mbarrier per slot, one for the offset window
-    l.note = off;      off += (size_t)teams * D * 4;                       // the activation of the column in each slot
     off = (off + 15) / 16 * 16;
-    l.items = off;     off += (size_t)cap * 8;                             // work list: {column, x bits}
-    l.imeta = off;     off += (size_t)Sc * cap * 8;                        // per slab of the block: {offset/16, bytes}
-    l.next = off;      off += 64;                                          // per slab: next list position to hand out
+    l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
+    l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
     l.zero = off;      off += 16;                                          // the all-zero group that idle lanes fetch
-    l.keep = off;      off += words;                                       // one keep bit per activation
-    l.wrel = off;      off += words;                                       // survivors before each keep word, in its block of 32
-    l.blk = off;       off += blocks;                                      // survivors in each block of 32 keep words
-    l.blkx = off;      off += blocks;                                      // survivors before each block
+    l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
+    l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 32
+    l.blk = off;       off += ((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16; // survivors in each block of 32 keep words
+    l.blkw = off;      off += 16 * (((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
     l.total = off;
     return l;
 }
@@ -341,21 +296,21 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     // derived from it) is the same for all lanes, and keeps the streaming loop free of divergence handling
     const int warp = __shfl_sync(kFull, tid >> 5, 0);
     const int slab_words = (p.R + kTileSlack) * 32;
-    // Warps [0, teams) stream columns, one warp per team; the others only help with the phases that are plain
-    // data-parallel work (thresholding, the work list, clearing, the merge).
+    // Warps [0, teams) stream columns, one warp per team; the others only help with the phases that
+    // are plain data-parallel work (thresholding, clearing, storing and summing partial vectors).
     const int teams = p.G * p.Sc;
     const bool streams = warp < teams;
     const int team = streams ? warp : 0;
-    const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.Sc, p.D, p.slot_bytes, p.cap);
+    const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.D, p.slot_bytes, p.cap);
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
-    int2 *items = reinterpret_cast<int2 *>(smem + lay.items);                             // [cap] {column, x bits}
-    int *next = reinterpret_cast<int *>(smem + lay.next);                                 // [Sc]
+    int2 *items = reinterpret_cast<int2 *>(smem + lay.items) + (size_t)team * p.cap;      // [cap] {column, x bits}
+    uint2 *imeta = reinterpret_cast<uint2 *>(smem + lay.imeta) + (size_t)team * p.cap;    // [cap] {offset/16, bytes}
     int *zero_group = reinterpret_cast<int *>(smem + lay.zero);                           // 16 bytes of zeros
     int *wrel = reinterpret_cast<int *>(smem + lay.wrel);                                 // [nwords]
-    int *blk = reinterpret_cast<int *>(smem + lay.blk);                                   // [nwords / 32] counts
-    int *blkx = reinterpret_cast<int *>(smem + lay.blkx);                                 // [nwords / 32] exclusive prefix
+    const int *blk = reinterpret_cast<const int *>(smem + lay.blk);                       // [nwords / 32] counts
+    int *myblk = reinterpret_cast<int *>(smem + lay.blkw) + (size_t)warp * ((lay.blkw - lay.blk) / 4);   // this warp's prefix
     uint32_t *kbw = reinterpret_cast<uint32_t *>(smem + lay.keep);
 
     // Row part and column slice of this block.  The blocks of a cluster work on the same row part (they add
@@ -422,7 +377,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     // and the warp scans the survivor counts of its block of 32 words:
     //   kbw[w]  keep bits of activations 32w .. 32w+31,
     //   wrel[w] survivors in the words before w of the same block of 32 words,
-    //   blk[e]  survivors in block e.
+    //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
     const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 31) >> 5;
     {
@@ -469,7 +424,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 kbw[w] = word;
                 wrel[w] = incl - cnt;
             }
-            if (lane == 31 && (w >> 5) < nblk) blk[w >> 5] = incl;
+            if (lane == 31 && (w >> 5) < nblk) const_cast<int *>(blk)[w >> 5] = incl;
         }
     }
     CELTY_MARK(10);
@@ -481,11 +436,11 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         failed = true;
         win_n = 0;
     }
-    // ---- ranks: every warp turns the block counts into survivors before each block for itself, 32 blocks at a
-    // time.  All warps store the same numbers into the one table and each reads only what it has stored itself,
-    // which saves a block-wide barrier behind a single scanning warp.
+    // ---- ranks: every streaming warp turns the block counts into survivors before each block for itself, 32
+    // blocks at a time (a copy per warp costs a few hundred bytes and saves a block-wide barrier behind a single
+    // warp); the list is then cut into equal shares for the groups that work on different columns.
     int n_surv = 0;
-    {
+    if (streams) {
         int carry = 0;
         for (int e0 = 0; e0 < nblk; e0 += 32) {
             const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
@@ -495,177 +450,165 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 const int up = __shfl_up_sync(kFull, incl, d);
                 if (lane >= d) incl += up;
             }
-            if (e < nblk) blkx[e] = carry + incl - cnt;
+            if (e < nblk) myblk[e] = carry + incl - cnt;
             carry += __shfl_sync(kFull, incl, 31);
         }
         __syncwarp();
         n_surv = carry;
-        if (blockIdx.x == 0 && tid == 0) *p.count = carry;
-    }
-    // The survivor list is cut into nK runs of ranks, one per block of this row part: n / nK each, the first
-    // n mod nK blocks one more.  n / nK without a division: slices_inv = floor(2^32 / nK) gives a quotient that is
-    // at most one too small.
-    int rb0, rb1;
-    {
-        const uint32_t inv = long_part ? p.slices_inv_long : p.slices_inv;
-        uint32_t share = __umulhi((uint32_t)n_surv, inv), extra = (uint32_t)n_surv - share * (uint32_t)nK;
-        if (extra >= (uint32_t)nK) { ++share; extra -= (uint32_t)nK; }
-        rb0 = kslice * (int)share + min(kslice, (int)extra);
-        rb1 = rb0 + (int)share + (kslice < (int)extra ? 1 : 0);
+        if (blockIdx.x == 0 && warp == 0 && lane == 0) *p.count = carry;
     }
     CELTY_MARK(2);
 
-    // ---- a2-a4, in passes of at most `cap` columns (one pass on every configured shape)
-    const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
-    const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
-    const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
-    const uint32_t bar0 = smem_u32(&bars[team * p.D]);
-    const uint32_t note0 = smem_u32(smem + lay.note) + 4u * (uint32_t)(team * p.D);
-    uint2 *imeta_all = reinterpret_cast<uint2 *>(smem + lay.imeta);           // [Sc][cap] {offset/16, bytes}
-    const uint2 *imeta = imeta_all + (size_t)sl * p.cap;                      // this team's slab
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    const uint32_t zeros = smem_u32(zero_group);
-    bool zeroed = false;
-    uint32_t slot = 0, parity = 0, islot = 0;                      // ring position: consumed % D, its phase, issued % D
-    StepBuf b0, b1;                                                // pipeline registers, live across columns
+    if (streams) {
+        // team u of nK * G owns n / units ranks, the first n mod units teams one more.  n / units without a
+        // division: units_inv = floor(2^32 / units) gives a quotient that is at most one too small
+        const uint32_t units = (uint32_t)(nK * p.G), units_inv = long_part ? p.units_inv_long : p.units_inv;
+        uint32_t share = __umulhi((uint32_t)n_surv, units_inv), extra = (uint32_t)n_surv - share * units;
+        if (extra >= units) { ++share; extra -= units; }
+        const int u = kslice * p.G + g;
+        const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
+        const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
+        const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
+        const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
+        const uint32_t bar0 = smem_u32(&bars[team * p.D]);
+        bool zeroed = false;
+        const uint32_t lt_mask = (1u << lane) - 1u;
+        const uint32_t items0 = smem_u32(items);
+        uint32_t issued = 0, consumed = 0;                            // copies asked for / used up by this team
+        uint32_t slot = 0, parity = 0, islot = 0;                     // consumed % D, (consumed / D) & 1, issued % D
+        StepBuf b0, b1;                                               // pipeline registers, live across items
+        const uint32_t zeros = smem_u32(zero_group);
 
-    for (int w0 = rb0; w0 < rb1; w0 += p.cap) {
-        const int w1 = min(rb1, w0 + p.cap), n = w1 - w0;
-        if (w0 > rb0) __syncthreads();                             // everybody is done with the previous pass's list
-        // every team starts with D columns of its own (positions g, g + G, ...); the rest are handed out one at a time
-        if (tid < p.Sc) next[tid] = p.D * p.G;
-        // ---- the threads write the columns of ranks [w0, w1) into the list: a keep word knows the rank of its
-        // first survivor (survivors before its block + before it within the block)
-        for (int w = tid; w < nwords; w += nthreads) {
-            const int base = blkx[w >> 5] + wrel[w];
-            uint32_t word = kbw[w];
-            if (base >= w1 || base + __popc(word) <= w0) continue;
-            for (int r = base; word; ++r) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                if (r >= w0 && r < w1) items[r - w0].x = 32 * w + b;
-            }
-        }
-        __syncthreads();
-        CELTY_MARK(11);
-        if (!streams) continue;
-        // ---- the streaming warps fetch, for every listed column, its activation and the offsets of its sub-blocks
-        // (one round trip to L2 for the lot); row part 0 also writes the list for the API
-        for (int i = warp * 32 + lane; i < n; i += teams * 32) {
-            int j = items[i].x;
-            if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
-            const uint16_t xb = __ldg(p.x + j);                      // x went through L1 in the thresholding pass
-            for (int f = 0; f < p.Sc; ++f) {
-                const int sf = part * p.Sc + f;
-                if (sf >= p.S) break;
-                const int wq = j * p.S + sf - win_w0;                  // the window is there in the first pass only
-                uint32_t o0, o1;
-                if (w0 == rb0 && wq >= 0 && wq + 1 < win_n) {
-                    o0 = win[wq];
-                    o1 = win[wq + 1];
-                } else {
-                    o0 = p.meta[(size_t)j * p.S + sf];
-                    o1 = p.meta[(size_t)j * p.S + sf + 1];
+        for (int rb = r_begin;; rb += p.cap) {                        // at least one trip: the teams meet at a barrier in it
+            const int cnt = failed ? 0 : max(0, min(p.cap, r_end - rb));
+            // ---- column of rank r: the block of keep words that holds it, then the word, then the bit
+            for (int i = lane; i < cnt; i += 32) {
+                const int r = rb + i;
+                // the block of 32 keep words that holds rank r (the last one with blk[e] <= r), the word in it
+                // (the last one with wrel[w] <= what is left) ...
+                int e = 0;
+                for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
+                    if (e + step < nblk && myblk[e + step] <= r) e += step;
+                int k = r - myblk[e], w = 32 * e;
+#pragma unroll
+                for (int step = 16; step; step >>= 1)
+                    if (w + step < nwords && wrel[w + step] <= k) w += step;
+                k -= wrel[w];
+                // ... and the bit in it: halve the word, keep the half that holds the wanted set bit
+                const uint32_t word = kbw[w];
+                int pos = 0;
+#pragma unroll
+                for (int sh = 16; sh; sh >>= 1) {
+                    const int c = __popc((word >> pos) & ((1u << sh) - 1u));
+                    if (k >= c) { k -= c; pos += sh; }
                 }
-                uint2 im = make_uint2(o0, (o1 - o0) * 16u);
-                if (!CELTY_CHECK(o1 > o0 && (o1 - o0) * 16u <= (uint32_t)p.slot_bytes &&
-                                     (long long)o1 * 16 <= p.stream_bytes, 4, o1 - o0))
-                    im = make_uint2(0u, (uint32_t)kSubHeader);
-                imeta_all[(size_t)f * p.cap + i] = im;
+                if (!CELTY_CHECK(((word >> pos) & 1u) != 0 && k == 0, 8, w)) pos = 0;
+                int j = 32 * w + pos;
+                if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
+                const uint16_t xb = __ldg(p.x + j);                  // x went through L1 in the thresholding pass
+                items[i] = make_int2(j, (int)xb);
+                if (part == 0 && sl == 0 && CELTY_CHECK(r >= 0 && r < p.K, 10, r)) {
+                    p.idx[r] = j;
+                    p.val[r] = xb;
+                }
+                if (s < p.S) {
+                    // the two offsets of sub-block (j, s): from the block's window of the table if they are in it
+                    const int wq = j * p.S + s - win_w0;
+                    uint32_t o0, o1;
+                    if (wq >= 0 && wq + 1 < win_n) {
+                        o0 = win[wq];
+                        o1 = win[wq + 1];
+                    } else {
+                        o0 = p.meta[(size_t)j * p.S + s];
+                        o1 = p.meta[(size_t)j * p.S + s + 1];
+                    }
+                    imeta[i] = make_uint2(o0, (o1 - o0) * 16u);
+                    if (!CELTY_CHECK(o1 > o0 && (o1 - o0) * 16u <= (uint32_t)p.slot_bytes &&
+                                         (long long)o1 * 16 <= p.stream_bytes, 4, o1 - o0))
+                        imeta[i] = make_uint2(0u, (uint32_t)kSubHeader);
+                }
             }
-            items[i].y = (int)xb;
-            if (part == 0) {
-                p.idx[w0 + i] = j;
-                p.val[w0 + i] = xb;
+            // The accumulators take the place of the window: every team has to be through with its look-ups
+            // before any team clears its slab.  (Teams with more than `cap` columns come back here for their
+            // later batches, and find the offsets in global memory then.)
+            if (rb == r_begin) asm volatile("bar.sync 1, %0;" ::"r"(teams * 32) : "memory");
+            else __syncwarp();
+            win_n = 0;
+            if (rb + p.cap >= r_end && (cnt == 0 || s >= p.S)) break;
+            if (cnt == 0 || s >= p.S) continue;
+            // ---- a2: keep D copies in flight.  The team issues the first D of a batch and refills a slot whenever
+            // it has finished with it.  Every lane calls issue(), converged, and keeps the ring position; one
+            // elected lane (elect.sync) runs the two instructions under a predicate -- 3 % faster at 28672 x 8192
+            // than a branch on lane 0, around which the warp diverges and reconverges for every sub-block.
+            auto issue_im = [&](const uint2 im) {
+                bulk_load_elected(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y,
+                                  bar0 + 8u * islot);
+                ++issued;
+                if (++islot == (uint32_t)p.D) islot = 0;
+            };
+            for (int i = 0; i < min(cnt, p.D); ++i) issue_im(imeta[i]);
+            CELTY_MARK(3);
+            if (!zeroed) {                                          // clear the slab while the first copies fly
+                float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
+                for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                zeroed = true;
+                __syncwarp();
             }
+            for (int i = 0; i < cnt; ++i) {
+                uint32_t xbits;                                       // the column's activation: asked for before the wait
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(items0 + 8u * (uint32_t)i + 4u));
+                if (!mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
+                failed = __any_sync(kFull, failed);
+                if (failed) break;                                    // the copies still in flight are awaited below
+                if (i == 0) CELTY_MARK(4);
+                const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
+                // what the refill at the end of this sub-block will need, read now so that it does not wait then
+                const bool refill = i + p.D < cnt;
+                const uint2 next_im = refill ? imeta[i + p.D] : make_uint2(0u, 0u);
+                const uint16_t xj = (uint16_t)xbits;
+                // ---- a3 + a4.  Header: groups per lane, vectors and steps (see kSubHeader).
+                uint32_t gl, hw;
+                asm volatile("ld.shared.u8 %0, [%1];" : "=r"(gl) : "r"(sub + lane));
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw) : "r"(sub + 32));       // vectors | steps << 16
+                const uint32_t steps = hw >> 16, Gs = hw & 0xFFFFu;
+                const uint32_t vbase = sub + kSubHeader, rbase = vbase + 16 * Gs;
+                const uint32_t slot_end = sub + (uint32_t)p.slot_bytes;
+                uint32_t cum = 0, cell = cell0;
+                const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
+                step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                step_decode(b0, cell, spare, slab0, slab_end);                                    // step 0
+                step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                uint32_t q = 1;
+#pragma unroll 2
+                for (; q + 1 < steps; q += 2) {                                            // two real steps per pass
+                    step_decode(b1, cell, spare, slab0, slab_end);                                // step q
+                    step_finish(b0, xj);                                                   // step q-1
+                    step_fetch(b1, gl, q + 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                    step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
+                    step_finish(b1, xj);                                                   // step q
+                    step_fetch(b0, gl, q + 3, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                }
+                if (q < steps) {                                                           // one real step left
+                    step_decode(b1, cell, spare, slab0, slab_end);
+                    step_finish(b0, xj);
+                    step_finish(b1, xj);
+                } else {                                                                   // only the last one to finish
+                    step_finish(b0, xj);
+                }
+                // The slot's contents were consumed by loads whose values have been used, and the barrier orders
+                // every lane's reads before this point: the copy may overwrite it.
+                __syncwarp();
+                if (refill) issue_im(next_im);
+                ++consumed;
+                if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
+            }
+            __syncwarp();                                         // items / imeta are rewritten by the next batch
+            if (failed || rb + p.cap >= r_end) break;
         }
-        asm volatile("bar.sync 1, %0;" ::"r"(teams * 32) : "memory");      // the streaming warps only
-        if (s >= p.S) continue;
-        // ---- a2: keep D copies in flight.  Every lane calls issue(), converged, and keeps the ring position; one
-        // elected lane (elect.sync) runs the instructions under a predicate -- measured 3 % faster at 28672 x 8192
-        // than a branch on lane 0, around which the warp diverges and reconverges for every sub-block.
-        uint32_t issued = 0, consumed = 0;
-        auto issue = [&](const uint2 im, uint32_t xbits) {
-            bulk_load_elected(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y,
-                              bar0 + 8u * islot, note0 + 4u * islot, xbits);
-            ++issued;
-            if (++islot == (uint32_t)p.D) islot = 0;
-        };
-        const uint32_t next_addr = smem_u32(&next[sl]);
-        uint32_t taken = (uint32_t)n, leader = 0;                  // the list position for the refill after next
-        if (!failed)
-            for (int d = 0, i = g; d < p.D && i < n; ++d, i += p.G) issue(imeta[i], (uint32_t)items[i].y);
-        if (issued == (uint32_t)p.D) {
-            if (p.fixed_deal) taken = (uint32_t)(g + p.D * p.G);
-            else take_elected(next_addr, taken, leader);
-        }
-        CELTY_MARK(3);
-        if (!zeroed) {                                              // clear the slab while the first copies fly
+        if (!zeroed && s < p.S) {                                     // a team without columns still owns a slab
             float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
             for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            zeroed = true;
-        }
-        __syncwarp();
-        while (consumed < issued) {
-            uint32_t xbits;                                           // the column's activation: asked for before the wait
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(note0 + 4u * slot));
-            if (!mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
-            failed = __any_sync(kFull, failed);
-            if (failed) break;                                        // the copies still in flight are awaited below
-            if (consumed == 0) CELTY_MARK(4);
-            const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
-            // what the refill at the end of this sub-block will need, read now so that it does not wait then
-            const int pend = (int)__shfl_sync(kFull, taken, leader);
-            const bool refill = pend < n;
-            const uint2 next_im = refill ? imeta[pend] : make_uint2(0u, 0u);
-            const uint32_t next_x = refill ? (uint32_t)items[pend].y : 0u;
-            const uint16_t xj = (uint16_t)xbits;
-            // ---- a3 + a4.  Header: groups per lane, vectors and steps (see kSubHeader).
-            uint32_t gl, hw;
-            asm volatile("ld.shared.u8 %0, [%1];" : "=r"(gl) : "r"(sub + lane));
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw) : "r"(sub + 32));       // vectors | steps << 16
-            const uint32_t steps = hw >> 16, Gs = hw & 0xFFFFu;
-            const uint32_t vbase = sub + kSubHeader, rbase = vbase + 16 * Gs;
-            const uint32_t slot_end = sub + (uint32_t)p.slot_bytes;
-            uint32_t cum = 0, cell = cell0;
-            const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
-            step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-            step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-            step_decode(b0, cell, spare, slab0, slab_end);                                    // step 0
-            step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-            uint32_t q = 1;
-#pragma unroll 2
-            for (; q + 1 < steps; q += 2) {                                            // two real steps per pass
-                step_decode(b1, cell, spare, slab0, slab_end);                                // step q
-                step_finish(b0, xj);                                                   // step q-1
-                step_fetch(b1, gl, q + 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
-                step_finish(b1, xj);                                                   // step q
-                step_fetch(b0, gl, q + 3, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-            }
-            if (q < steps) {                                                           // one real step left
-                step_decode(b1, cell, spare, slab0, slab_end);
-                step_finish(b0, xj);
-                step_finish(b1, xj);
-            } else {                                                                   // only the last one to finish
-                step_finish(b0, xj);
-            }
-            // The slot's contents were consumed by loads whose values have been used, and the barrier orders
-            // every lane's reads before this point: the copy may overwrite it.
-            __syncwarp();
-            if (refill) {                                           // copy + the take for the refill after this one
-                if (p.fixed_deal) {
-                    issue(next_im, next_x);
-                    taken += (uint32_t)p.G;
-                } else {
-                    bulk_load_elected_take(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)next_im.x * 16,
-                                           next_im.y, bar0 + 8u * islot, note0 + 4u * islot, next_x, next_addr, taken, leader);
-                    ++issued;
-                    if (++islot == (uint32_t)p.D) islot = 0;
-                }
-            }
-            ++consumed;
-            if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
         }
         if (failed) {
             // give the copies that are still in flight a last (bounded) chance to land before the block goes on
@@ -675,11 +618,6 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             }
             if (lane == 0) atomicOr(p.status, kStatusTimeout);
         }
-    }
-    if (failed && lane == 0) atomicOr(p.status, kStatusTimeout);
-    if (streams && !zeroed && s < p.S) {                              // a team without columns still owns a slab
-        float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
-        for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     __syncthreads();
     CELTY_MARK(5);
@@ -768,85 +706,86 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         return;
     }
 
-    // ---- a5, ordered: stage 1 adds the G accumulators and stores the block's partial (accumulator layout, no
-    // slack rows).  (Clusters are not used with this merge: cl == 1, so block b of part `part` is b * P + part.)
-    const int tile_words = p.R * 32, part_words = p.Sc * tile_words;
     {
-        float4 *mine4 = reinterpret_cast<float4 *>(p.partials + (size_t)blockIdx.x * part_words);
-        const float4 *acc4 = reinterpret_cast<const float4 *>(acc);
-        const int tile4 = tile_words >> 2, slab4 = slab_words >> 2, group4 = p.Sc * slab4;
-        for (int fsl = 0; fsl < p.Sc; ++fsl)
-            for (int q4 = tid; q4 < tile4; q4 += nthreads) {
-                const float4 *src = acc4 + fsl * slab4 + q4;
-                float4 v = src[0];
-                for (int gg = 1; gg < p.G; ++gg) {
-                    const float4 t = src[gg * group4];
-                    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+        // ---- a5, ordered (clusters are not used with this merge).  Stage 1: add the G accumulators, store the block's partial (accumulator layout, no slack rows)
+        const int tile_words = p.R * 32, part_words = p.Sc * tile_words;
+        {
+            float4 *mine4 = reinterpret_cast<float4 *>(p.partials + (size_t)blockIdx.x * part_words);
+            const float4 *acc4 = reinterpret_cast<const float4 *>(acc);
+            const int tile4 = tile_words >> 2, slab4 = slab_words >> 2, group4 = p.Sc * slab4;
+            for (int fsl = 0; fsl < p.Sc; ++fsl)
+                for (int q4 = tid; q4 < tile4; q4 += nthreads) {
+                    const float4 *src = acc4 + fsl * slab4 + q4;
+                    float4 v = src[0];
+                    for (int gg = 1; gg < p.G; ++gg) {
+                        const float4 t = src[gg * group4];
+                        v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+                    }
+                    __stcg(mine4 + fsl * tile4 + q4, v);
                 }
-                __stcg(mine4 + fsl * tile4 + q4, v);
-            }
-    }
-    __syncthreads();
-    CELTY_MARK(6);
-    if (tid == 0) {
-        __threadfence();                                          // the block's stores, ordered by the barrier above
-        atomicAdd(&p.tickets[0], 1u);
-        bool ok = false;
-        for (uint32_t it = 0; it < p.spin_limit; ++it) {
-            if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
-            __nanosleep(32);
         }
-        if (!ok) atomicOr(p.status, kStatusTimeout);
-    }
-    __syncthreads();
-    CELTY_MARK(7);
+        __syncthreads();
+        CELTY_MARK(6);
+        if (tid == 0) {
+            __threadfence();                                          // the block's stores, ordered by the barrier above
+            atomicAdd(&p.tickets[0], 1u);
+            bool ok = false;
+            for (uint32_t it = 0; it < p.spin_limit; ++it) {
+                if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
+                __nanosleep(32);
+            }
+            if (!ok) atomicOr(p.status, kStatusTimeout);
+        }
+        __syncthreads();
+        CELTY_MARK(7);
 
-    // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
-    // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
-    // every lane has up to 16 loads in flight, then the ranges are added in a fixed order.
-    {
-        float *red = reinterpret_cast<float *>(smem + lay.acc);   // the accumulators are no longer needed
-        const int wpc = (((part_words + nK - 1) / nK) + 31) & ~31;
-        const int wb = kslice * wpc, we = min(part_words, wb + wpc);
-        const int nchunks = max(0, (we - wb + 31) >> 5);
-        const size_t stride = (size_t)p.P * part_words;
-        for (int c0 = 0; c0 < nchunks; c0 += nwarps) {
-            const int pass_chunks = min(nwarps, nchunks - c0);
-            const int nsplit = nwarps / pass_chunks;              // warps per chunk in this pass
-            const int my_chunk = warp % pass_chunks, my_split = warp / pass_chunks;
-            const int word = wb + 32 * (c0 + my_chunk) + lane;
-            if (my_split < nsplit) {
-                float sum = 0.f;
-                if (word < we) {
-                    const int per = (nK + nsplit - 1) / nsplit;
-                    const int b_lo = my_split * per, b_hi = min(nK, b_lo + per);
-                    const float *src = p.partials + (size_t)part * part_words + word;
-                    for (int bb = b_lo; bb < b_hi; bb += 16) {
-                        float t[16];
-#pragma unroll
-                        for (int k = 0; k < 16; ++k)
-                            t[k] = (bb + k < b_hi && CELTY_CHECK((size_t)(bb + k) * stride + (size_t)part * part_words + word <
-                                                                     (size_t)gridDim.x * part_words, 13, bb + k))
-                                       ? __ldcg(src + (size_t)(bb + k) * stride) : 0.f;
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) sum += t[k];
+        // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
+        // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
+        // every lane has up to 16 loads in flight, then the ranges are added in a fixed order.
+        {
+            float *red = reinterpret_cast<float *>(smem + lay.acc);   // the accumulators are no longer needed
+            const int wpc = (((part_words + nK - 1) / nK) + 31) & ~31;
+            const int wb = kslice * wpc, we = min(part_words, wb + wpc);
+            const int nchunks = max(0, (we - wb + 31) >> 5);
+            const size_t stride = (size_t)p.P * part_words;
+            for (int c0 = 0; c0 < nchunks; c0 += nwarps) {
+                const int pass_chunks = min(nwarps, nchunks - c0);
+                const int nsplit = nwarps / pass_chunks;              // warps per chunk in this pass
+                const int my_chunk = warp % pass_chunks, my_split = warp / pass_chunks;
+                const int word = wb + 32 * (c0 + my_chunk) + lane;
+                if (my_split < nsplit) {
+                    float sum = 0.f;
+                    if (word < we) {
+                        const int per = (nK + nsplit - 1) / nsplit;
+                        const int b_lo = my_split * per, b_hi = min(nK, b_lo + per);
+                        const float *src = p.partials + (size_t)part * part_words + word;
+                        for (int b0 = b_lo; b0 < b_hi; b0 += 16) {
+                            float t[16];
+    #pragma unroll
+                            for (int k = 0; k < 16; ++k)
+                                t[k] = (b0 + k < b_hi && CELTY_CHECK((size_t)(b0 + k) * stride + (size_t)part * part_words + word <
+                                                                         (size_t)gridDim.x * part_words, 13, b0 + k))
+                                           ? __ldcg(src + (size_t)(b0 + k) * stride) : 0.f;
+    #pragma unroll
+                            for (int k = 0; k < 16; ++k) sum += t[k];
+                        }
+                    }
+                    red[(my_split * pass_chunks + my_chunk) * 32 + lane] = sum;
+                }
+                __syncthreads();
+                if (warp < pass_chunks) {
+                    const int w2 = wb + 32 * (c0 + warp) + lane;
+                    if (w2 < we) {
+                        float total = 0.f;
+                        for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
+                        const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
+                        const int sfull = part * p.Sc + fsl;
+                        const int64_t row = tile_row(p.S, p.C, sfull, rem & 31, rem >> 5);
+                        if (sfull < p.S && row < p.M) p.y[row] = total;
                     }
                 }
-                red[(my_split * pass_chunks + my_chunk) * 32 + lane] = sum;
+                __syncthreads();
             }
-            __syncthreads();
-            if (warp < pass_chunks) {
-                const int w2 = wb + 32 * (c0 + warp) + lane;
-                if (w2 < we) {
-                    float total = 0.f;
-                    for (int sp = 0; sp < nsplit; ++sp) total += red[(sp * pass_chunks + warp) * 32 + lane];
-                    const int fsl = w2 / tile_words, rem = w2 - fsl * tile_words;
-                    const int sfull = part * p.Sc + fsl;
-                    const int64_t row = tile_row(p.S, p.C, sfull, rem & 31, rem >> 5);
-                    if (sfull < p.S && row < p.M) p.y[row] = total;
-                }
-            }
-            __syncthreads();
         }
     }
     CELTY_MARK(8);
@@ -868,5 +807,5 @@ struct FusedPlan {
 
 inline size_t fused_smem_bytes(int R, int K, int G, int Sc, int D, int slot_bytes, int cap)
 {
-    return fused_smem_layout(R, K, G * Sc, Sc, D, slot_bytes, cap).total;
+    return fused_smem_layout(R, K, G * Sc, D, slot_bytes, cap).total;
 }

@@ -395,7 +395,7 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     pl.Sc = m->Sc;
     if (pl.Sc > 16) return CELTY_EINVAL;      // one warp per team, 16 warps per block
     pl.slot_bytes = (int)round_up((size_t)m->max_unit16 * 16, 128);
-    pl.cap = pl.Sc <= 2 ? 512 : pl.Sc <= 4 ? 256 : 128;
+    pl.cap = 64;
     const size_t budget = (size_t)di.max_smem_optin;
     // Teams first (each needs its own accumulator), then as many ring slots as still fit (at least two, to
     // keep a copy in flight).
@@ -577,14 +577,13 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
             fp.win_cols = (int)std::min<int64_t>(m->K, words >= 8 ? (int64_t)((words - 8) / m->S) : 0);
         }
         if (m->exp_flags & 1) fp.win_cols = 0;
-        fp.fixed_deal = (m->exp_flags & 2) ? 1 : 0;
         fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
         fp.spin_limit = m->spin_limit ? m->spin_limit : kSpinLimit;
         auto inverse = [](uint64_t units) { return units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / units); };
         const int nclusters = plan.grid / plan.cl;
-        fp.slices_inv = inverse((uint64_t)plan.cl * std::max(1, nclusters / plan.P));
-        fp.slices_inv_long = inverse((uint64_t)plan.cl * (nclusters / plan.P + 1));
+        fp.units_inv = inverse((uint64_t)plan.cl * std::max(1, nclusters / plan.P) * plan.G);
+        fp.units_inv_long = inverse((uint64_t)plan.cl * (nclusters / plan.P + 1) * plan.G);
         // the tickets count blocks of one launch shape: start them over when the shape changes
         if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
             CELTY_CUDA(cudaMemsetAsync(m->d_ws + m->ws.status_off + 8, 0, 8, st));
