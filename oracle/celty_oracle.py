@@ -17,6 +17,10 @@ Functions and the passage each follows:
   spmspv_rlc              decode + scatter-accumulate from the encoded arrays (Section 3.3).
   rlc_encode_column_py    the same encoding rule as a literal Python loop over one column,
                           for tiny cases and for replaying the printed example.
+  silu, swiglu, to_half,  the element-wise step between the gate/up projections and the down
+  swiglu_epilogue         projection of a decode layer (Section 6.2 runs the seven products of a LLaMA-2
+                          layer; the MLP's activation is SiLU(gate) * up): plain definition in fp64, one
+                          rounding to FP16 (nearest, ties to even), then the thresholded list.
 
 Every function here is pinned by tests that do not call it to produce their expectation
 (printed example, hand-derived vectors, closed forms, invariants, brute force).
@@ -197,6 +201,41 @@ def spmspv_rlc(enc, x, tau: float):
     _load().orc_spmspv_rlc(_p(enc.vals), _p(enc.rows), _p(enc.block_ptr), enc.K, enc.M,
                            enc.tile_rows, _p(xb), _p(keep), _p(y), _p(a))
     return y, a
+
+
+# ----------------------------------------------------------------------------- MLP element-wise step
+def silu(v) -> np.ndarray:
+    """SiLU(v) = v / (1 + exp(-v)) in fp64 (the activation of the LLaMA MLP whose products Section 6.2 times)."""
+    v = np.asarray(v, dtype=np.float64)
+    with np.errstate(over="ignore"):
+        return v / (1.0 + np.exp(-v))
+
+
+def swiglu(gate, up) -> np.ndarray:
+    """SiLU(gate) * up, element by element, fp64."""
+    return silu(gate) * np.asarray(up, dtype=np.float64)
+
+
+def to_half(v) -> np.ndarray:
+    """fp64 -> FP16 bit patterns, one rounding, to nearest with ties to even; beyond the largest finite
+    value (65520 and up) the result is infinity."""
+    with np.errstate(over="ignore"):
+        return np.asarray(v, dtype=np.float64).astype(np.float16).view(np.uint16)
+
+
+def swiglu_epilogue(y, tau: float):
+    """The step between the stacked [gate; up] product and the down projection.
+
+    y holds the 2I results of the stacked product, gate rows first: h_i = SiLU(y_i) * y_{I+i} in fp64,
+    rounded once to FP16; the list keeps i iff not(|h_i| <= tau) on the rounded value (compared in fp32,
+    like every thresholding decision here).  Returns (h FP16 bit patterns, idx int32 ascending, val, n).
+    """
+    y = np.asarray(y, dtype=np.float64)
+    assert y.ndim == 1 and y.size % 2 == 0
+    half = y.size // 2
+    h = to_half(swiglu(y[:half], y[half:]))
+    idx, val, n = compact(h, tau)
+    return h, idx, val, n
 
 
 def rlc_encode_column_py(column, kept, run_bits: int):

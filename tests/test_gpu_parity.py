@@ -459,6 +459,34 @@ def test_back_to_back_calls_do_not_interfere():
         _check_y(y.cpu().numpy(), W, mask, xs[i], taus[i])
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
+    """Every wait inside the fused kernel has a poll limit.  Here one is made to run out without faulting or
+    hanging anything: the limit is set low and the ticket counter that tells a block when every other block has
+    cleared its share of y is moved ahead by hand, so that five blocks wait for a count that never comes.  The
+    kernel must return by itself, celty_last_status must say CELTY_ETIMEOUT (and repair the counter), and the
+    next call on the handle must be right again."""
+    M, K = 4096, 1024
+    W = synth.weights(91, M, K)
+    mask = synth.mask_bernoulli(91, M, K, 0.5)
+    x = synth.activations(91, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.5)
+    m = celty.Matrix(W, mask, device="cuda")
+    grid = m.launch_plan()["grid"]
+    _check_y(_run(m, x, tau), W, mask, x, tau)                   # a normal call: the counter now stands at `grid`
+    tickets = m._ws[8:16].view(torch.int32)
+    assert int(tickets[0].item()) == grid % (2 * grid)
+    m.set_wait_limit(2000)
+    tickets[0] = grid + 5                                        # five blocks will land in the other half
+    m.spmspv(_dev(x), tau)
+    torch.cuda.synchronize()                                     # the kernel came back by itself
+    assert m.last_status() == -5                                 # CELTY_ETIMEOUT
+    assert celty.load().celty_strerror(-5) == b"a bounded wait inside a kernel ran out"
+    m.set_wait_limit(0)
+    assert m.last_status() == 0                                  # the status word was cleared
+    for _ in range(2):
+        _check_y(_run(m, x, tau), W, mask, x, tau)
+
+
 def test_host_buffer_entry_point():
     M, K = 1024, 1024
     W = synth.weights(1, M, K)
