@@ -193,6 +193,52 @@ int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *idx_dev, uin
 int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, celty_stream_t stream);
 
 /*
+ * Work on y after the merge, inside the same launch (LANE_TILE handles, single-launch kernel, bulk reduce-add
+ * merge).  Section 6.2 times the seven products of a decode layer; between the gate/up and the down projection of
+ * its MLP sits SiLU(gate) * up, and every product's output feeds FP16 consumers.
+ *   CELTY_EPILOGUE_FP16    out_fp16[i] = y[i] rounded to FP16 (nearest even), i < M; y keeps the FP32 values.
+ *   CELTY_EPILOGUE_SWIGLU  the handle holds the gate projection's rows stacked on the up projection's
+ *                          (M = 2I rows): h_i = SiLU(y_i) * y_{I+i} for i < I, evaluated in FP32, rounded once to
+ *                          FP16 and stored in out_fp16[i]; every i with not(|h_i| <= tau) (the comparator of
+ *                          celty_compact, applied to the rounded value) is appended to the list
+ *                          (list_idx, list_val, list_count[0]), which celty_spmspv_list takes as the survivors of
+ *                          the down projection.  The list comes out in no particular order (thread blocks append
+ *                          to it as they finish); as a set it is exactly the thresholded h.  list_idx and list_val
+ *                          need room for I entries.
+ * All pointers are device memory of the current device.
+ */
+enum { CELTY_EPILOGUE_NONE = 0, CELTY_EPILOGUE_FP16 = 1, CELTY_EPILOGUE_SWIGLU = 2 };
+
+typedef struct {
+    int32_t kind;         /* CELTY_EPILOGUE_*                                              */
+    void *out_fp16;       /* FP16: M values; SWIGLU: M / 2 values                          */
+    float tau;            /* SWIGLU: threshold of the emitted list (finite, >= 0)          */
+    int32_t *list_idx;    /* SWIGLU: int32[M / 2]                                          */
+    uint16_t *list_val;   /* SWIGLU: FP16 bit patterns [M / 2]                             */
+    int32_t *list_count;  /* SWIGLU: int32[1], overwritten                                 */
+} celty_epilogue;
+
+/*
+ * celty_spmspv_ex -- celty_spmspv followed, in the same launch, by the work `ep` describes (NULL = none).
+ * Errors: those of celty_spmspv; CELTY_EINVAL also for a COLUMN handle, the two-launch or the ordered-merge
+ * variant, a missing output pointer, an odd M with SWIGLU.
+ */
+int celty_spmspv_ex(celty_matrix *m, const void *x_dev, float tau, void *y_dev, const celty_epilogue *ep,
+                    celty_stream_t stream);
+
+/*
+ * celty_spmspv_list -- the same product when the thresholding (step a1) has already been done by whoever produced
+ * the activations: y = sum over the n = count_dev[0] listed columns idx_dev[r] of column idx_dev[r] times the FP16
+ * value val_dev[r].  The list may be in any order; every column at most once; n <= K.  This is how the down
+ * projection consumes the list that CELTY_EPILOGUE_SWIGLU emits (the call reads the count on the device, so the
+ * two calls can follow each other on a stream without a host round trip).  `ep` as in celty_spmspv_ex.
+ * celty_last_compaction is not updated by this call (the count it reports is n).
+ * Errors: CELTY_EINVAL, CELTY_ESTATE, CELTY_ECUDA.
+ */
+int celty_spmspv_list(celty_matrix *m, const int32_t *idx_dev, const uint16_t *val_dev, const int32_t *count_dev,
+                      void *y_dev, const celty_epilogue *ep, celty_stream_t stream);
+
+/*
  * celty_spmspv_host -- the same call for HOST vectors: copies x_host (K FP16) to x_stage_dev,
  * runs celty_spmspv into y_stage_dev, copies it to y_host (M FP32) and synchronises `stream`
  * before returning.  Use page-locked host memory for the copies to be asynchronous.

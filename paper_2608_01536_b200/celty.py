@@ -35,6 +35,8 @@ SIGNATURES = {
     "celty_bind_device": (ctypes.c_int, [_vp, _vp, _sz, _vp, _sz, _vp]),
     "celty_compact": (ctypes.c_int, [_vp, _i64, _f32, _vp, _vp, _vp, _vp]),
     "celty_spmspv": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp]),
+    "celty_spmspv_ex": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp]),
+    "celty_spmspv_list": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "celty_spmspv_static": (ctypes.c_int, [_vp, _vp, _vp, _f32, _vp, _vp]),
     "celty_spmspv_host": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp, _vp]),
     "celty_last_compaction": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
@@ -95,6 +97,28 @@ def _stream_ptr(stream):
 
 class _Opts(ctypes.Structure):
     _fields_ = [("run_bits", _i32), ("layout", _i32), ("tile_rows", _i32), ("slabs_per_block", _i32)]
+
+
+class _Epilogue(ctypes.Structure):
+    _fields_ = [("kind", _i32), ("out_fp16", _vp), ("tau", _f32), ("list_idx", _vp), ("list_val", _vp),
+                ("list_count", _vp)]
+
+
+class SwigluOut:
+    """Device buffers the SiLU(gate) * up epilogue of a stacked [gate; up] product fills: h (FP16, I values) and the
+    thresholded list (idx, val, count) that `Matrix.spmspv_list` of the down projection consumes."""
+
+    def __init__(self, I: int, tau: float, device):
+        import torch
+        self.tau = float(tau)
+        self.h = torch.empty(I, dtype=torch.float16, device=device)
+        self.idx = torch.empty(I, dtype=torch.int32, device=device)
+        self.val = torch.empty(I, dtype=torch.int16, device=device)
+        self.count = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def _struct(self):
+        return _Epilogue(2, self.h.data_ptr(), self.tau, self.idx.data_ptr(), self.val.data_ptr(),
+                         self.count.data_ptr())
 
 
 class Matrix:
@@ -231,6 +255,39 @@ class Matrix:
         assert x.dtype == torch.float16 and x.numel() == self.K and x.is_contiguous()
         assert y.dtype == torch.float32 and y.numel() == self.M and y.is_contiguous()
         _check(load().celty_spmspv(self._h, x.data_ptr(), tau, y.data_ptr(), _stream_ptr(stream)), "celty_spmspv")
+        return y
+
+    def spmspv_ex(self, x, tau: float, y=None, fp16_out=None, swiglu: "SwigluOut | None" = None, stream=None):
+        """spmspv followed in the same launch by an FP16 copy of y (fp16_out: M float16) or by the SiLU(gate) * up
+        step of a stacked [gate; up] matrix (swiglu: a SwigluOut)."""
+        import torch
+        if y is None:
+            y = torch.empty(self.M, dtype=torch.float32, device=x.device)
+        assert x.dtype == torch.float16 and x.numel() == self.K and x.is_contiguous()
+        assert y.dtype == torch.float32 and y.numel() == self.M and y.is_contiguous()
+        ep = None
+        if swiglu is not None:
+            ep = swiglu._struct()
+        elif fp16_out is not None:
+            assert fp16_out.dtype == torch.float16 and fp16_out.numel() == self.M
+            ep = _Epilogue(1, fp16_out.data_ptr(), 0.0, None, None, None)
+        _check(load().celty_spmspv_ex(self._h, x.data_ptr(), tau, y.data_ptr(), ctypes.byref(ep) if ep else None,
+                                      _stream_ptr(stream)), "celty_spmspv_ex")
+        return y
+
+    def spmspv_list(self, idx, val, count, y=None, fp16_out=None, stream=None):
+        """The product from a ready-made survivor list (device tensors: int32 columns, FP16 bit patterns, int32[1]
+        count), e.g. the one a SwigluOut holds."""
+        import torch
+        if y is None:
+            y = torch.empty(self.M, dtype=torch.float32, device=idx.device)
+        assert idx.dtype == torch.int32 and val.dtype in (torch.int16, torch.float16) and count.dtype == torch.int32
+        ep = None
+        if fp16_out is not None:
+            assert fp16_out.dtype == torch.float16 and fp16_out.numel() == self.M
+            ep = _Epilogue(1, fp16_out.data_ptr(), 0.0, None, None, None)
+        _check(load().celty_spmspv_list(self._h, idx.data_ptr(), val.data_ptr(), count.data_ptr(), y.data_ptr(),
+                                        ctypes.byref(ep) if ep else None, _stream_ptr(stream)), "celty_spmspv_list")
         return y
 
     def spmspv_static(self, x, tau: float, y=None, stream=None):

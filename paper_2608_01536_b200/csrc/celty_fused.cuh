@@ -50,6 +50,20 @@ struct FusedParams {
     uint32_t units_inv, units_inv_long;
     int merge;                 // 0: partial vectors + ordered final sum; 1: bulk reduce-add of row segments into y
     uint32_t spin_limit;       // polls a bounded wait makes before it gives up
+    // a1 done by the producer of the activations: when list_count is not null the surviving columns and their
+    // values come from this list (any order, every column at most once) and x and tau are not looked at
+    const int32_t *list_idx;
+    const uint16_t *list_val;
+    const int32_t *list_count;
+    // Work on y after the merge (bulk reduce-add merge only): 0 none; 1 an FP16 copy of y; 2 y holds a stacked
+    // [gate; up] product of 2I rows: h_i = SiLU(y_i) * y_{I+i} rounded to FP16, stored, and the (i, h_i) with
+    // |h_i| > ep_tau appended to a list that the next product takes as its survivors
+    int ep_kind;
+    uint16_t *ep_out;
+    float ep_tau;
+    int32_t *ep_idx;
+    uint16_t *ep_val;
+    int32_t *ep_count;
 };
 
 constexpr uint32_t kSpinLimit = 1u << 21;   // default for FusedParams::spin_limit
@@ -365,6 +379,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     if (p.merge == 1 && warp == nwarps - 1) {
         const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
         for (int i = r0 + lane; i < r1; i += 32) p.y[i] = 0.f;
+        if (p.ep_kind == 2 && blockIdx.x == 0 && lane == 0) *p.ep_count = 0;   // appended to after the merge
         __syncwarp();
         if (lane == 0) {
             __threadfence();
@@ -380,7 +395,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
     const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 31) >> 5;
-    {
+    const bool from_list = p.list_count != nullptr;               // a1 was done by whoever produced the activations
+    if (!from_list) {
         const __half2 tau2 = __half2half2(__float2half_rd(p.tau));
         for (int w0 = 0; w0 < nwords; w0 += nthreads) {             // the same trip count for every thread
             const int w = w0 + tid;
@@ -440,7 +456,10 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     // blocks at a time (a copy per warp costs a few hundred bytes and saves a block-wide barrier behind a single
     // warp); the list is then cut into equal shares for the groups that work on different columns.
     int n_surv = 0;
-    if (streams) {
+    if (from_list) {
+        n_surv = max(0, min(p.K, __ldcg(p.list_count)));
+        if (blockIdx.x == 0 && tid == 0) *p.count = n_surv;
+    } else if (streams) {
         int carry = 0;
         for (int e0 = 0; e0 < nblk; e0 += 32) {
             const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
@@ -484,6 +503,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             // ---- column of rank r: the block of keep words that holds it, then the word, then the bit
             for (int i = lane; i < cnt; i += 32) {
                 const int r = rb + i;
+                int j;
+                uint16_t xb;
+                if (from_list) {
+                    j = min(max(__ldcg(p.list_idx + r), 0), p.K - 1);
+                    xb = __ldcg(p.list_val + r);
+                } else {
                 // the block of 32 keep words that holds rank r (the last one with blk[e] <= r), the word in it
                 // (the last one with wrel[w] <= what is left) ...
                 int e = 0;
@@ -503,11 +528,12 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                     if (k >= c) { k -= c; pos += sh; }
                 }
                 if (!CELTY_CHECK(((word >> pos) & 1u) != 0 && k == 0, 8, w)) pos = 0;
-                int j = 32 * w + pos;
+                j = 32 * w + pos;
                 if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
-                const uint16_t xb = __ldg(p.x + j);                  // x went through L1 in the thresholding pass
+                xb = __ldg(p.x + j);                                 // x went through L1 in the thresholding pass
+                }
                 items[i] = make_int2(j, (int)xb);
-                if (part == 0 && sl == 0 && CELTY_CHECK(r >= 0 && r < p.K, 10, r)) {
+                if (!from_list && part == 0 && sl == 0 && CELTY_CHECK(r >= 0 && r < p.K, 10, r)) {
                     p.idx[r] = j;
                     p.val[r] = xb;
                 }
@@ -703,6 +729,68 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         }
         CELTY_MARK(7);
         if (p.cl > 1) cluster_sync();                               // no block leaves while a peer may still read it
+        if (p.ep_kind == 0) return;
+        // ---- work on the finished y.  This block's adds must have been performed (not merely read out of shared
+        // memory), then every block's: a second wrap-around ticket, as for the clearing of y.
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __threadfence();
+        __syncthreads();
+        __shared__ int ep_warp[17];
+        if (tid == 0) {
+            __threadfence();
+            const uint32_t t = atomicInc(&p.tickets[1], 2u * gridDim.x - 1u);
+            const bool low_half = t < gridDim.x;
+            bool ok = false;
+            for (uint32_t it = 0; it < p.spin_limit; ++it) {
+                const uint32_t cur = ld_relaxed_u32(&p.tickets[1]);
+                if (low_half ? (cur >= gridDim.x) : (cur < gridDim.x)) { ok = true; break; }
+                __nanosleep(64);
+            }
+            __threadfence();
+            if (!ok) atomicOr(p.status, kStatusTimeout);
+        }
+        __syncthreads();
+        // every block takes an equal share of the rows; y is read past L1 (it was written by adds in L2)
+        if (p.ep_kind == 1) {
+            const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
+            for (int i = r0 + tid; i < r1; i += nthreads) p.ep_out[i] = __half_as_ushort(__float2half_rn(__ldcg(p.y + i)));
+            return;
+        }
+        const int half_rows = p.M / 2;
+        const int r0 = (int)((int64_t)blockIdx.x * half_rows / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * half_rows / gridDim.x);
+        for (int base = r0; base < r1; base += nthreads) {          // the same trip count for every thread
+            const int i = base + tid;
+            bool keep = false;
+            uint16_t hb = 0;
+            if (i < r1) {
+                const float gt = __ldcg(p.y + i), up = __ldcg(p.y + half_rows + i);
+                const __half h = __float2half_rn(gt / (1.f + expf(-gt)) * up);       // SiLU(gate) * up, one FP16 value
+                hb = __half_as_ushort(h);
+                p.ep_out[i] = hb;
+                keep = !(fabsf(__half2float(h)) <= p.ep_tau);                       // the comparator of a1
+            }
+            // positions in the list: within the warp by ballot, across the warps by a small scan, across the blocks
+            // by one atomic add per block and pass (the list comes out in no particular order)
+            const uint32_t bal = __ballot_sync(kFull, keep);
+            if (lane == 0) ep_warp[warp] = __popc(bal);
+            __syncthreads();
+            if (tid == 0) {
+                int total = 0;
+                for (int w = 0; w < nwarps; ++w) {
+                    const int c = ep_warp[w];
+                    ep_warp[w] = total;
+                    total += c;
+                }
+                ep_warp[16] = total ? atomicAdd(p.ep_count, total) : 0;
+            }
+            __syncthreads();
+            if (keep) {
+                const int pos = ep_warp[16] + ep_warp[warp] + __popc(bal & ((1u << lane) - 1u));
+                p.ep_idx[pos] = i;
+                p.ep_val[pos] = hb;
+            }
+            __syncthreads();
+        }
         return;
     }
 

@@ -535,15 +535,38 @@ extern "C" int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *i
     return launch_compact(x_dev, K, tau, idx_dev, val_dev, count_dev, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
-extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, celty_stream_t stream)
+namespace {
+
+struct ListInput { const int32_t *idx; const uint16_t *val; const int32_t *count; };
+
+int check_epilogue(const celty_matrix *m, const celty_epilogue *ep)
 {
-    if (!m || !x_dev || !y_dev) return CELTY_EINVAL;
-    if (!(tau >= 0.f) || !std::isfinite(tau)) return CELTY_EINVAL;
+    if (!ep || ep->kind == CELTY_EPILOGUE_NONE) return CELTY_OK;
+    if (ep->kind == CELTY_EPILOGUE_FP16) return ep->out_fp16 ? CELTY_OK : CELTY_EINVAL;
+    if (ep->kind != CELTY_EPILOGUE_SWIGLU) return CELTY_EINVAL;
+    if (!ep->out_fp16 || !ep->list_idx || !ep->list_val || !ep->list_count || (m->M & 1)) return CELTY_EINVAL;
+    if (!(ep->tau >= 0.f) || !std::isfinite(ep->tau)) return CELTY_EINVAL;
+    return CELTY_OK;
+}
+
+// The product for every entry point: x thresholded by the kernel (list == nullptr) or the survivors given as a
+// list; optional work on y after the merge.
+int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *list, void *y_dev,
+                const celty_epilogue *ep, celty_stream_t stream)
+{
+    if (!m || !y_dev || (!x_dev && !list)) return CELTY_EINVAL;
+    if (list && (!list->idx || !list->val || !list->count)) return CELTY_EINVAL;
+    if (!list && (!(tau >= 0.f) || !std::isfinite(tau))) return CELTY_EINVAL;
     if (((uintptr_t)x_dev | (uintptr_t)y_dev) & 15) return CELTY_EINVAL;
     if (!m->d_image || !m->d_ws) return CELTY_ESTATE;
+    int rc = check_epilogue(m, ep);
+    if (rc) return rc;
+    const bool extras = list || (ep && ep->kind != CELTY_EPILOGUE_NONE);
+    // lists and work after the merge exist in the single-launch kernel with the bulk reduce-add merge only
+    if (extras && !(m->layout == CELTY_LAYOUT_LANE_TILE && m->variant == 0 && m->merge != 0)) return CELTY_EINVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DeviceInfo di;
-    int rc = device_info(&di);
+    rc = device_info(&di);
     if (rc) return rc;
     uint32_t *status = reinterpret_cast<uint32_t *>(m->d_ws + m->ws.status_off);
     int32_t *count = reinterpret_cast<int32_t *>(status + 1);
@@ -559,10 +582,23 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
         if (rc) return rc;
         rc = fit_clusters(&plan);
         if (rc) return rc;
-        FusedParams fp;
+        FusedParams fp{};
+        if (list) {
+            fp.list_idx = list->idx;
+            fp.list_val = list->val;
+            fp.list_count = list->count;
+        }
+        if (ep && ep->kind != CELTY_EPILOGUE_NONE) {
+            fp.ep_kind = ep->kind;
+            fp.ep_out = static_cast<uint16_t *>(ep->out_fp16);
+            fp.ep_tau = ep->tau;
+            fp.ep_idx = ep->list_idx;
+            fp.ep_val = ep->list_val;
+            fp.ep_count = ep->list_count;
+        }
         fp.meta = reinterpret_cast<const uint32_t *>(m->d_image);
         fp.stream = stream_base;
-        fp.x = static_cast<const uint16_t *>(x_dev);
+        fp.x = static_cast<const uint16_t *>(x_dev);           // not looked at when the survivors come as a list
         fp.tau = tau;
         fp.y = y;
         fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
@@ -646,6 +682,28 @@ extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void 
     }
     CELTY_CUDA(cudaGetLastError());
     return CELTY_OK;
+}
+
+}  // namespace
+
+extern "C" int celty_spmspv(celty_matrix *m, const void *x_dev, float tau, void *y_dev, celty_stream_t stream)
+{
+    if (!x_dev) return CELTY_EINVAL;
+    return run_product(m, x_dev, tau, nullptr, y_dev, nullptr, stream);
+}
+
+extern "C" int celty_spmspv_ex(celty_matrix *m, const void *x_dev, float tau, void *y_dev, const celty_epilogue *ep,
+                               celty_stream_t stream)
+{
+    if (!x_dev) return CELTY_EINVAL;
+    return run_product(m, x_dev, tau, nullptr, y_dev, ep, stream);
+}
+
+extern "C" int celty_spmspv_list(celty_matrix *m, const int32_t *idx_dev, const uint16_t *val_dev,
+                                 const int32_t *count_dev, void *y_dev, const celty_epilogue *ep, celty_stream_t stream)
+{
+    const ListInput list{idx_dev, val_dev, count_dev};
+    return run_product(m, nullptr, 0.f, &list, y_dev, ep, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
