@@ -359,6 +359,64 @@ def run_sweep(args):
         # the same layer with the products that share an input stacked row-wise into one matrix ([q; k; v] and
         # [gate; up]): 4 calls per layer, one thresholding pass per shared x, for the sparse and the dense side alike
         extra["chain_stacked"] = chain([(15360, 5120), (5120, 5120), (27648, 5120), (5120, 13824)], "stacked")
+
+        # the stacked layer with the work between the products inside the launches: FP16 outputs, SiLU(gate) * up and
+        # its thresholded list behind the gate/up product, the down projection fed from that list (no thresholding
+        # pass of its own).  The dense side runs the four GEMVs and the element-wise step as its own kernel.
+        def chain_fused():
+            H, I = 5120, 13824
+            calls, dcalls, tot_bytes = [], [], 0.0
+            for layer in range(2):
+                mats, Wds = [], []
+                for k, (M, K) in enumerate([(3 * H, H), (H, H), (2 * I, H), (H, I)]):
+                    seed = synth.point_seed(4, 10 * layer + k + 100)
+                    W = synth.weights(seed, M, K)
+                    mask = synth.mask_bernoulli(seed, M, K, 0.5)
+                    mats.append(celty.Matrix(W, mask, device=dev))
+                    Wds.append(torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev))
+                xs = [torch.from_numpy(synth.activations(synth.point_seed(4, 200 + 10 * layer + k), H, "laplace")).to(dev)
+                      for k in range(3)]
+                taus = [synth.threshold_for_density(x.cpu().numpy(), 0.4) for x in xs]
+                ys = [torch.empty(m.M, dtype=torch.float32, device=dev) for m in mats]
+                y16 = [torch.empty(m.M, dtype=torch.float16, device=dev) for m in mats]
+                out = celty.SwigluOut(I, 0.0, dev)
+                mats[2].spmspv_ex(xs[2], taus[2], ys[2], swiglu=out)        # once, to place the list's threshold
+                torch.cuda.synchronize()
+                out.tau = synth.threshold_for_density(out.h.cpu().numpy(), 0.4)
+
+                def sparse_layer(mats=mats, xs=xs, taus=taus, ys=ys, y16=y16, out=out):
+                    mats[0].spmspv_ex(xs[0], taus[0], ys[0], fp16_out=y16[0])
+                    mats[1].spmspv_ex(xs[1], taus[1], ys[1], fp16_out=y16[1])
+                    mats[2].spmspv_ex(xs[2], taus[2], ys[2], swiglu=out)
+                    mats[3].spmspv_list(out.idx, out.val, out.count, ys[3], fp16_out=y16[3])
+                sparse_layer()
+                torch.cuda.synchronize()
+                assert all(m.last_status() == 0 for m in mats)
+                for k in range(3):
+                    idx, _ = mats[k].last_compaction()
+                    tot_bytes += mats[k].fetched_bytes(idx.cpu().numpy())[1]
+                n = int(out.count.item())
+                tot_bytes += mats[3].fetched_bytes(np.sort(out.idx[:n].cpu().numpy()))[1]
+                calls.append(sparse_layer)
+                yd = [torch.empty(m.M, dtype=torch.float16, device=dev) for m in mats]
+                hd = torch.empty(I, dtype=torch.float16, device=dev)
+
+                def dense_layer(Wds=Wds, xs=xs, yd=yd, hd=hd):
+                    torch.mv(Wds[0], xs[0], out=yd[0])
+                    torch.mv(Wds[1], xs[1], out=yd[1])
+                    torch.mv(Wds[2], xs[2], out=yd[2])
+                    torch.mul(torch.nn.functional.silu(yd[2][:I]), yd[2][I:], out=hd)
+                    torch.mv(Wds[3], hd, out=yd[3])
+                dcalls.append(dense_layer)
+            us = rotation_us(calls)
+            dus = rotation_us(dcalls)
+            return {"calls_per_layer": 4, "layers_in_rotation": 2, "us_per_layer": us,
+                    "fetched_bytes_per_layer": tot_bytes / 2, "GBps": tot_bytes / 2 / us / 1e3,
+                    "roofline_frac": tot_bytes / 2 / us / 1e3 / peak, "cublas_gemv_us_per_layer": dus,
+                    "speedup_vs_cublas": dus / us,
+                    "note": "FP16 outputs, SiLU(gate)*up and its list inside the gate/up launch, down projection from "
+                            "the list; the dense side adds the element-wise step as a kernel of its own"}
+        extra["chain_stacked_fused"] = chain_fused()
     print(json.dumps({"sweep": args.sweep, "protocol": "rotation over device copies of the layer (> 2x L2) captured in one "
                       "CUDA graph, CUDA events around the replays", "peak_GBps": peak, "points": points, **extra}))
 

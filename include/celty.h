@@ -239,6 +239,31 @@ int celty_spmspv_list(celty_matrix *m, const int32_t *idx_dev, const uint16_t *v
                       void *y_dev, const celty_epilogue *ep, celty_stream_t stream);
 
 /*
+ * celty_spmspv_batch -- the product for a small batch of N = 1 .. 8 activation vectors against the same matrix
+ * (LANE_TILE handles):  y[n] = W . threshold(x[n], tau)  for every n.  Sections 2.2-2.3 place the method against
+ * SpMM kernels that need N >= 8; this call keeps the batch-1 scheme and widens it: a column is fetched once when any
+ * of the N activations in it survives (the union of the surviving columns), and every stored entry is multiplied
+ * into N accumulators.  Two launches (union compaction, product with plain loads and an atomic merge).
+ *   x_dev  N rows of K FP16 values, row n at x_dev + n * ldx (elements), not modified
+ *   y_dev  N rows of M FP32 values, row n at y_dev + n * ldy, overwritten
+ *   list_scratch_dev  device scratch, 256-byte aligned, at least 256 + round_up(4 K, 256) + 16 K bytes (union list
+ *                     and the N values of every listed column)
+ * Errors: CELTY_EINVAL, CELTY_ESTATE, CELTY_ENOMEM (scratch too small or misaligned), CELTY_ELIMIT (the N
+ * accumulators of one slab of rows do not fit shared memory), CELTY_ECUDA.
+ */
+int celty_spmspv_batch(celty_matrix *m, const void *x_dev, int64_t ldx, int32_t N, float tau, void *y_dev, int64_t ldy,
+                       void *list_scratch_dev, size_t scratch_bytes, celty_stream_t stream);
+
+/*
+ * celty_shard_columns -- the column range [k_begin, k_end) of rank `rank` of `world` when a layer is sharded by
+ * columns over several GPUs (each GPU encodes its own columns whole, thresholds its own slice of x and produces
+ * a partial y; one all-reduce of M FP32 values then gives y -- the exchange is the caller's, e.g. NCCL through
+ * torch.distributed).  The ranges tile [0, K) in rank order and start on multiples of 8 columns, so that a
+ * shard's slice of x is 16-byte aligned.  Host-only.  Errors: CELTY_EINVAL.
+ */
+int celty_shard_columns(int64_t K, int32_t world, int32_t rank, int64_t *k_begin, int64_t *k_end);
+
+/*
  * celty_spmspv_host -- the same call for HOST vectors: copies x_host (K FP16) to x_stage_dev,
  * runs celty_spmspv into y_stage_dev, copies it to y_host (M FP32) and synchronises `stream`
  * before returning.  Use page-locked host memory for the copies to be asynchronous.

@@ -37,6 +37,8 @@ SIGNATURES = {
     "celty_spmspv": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp]),
     "celty_spmspv_ex": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp]),
     "celty_spmspv_list": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "celty_spmspv_batch": (ctypes.c_int, [_vp, _vp, _i64, _i32, _f32, _vp, _i64, _vp, _sz, _vp]),
+    "celty_shard_columns": (ctypes.c_int, [_i64, _i32, _i32, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
     "celty_spmspv_static": (ctypes.c_int, [_vp, _vp, _vp, _f32, _vp, _vp]),
     "celty_spmspv_host": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp, _vp]),
     "celty_last_compaction": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
@@ -290,6 +292,22 @@ class Matrix:
                                         ctypes.byref(ep) if ep else None, _stream_ptr(stream)), "celty_spmspv_list")
         return y
 
+    def spmspv_batch(self, x, tau: float, y=None, stream=None):
+        """y[n] = W . threshold(x[n], tau) for a batch x of shape (N, K), N <= 8; y: (N, M) float32."""
+        import torch
+        assert x.dtype == torch.float16 and x.dim() == 2 and x.shape[1] == self.K and x.stride(1) == 1
+        N = x.shape[0]
+        if y is None:
+            y = torch.empty(N, self.M, dtype=torch.float32, device=x.device)
+        assert y.dtype == torch.float32 and y.shape == (N, self.M) and y.stride(1) == 1
+        need = 256 + (4 * self.K + 255) // 256 * 256 + 16 * self.K
+        if getattr(self, "_batch_scratch", None) is None or self._batch_scratch.numel() < need:
+            self._batch_scratch = torch.empty(need, dtype=torch.uint8, device=x.device)
+        _check(load().celty_spmspv_batch(self._h, x.data_ptr(), x.stride(0), N, tau, y.data_ptr(), y.stride(0),
+                                         self._batch_scratch.data_ptr(), self._batch_scratch.numel(),
+                                         _stream_ptr(stream)), "celty_spmspv_batch")
+        return y
+
     def spmspv_static(self, x, tau: float, y=None, stream=None):
         """Same product through the entry point that needs no workspace: its scratch is a fixed array inside
         the library, for callers that cannot allocate device memory.  K <= 32768; calls that overlap on the
@@ -350,6 +368,46 @@ def compact(x, tau: float, stream=None):
                                 _stream_ptr(stream)), "celty_compact")
     n = int(cnt.item())
     return idx[:n], val[:n]
+
+
+def shard_columns(K: int, world: int, rank: int):
+    """Column range [k0, k1) of `rank` when a layer is sharded by columns over `world` GPUs."""
+    a, b = _i64(), _i64()
+    _check(load().celty_shard_columns(K, world, rank, ctypes.byref(a), ctypes.byref(b)), "celty_shard_columns")
+    return a.value, b.value
+
+
+class ColumnShard:
+    """One rank's share of a layer sharded by columns (K-sharding): it packs columns [k0, k1) of W, thresholds its
+    own slice of x, and the partial results of all ranks are summed by one all-reduce of M floats over the default
+    torch.distributed process group (NCCL between GPUs).  With a world of one it is the plain product."""
+
+    def __init__(self, W, mask=None, rank: int = 0, world: int = 1, device=None, **kw):
+        W = np.asarray(W)
+        self.K_full = W.shape[1]
+        self.rank, self.world = rank, world
+        self.k0, self.k1 = shard_columns(self.K_full, world, rank)
+        self.empty = self.k1 <= self.k0
+        if not self.empty:
+            Ws = np.ascontiguousarray(W[:, self.k0:self.k1])
+            ms = None if mask is None else np.ascontiguousarray(np.asarray(mask)[:, self.k0:self.k1])
+            self.local = Matrix(Ws, ms, device=device, **kw)
+        self.M = W.shape[0]
+
+    def spmspv(self, x, tau: float, y=None, stream=None):
+        """x: the FULL activation vector (K float16, on this rank's device); returns y = W . threshold(x, tau),
+        identical on every rank after the all-reduce."""
+        import torch
+        import torch.distributed as dist
+        if y is None:
+            y = torch.empty(self.M, dtype=torch.float32, device=x.device)
+        if self.empty:
+            y.zero_()
+        else:
+            self.local.spmspv(x[self.k0:self.k1], tau, y, stream=stream)
+        if self.world > 1:
+            dist.all_reduce(y, op=dist.ReduceOp.SUM)
+        return y
 
 
 def count_entries(mask, run_bits: int = 4):

@@ -302,6 +302,89 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     return l;
 }
 
+// Work on the finished y (FusedParams::ep_kind), every block on an equal share of the rows.  A function of its own
+// (not inlined), so that what it needs in registers does not weigh on the streaming loop of the kernel.
+struct EpilogueArgs {
+    const float *y;
+    uint32_t *tickets, *status;
+    uint32_t spin_limit;
+    int M, ep_kind;
+    uint16_t *ep_out;
+    float ep_tau;
+    int32_t *ep_idx;
+    uint16_t *ep_val;
+    int32_t *ep_count;
+};
+
+__device__ __noinline__ void fused_epilogue(const EpilogueArgs p)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nwarps = nthreads >> 5;
+    // ---- work on the finished y.  This block's adds must have been performed (not merely read out of shared
+    // memory), then every block's: a second wrap-around ticket, as for the clearing of y.
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __threadfence();
+    __syncthreads();
+    __shared__ int ep_warp[17];
+    if (tid == 0) {
+        __threadfence();
+        const uint32_t t = atomicInc(&p.tickets[1], 2u * gridDim.x - 1u);
+        const bool low_half = t < gridDim.x;
+        bool ok = false;
+        for (uint32_t it = 0; it < p.spin_limit; ++it) {
+            const uint32_t cur = ld_relaxed_u32(&p.tickets[1]);
+            if (low_half ? (cur >= gridDim.x) : (cur < gridDim.x)) { ok = true; break; }
+            __nanosleep(64);
+        }
+        __threadfence();
+        if (!ok) atomicOr(p.status, kStatusTimeout);
+    }
+    __syncthreads();
+    // every block takes an equal share of the rows; y is read past L1 (it was written by adds in L2)
+    if (p.ep_kind == 1) {
+        const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
+        for (int i = r0 + tid; i < r1; i += nthreads) p.ep_out[i] = __half_as_ushort(__float2half_rn(__ldcg(p.y + i)));
+        return;
+    }
+    const int half_rows = p.M / 2;
+    const int r0 = (int)((int64_t)blockIdx.x * half_rows / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * half_rows / gridDim.x);
+    for (int base = r0; base < r1; base += nthreads) {          // the same trip count for every thread
+        const int i = base + tid;
+        bool keep = false;
+        uint16_t hb = 0;
+        if (i < r1) {
+            const float gt = __ldcg(p.y + i), up = __ldcg(p.y + half_rows + i);
+            const __half h = __float2half_rn(gt / (1.f + expf(-gt)) * up);       // SiLU(gate) * up, one FP16 value
+            hb = __half_as_ushort(h);
+            p.ep_out[i] = hb;
+            keep = !(fabsf(__half2float(h)) <= p.ep_tau);                       // the comparator of a1
+        }
+        // positions in the list: within the warp by ballot, across the warps by a small scan, across the blocks
+        // by one atomic add per block and pass (the list comes out in no particular order)
+        const uint32_t bal = __ballot_sync(kFull, keep);
+        if (lane == 0) ep_warp[warp] = __popc(bal);
+        __syncthreads();
+        if (tid == 0) {
+            int total = 0;
+            for (int w = 0; w < nwarps; ++w) {
+                const int c = ep_warp[w];
+                ep_warp[w] = total;
+                total += c;
+            }
+            ep_warp[16] = total ? atomicAdd(p.ep_count, total) : 0;
+        }
+        __syncthreads();
+        if (keep) {
+            const int pos = ep_warp[16] + ep_warp[warp] + __popc(bal & ((1u << lane) - 1u));
+            p.ep_idx[pos] = i;
+            p.ep_val[pos] = hb;
+        }
+        __syncthreads();
+    }
+}
+
+// kExtras = false compiles the list input and the work after the merge out: the plain product keeps its
+// register budget (92 registers against 128 with them), which the streaming loop's scheduling depends on.
+template <bool kExtras>
 __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -379,7 +462,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     if (p.merge == 1 && warp == nwarps - 1) {
         const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
         for (int i = r0 + lane; i < r1; i += 32) p.y[i] = 0.f;
-        if (p.ep_kind == 2 && blockIdx.x == 0 && lane == 0) *p.ep_count = 0;   // appended to after the merge
+        if (kExtras && p.ep_kind == 2 && blockIdx.x == 0 && lane == 0) *p.ep_count = 0;   // appended to after the merge
         __syncwarp();
         if (lane == 0) {
             __threadfence();
@@ -395,7 +478,7 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
     //   blk[e]  survivors in block e (turned into survivors before block e by the scan below).
     // |x| > tau in FP32 is the same decision as |x| > (tau rounded down to FP16) in FP16; NaN is kept.
     const int ngroups = (p.K + 7) >> 3, nwords = (p.K + 31) >> 5, nblk = (nwords + 31) >> 5;
-    const bool from_list = p.list_count != nullptr;               // a1 was done by whoever produced the activations
+    const bool from_list = kExtras && p.list_count != nullptr;    // a1 was done by whoever produced the activations
     if (!from_list) {
         const __half2 tau2 = __half2half2(__float2half_rd(p.tau));
         for (int w0 = 0; w0 < nwords; w0 += nthreads) {             // the same trip count for every thread
@@ -729,71 +812,11 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         }
         CELTY_MARK(7);
         if (p.cl > 1) cluster_sync();                               // no block leaves while a peer may still read it
-        if (p.ep_kind == 0) return;
-        // ---- work on the finished y.  This block's adds must have been performed (not merely read out of shared
-        // memory), then every block's: a second wrap-around ticket, as for the clearing of y.
-        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        __threadfence();
-        __syncthreads();
-        __shared__ int ep_warp[17];
-        if (tid == 0) {
-            __threadfence();
-            const uint32_t t = atomicInc(&p.tickets[1], 2u * gridDim.x - 1u);
-            const bool low_half = t < gridDim.x;
-            bool ok = false;
-            for (uint32_t it = 0; it < p.spin_limit; ++it) {
-                const uint32_t cur = ld_relaxed_u32(&p.tickets[1]);
-                if (low_half ? (cur >= gridDim.x) : (cur < gridDim.x)) { ok = true; break; }
-                __nanosleep(64);
-            }
-            __threadfence();
-            if (!ok) atomicOr(p.status, kStatusTimeout);
-        }
-        __syncthreads();
-        // every block takes an equal share of the rows; y is read past L1 (it was written by adds in L2)
-        if (p.ep_kind == 1) {
-            const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
-            for (int i = r0 + tid; i < r1; i += nthreads) p.ep_out[i] = __half_as_ushort(__float2half_rn(__ldcg(p.y + i)));
-            return;
-        }
-        const int half_rows = p.M / 2;
-        const int r0 = (int)((int64_t)blockIdx.x * half_rows / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * half_rows / gridDim.x);
-        for (int base = r0; base < r1; base += nthreads) {          // the same trip count for every thread
-            const int i = base + tid;
-            bool keep = false;
-            uint16_t hb = 0;
-            if (i < r1) {
-                const float gt = __ldcg(p.y + i), up = __ldcg(p.y + half_rows + i);
-                const __half h = __float2half_rn(gt / (1.f + expf(-gt)) * up);       // SiLU(gate) * up, one FP16 value
-                hb = __half_as_ushort(h);
-                p.ep_out[i] = hb;
-                keep = !(fabsf(__half2float(h)) <= p.ep_tau);                       // the comparator of a1
-            }
-            // positions in the list: within the warp by ballot, across the warps by a small scan, across the blocks
-            // by one atomic add per block and pass (the list comes out in no particular order)
-            const uint32_t bal = __ballot_sync(kFull, keep);
-            if (lane == 0) ep_warp[warp] = __popc(bal);
-            __syncthreads();
-            if (tid == 0) {
-                int total = 0;
-                for (int w = 0; w < nwarps; ++w) {
-                    const int c = ep_warp[w];
-                    ep_warp[w] = total;
-                    total += c;
-                }
-                ep_warp[16] = total ? atomicAdd(p.ep_count, total) : 0;
-            }
-            __syncthreads();
-            if (keep) {
-                const int pos = ep_warp[16] + ep_warp[warp] + __popc(bal & ((1u << lane) - 1u));
-                p.ep_idx[pos] = i;
-                p.ep_val[pos] = hb;
-            }
-            __syncthreads();
-        }
+        if (!kExtras || p.ep_kind == 0) return;
+        fused_epilogue(EpilogueArgs{p.y, p.tickets, p.status, p.spin_limit, p.M, p.ep_kind, p.ep_out, p.ep_tau, p.ep_idx,
+                                    p.ep_val, p.ep_count});
         return;
     }
-
     {
         // ---- a5, ordered (clusters are not used with this merge).  Stage 1: add the G accumulators, store the block's partial (accumulator layout, no slack rows)
         const int tile_words = p.R * 32, part_words = p.Sc * tile_words;

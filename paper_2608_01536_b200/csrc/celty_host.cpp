@@ -429,6 +429,18 @@ extern "C" int celty_stored_entries(const celty_matrix *m, const int32_t *idx, i
     return CELTY_OK;
 }
 
+extern "C" int celty_shard_columns(int64_t K, int32_t world, int32_t rank, int64_t *k_begin, int64_t *k_end)
+{
+    if (K <= 0 || world < 1 || rank < 0 || rank >= world || !k_begin || !k_end) return CELTY_EINVAL;
+    // groups of 8 columns (16 bytes of FP16 activations) dealt as evenly as they go: a shard's slice of x then
+    // starts on the 16-byte boundary the kernels ask for
+    const int64_t groups = (K + 7) / 8, base = groups / world, extra = groups % world;
+    const int64_t g0 = rank * base + std::min<int64_t>(rank, extra), g1 = g0 + base + (rank < extra ? 1 : 0);
+    *k_begin = std::min<int64_t>(K, g0 * 8);
+    *k_end = std::min<int64_t>(K, g1 * 8);
+    return CELTY_OK;
+}
+
 extern "C" int celty_count_entries(const uint8_t *mask, int64_t ldm, int64_t M, int64_t K, int run_bits,
                                    int64_t *nnz, int64_t *n_pad)
 {

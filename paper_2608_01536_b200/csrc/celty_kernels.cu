@@ -320,6 +320,132 @@ k_spmspv_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ str
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Small batches (N = 2 .. 8 activation vectors against the same matrix).  Section 2.2-2.3 place the method
+// against SpMM kernels that need N >= 8 to pay off; here the batch-1 scheme is kept and widened: a column
+// is fetched once if ANY of the N activations in it survives the threshold (the union of the surviving
+// columns), and every stored entry is multiplied into N accumulators, one per vector, with the activations
+// that did not survive replaced by zero (adding value * 0 changes nothing).
+//   k_compact_batch  one thread block: union list, and per listed column its N FP16 activations (zero where
+//                    dropped), vector-major: val[n * K + position]; clears y.
+//   k_spmspv_lane_batch<NB>  lane-tile kernel with plain loads; a block works on one slab of rows (so the
+//                    N accumulators of a slab fit shared memory whatever M is), its warps on different columns.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kCompactThreads)
+k_compact_batch(const uint16_t *__restrict__ x, int64_t ldx, int N, int K, float tau, int32_t *__restrict__ idx,
+                uint16_t *__restrict__ val, int32_t *__restrict__ count, float *__restrict__ y, int64_t ldy, int M)
+{
+    __shared__ int warp_tot[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int n = 0; n < N; ++n)
+        for (int i = tid; i < M; i += kCompactThreads) y[(size_t)n * ldy + i] = 0.f;
+    int base = 0;
+    for (int tile = 0; tile < K; tile += kCompactThreads) {
+        const int j = tile + tid;
+        uint16_t h[8];
+        bool any = false;
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+            h[n] = 0;
+            if (n < N && j < K) {
+                const uint16_t b = x[(size_t)n * ldx + j];
+                if (!(fabsf(__half2float(__ushort_as_half(b))) <= tau)) {
+                    h[n] = b;
+                    any = true;
+                }
+            }
+        }
+        const unsigned bal = __ballot_sync(kFull, any);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        if (warp == 0) {
+            const int t = warp_tot[lane];
+            int s = t;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(kFull, s, d);
+                if (lane >= d) s += up;
+            }
+            warp_tot[lane] = s;                     // inclusive totals over warps
+        }
+        __syncthreads();
+        if (any) {
+            const int o = base + (warp ? warp_tot[warp - 1] : 0) + __popc(bal & ((1u << lane) - 1u));
+            idx[o] = j;
+#pragma unroll
+            for (int n = 0; n < 8; ++n)
+                if (n < N) val[(size_t)n * K + o] = h[n];
+        }
+        base += warp_tot[31];
+        __syncthreads();
+    }
+    if (tid == 0) *count = base;
+}
+
+template <int NB>
+__global__ void __launch_bounds__(1024)
+k_spmspv_lane_batch(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ stream,
+                    const int32_t *__restrict__ idx, const uint16_t *__restrict__ val,
+                    const int32_t *__restrict__ count, float *__restrict__ y, int64_t ldy, int N, int M, int K, int R,
+                    int S, int C)
+{
+    extern __shared__ float acc[];                  // [warps][NB][(R + 8) * 32]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int slab_words = (R + kTileSlack) * 32;
+    for (int i = tid; i < nwarps * NB * slab_words; i += blockDim.x) acc[i] = 0.f;
+    __syncthreads();
+    const int s = blockIdx.x % S, kslice = blockIdx.x / S, nK = gridDim.x / S;      // grid = S * nK
+    const int n = *count;
+    const int64_t units = (int64_t)nK * nwarps, u = (int64_t)kslice * nwarps + warp;
+    const int p0 = (int)(u * n / units), p1 = (int)((u + 1) * n / units);
+    float *a = acc + (size_t)warp * NB * slab_words + lane;
+    for (int p = p0; p < p1; ++p) {
+        const int j = idx[p];
+        float xv[NB];
+#pragma unroll
+        for (int b = 0; b < NB; ++b) xv[b] = b < N ? __half2float(__ushort_as_half(val[(size_t)b * K + p])) : 0.f;
+        const uint8_t *sub = stream + (size_t)meta[(size_t)j * S + s] * 16;
+        const uint32_t gl = sub[lane];
+        const uint32_t steps = __reduce_max_sync(kFull, gl);
+        const uint32_t Gs = __reduce_add_sync(kFull, gl);
+        const uint8_t *vbase = sub + kSubHeader, *rbase = vbase + 16 * (size_t)Gs;
+        uint32_t slot0 = 0, row = 0;
+        for (uint32_t q = 0; q < steps; ++q) {
+            const bool active = gl > q;
+            const uint32_t ballot = __ballot_sync(kFull, active);
+            if (active) {
+                const uint32_t slot = slot0 + __popc(ballot & ((1u << lane) - 1u));
+                const uint4 v = *reinterpret_cast<const uint4 *>(vbase + 16 * (size_t)slot);
+                const uint32_t w = *reinterpret_cast<const uint32_t *>(rbase + 4 * (size_t)slot);
+                uint32_t even, odd, total;
+                decode_group(w, even, odd, total);
+#pragma unroll
+                for (int e = 0; e < kGroup; ++e) {
+                    const float wv = entry_value(v, e);
+                    float *cell = a + (row + entry_offset(even, odd, e)) * 32;
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) cell[(size_t)b * slab_words] = fmaf(wv, xv[b], cell[(size_t)b * slab_words]);
+                }
+                row += total + kGroup;
+            }
+            slot0 += __popc(ballot);
+        }
+    }
+    __syncthreads();
+    // merge: the block's warps are added, then one atomic add per (vector, row)
+    for (int w = warp; w < R; w += nwarps) {
+        const int64_t r = tile_row(S, C, s, lane, w);
+        if (r >= M) continue;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            if (b >= N) break;
+            float v = 0.f;
+            for (int g = 0; g < nwarps; ++g) v += acc[((size_t)g * NB + b) * slab_words + w * 32 + lane];
+            if (v != 0.f) atomicAdd(&y[(size_t)b * ldy + r], v);
+        }
+    }
+}
+
 // scratch[0 .. T] = the column's logical block pointers (entries before each tile), relative to scratch[0]
 __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *__restrict__ stream, int j,
                               int S, int C, const uint32_t *__restrict__ scratch, int32_t *rows,
@@ -362,7 +488,7 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
 // asked for), so that steady-state calls make no attribute calls.  The attribute belongs to the kernel,
 // so every entry point that launches a kernel shares that kernel's cache (g_granted_*): two caches for
 // one kernel could disagree about what the runtime currently allows.
-int g_granted_fused[64], g_granted_column[64], g_granted_lane[64];
+int g_granted_fused[64], g_granted_fused_extras[64], g_granted_column[64], g_granted_lane[64];
 
 template <typename Kernel>
 int ensure_smem(Kernel kernel, size_t bytes, int *granted /* [64], per device */)
@@ -459,7 +585,7 @@ int max_active_clusters(int cl, size_t smem, int threads, int *out)
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    CELTY_CUDA(cudaOccupancyMaxActiveClusters(&n, k_spmspv_fused, &cfg));
+    CELTY_CUDA(cudaOccupancyMaxActiveClusters(&n, k_spmspv_fused<false>, &cfg));
     if (used < 64) cache[used++] = Entry{dev, cl, kb, n};
     *out = n;
     return CELTY_OK;
@@ -493,7 +619,7 @@ extern "C" int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n)
     FusedPlan plan;
     rc = plan_fused(m, di, &plan);
     if (rc) return rc;
-    rc = ensure_smem(k_spmspv_fused, plan.smem, g_granted_fused);
+    rc = ensure_smem(k_spmspv_fused<false>, plan.smem, g_granted_fused);
     if (rc) return rc;
     rc = fit_clusters(&plan);
     if (rc) return rc;
@@ -578,7 +704,8 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         FusedPlan plan;
         rc = plan_fused(m, di, &plan);
         if (rc) return rc;
-        rc = ensure_smem(k_spmspv_fused, plan.smem, g_granted_fused);
+        rc = extras ? ensure_smem(k_spmspv_fused<true>, plan.smem, g_granted_fused_extras)
+                    : ensure_smem(k_spmspv_fused<false>, plan.smem, g_granted_fused);
         if (rc) return rc;
         rc = fit_clusters(&plan);
         if (rc) return rc;
@@ -649,7 +776,8 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         }
         cfg.attrs = attr;
         cfg.numAttrs = na;
-        CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused, fp));
+        if (extras) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true>, fp));
+        else CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false>, fp));
         return CELTY_OK;
     }
     // two launches: compaction (which also clears y), then the product.  Sizes are checked and the
@@ -772,6 +900,50 @@ extern "C" int celty_spmspv_static(const celty_matrix *m, const void *image_dev,
     k_spmspv_lane<<<di.sms, 32 * (int)m->S * G, smem, st>>>(reinterpret_cast<const uint32_t *>(image),
                                                             image + m->meta_bytes, idx, val, count, y, (int)m->M, m->R,
                                                             (int)m->S, m->C, G);
+    CELTY_CUDA(cudaGetLastError());
+    return CELTY_OK;
+}
+
+extern "C" int celty_spmspv_batch(celty_matrix *m, const void *x_dev, int64_t ldx, int32_t N, float tau, void *y_dev,
+                                  int64_t ldy, void *list_scratch_dev, size_t scratch_bytes, celty_stream_t stream)
+{
+    if (!m || !x_dev || !y_dev || !list_scratch_dev) return CELTY_EINVAL;
+    if (N < 1 || N > 8 || ldx < m->K || ldy < m->M) return CELTY_EINVAL;
+    if (!(tau >= 0.f) || !std::isfinite(tau)) return CELTY_EINVAL;
+    if (m->layout != CELTY_LAYOUT_LANE_TILE) return CELTY_EINVAL;
+    if (!m->d_image) return CELTY_ESTATE;
+    // scratch: count (256 bytes), int32 idx[K], FP16 val[8][K]
+    const size_t need = 256 + round_up((size_t)m->K * 4, 256) + (size_t)8 * m->K * 2;
+    if (scratch_bytes < need || ((uintptr_t)list_scratch_dev & 255)) return CELTY_ENOMEM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    uint8_t *sc = static_cast<uint8_t *>(list_scratch_dev);
+    int32_t *count = reinterpret_cast<int32_t *>(sc);
+    int32_t *idx = reinterpret_cast<int32_t *>(sc + 256);
+    uint16_t *val = reinterpret_cast<uint16_t *>(sc + 256 + round_up((size_t)m->K * 4, 256));
+    const int NB = N <= 2 ? 2 : N <= 4 ? 4 : 8;
+    const size_t slab_bytes = (size_t)(m->R + kTileSlack) * 32 * 4;
+    const int warps = (int)std::min<size_t>(16, (size_t)di.max_smem_optin / (slab_bytes * NB));
+    if (warps < 1) return CELTY_ELIMIT;
+    const size_t smem = slab_bytes * NB * warps;
+    static int granted[3][64];
+    auto launch = [&](auto kernel, int slot) -> int {
+        const int r = ensure_smem(kernel, smem, granted[slot]);
+        if (r) return r;
+        k_compact_batch<<<1, kCompactThreads, 0, st>>>(static_cast<const uint16_t *>(x_dev), ldx, N, (int)m->K, tau, idx, val,
+                                                       count, static_cast<float *>(y_dev), ldy, (int)m->M);
+        const int nK = std::max(1, di.sms / (int)m->S);
+        kernel<<<(int)m->S * nK, 32 * warps, smem, st>>>(reinterpret_cast<const uint32_t *>(m->d_image),
+                                                          m->d_image + m->meta_bytes, idx, val, count,
+                                                          static_cast<float *>(y_dev), ldy, N, (int)m->M, (int)m->K, m->R,
+                                                          (int)m->S, m->C);
+        return CELTY_OK;
+    };
+    rc = NB == 2 ? launch(k_spmspv_lane_batch<2>, 0) : NB == 4 ? launch(k_spmspv_lane_batch<4>, 1)
+                                                             : launch(k_spmspv_lane_batch<8>, 2);
+    if (rc) return rc;
     CELTY_CUDA(cudaGetLastError());
     return CELTY_OK;
 }
