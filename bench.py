@@ -363,7 +363,7 @@ def run_sweep(args):
         # the stacked layer with the work between the products inside the launches: FP16 outputs, SiLU(gate) * up and
         # its thresholded list behind the gate/up product, the down projection fed from that list (no thresholding
         # pass of its own).  The dense side runs the four GEMVs and the element-wise step as its own kernel.
-        def chain_fused():
+        def chain_fused(consumer_side):
             H, I = 5120, 13824
             calls, dcalls, tot_bytes = [], [], 0.0
             for layer in range(2):
@@ -380,11 +380,26 @@ def run_sweep(args):
                 ys = [torch.empty(m.M, dtype=torch.float32, device=dev) for m in mats]
                 y16 = [torch.empty(m.M, dtype=torch.float16, device=dev) for m in mats]
                 out = celty.SwigluOut(I, 0.0, dev)
+                hbuf = torch.empty(I, dtype=torch.float32, device=dev)
                 mats[2].spmspv_ex(xs[2], taus[2], ys[2], swiglu=out)        # once, to place the list's threshold
                 torch.cuda.synchronize()
                 out.tau = synth.threshold_for_density(out.h.cpu().numpy(), 0.4)
 
-                def sparse_layer(mats=mats, xs=xs, taus=taus, ys=ys, y16=y16, out=out):
+                def sparse_layer(mats=mats, xs=xs, taus=taus, ys=ys, y16=y16, out=out, hbuf=hbuf):
+                    if consumer_side == "kernel":                       # nothing fused: the step is a kernel between the calls
+                        mats[0].spmspv(xs[0], taus[0], ys[0])
+                        mats[1].spmspv(xs[1], taus[1], ys[1])
+                        mats[2].spmspv(xs[2], taus[2], ys[2])
+                        torch.mul(torch.nn.functional.silu(ys[2][:I]), ys[2][I:], out=hbuf)
+                        out.h.copy_(hbuf)
+                        mats[3].spmspv(out.h, out.tau, ys[3])
+                        return
+                    if consumer_side:
+                        mats[0].spmspv(xs[0], taus[0], ys[0])
+                        mats[1].spmspv(xs[1], taus[1], ys[1])
+                        mats[2].spmspv(xs[2], taus[2], ys[2])
+                        mats[3].spmspv_swiglu(ys[2], out.tau, ys[3], h_out=out.h)
+                        return
                     mats[0].spmspv_ex(xs[0], taus[0], ys[0], fp16_out=y16[0])
                     mats[1].spmspv_ex(xs[1], taus[1], ys[1], fp16_out=y16[1])
                     mats[2].spmspv_ex(xs[2], taus[2], ys[2], swiglu=out)
@@ -395,8 +410,11 @@ def run_sweep(args):
                 for k in range(3):
                     idx, _ = mats[k].last_compaction()
                     tot_bytes += mats[k].fetched_bytes(idx.cpu().numpy())[1]
-                n = int(out.count.item())
-                tot_bytes += mats[3].fetched_bytes(np.sort(out.idx[:n].cpu().numpy()))[1]
+                if consumer_side:
+                    tot_bytes += mats[3].fetched_bytes(mats[3].last_compaction()[0].cpu().numpy())[1] + 6 * I
+                else:
+                    n = int(out.count.item())
+                    tot_bytes += mats[3].fetched_bytes(np.sort(out.idx[:n].cpu().numpy()))[1]
                 calls.append(sparse_layer)
                 yd = [torch.empty(m.M, dtype=torch.float16, device=dev) for m in mats]
                 hd = torch.empty(I, dtype=torch.float16, device=dev)
@@ -414,9 +432,14 @@ def run_sweep(args):
                     "fetched_bytes_per_layer": tot_bytes / 2, "GBps": tot_bytes / 2 / us / 1e3,
                     "roofline_frac": tot_bytes / 2 / us / 1e3 / peak, "cublas_gemv_us_per_layer": dus,
                     "speedup_vs_cublas": dus / us,
-                    "note": "FP16 outputs, SiLU(gate)*up and its list inside the gate/up launch, down projection from "
-                            "the list; the dense side adds the element-wise step as a kernel of its own"}
-        extra["chain_stacked_fused"] = chain_fused()
+                    "note": ("plain products and a separate element-wise kernel (PyTorch) between gate/up and down"
+                             if consumer_side == "kernel" else "plain products; the down projection makes SiLU(gate)*up from the FP32 gate/up result while it "
+                             "thresholds" if consumer_side else
+                             "FP16 outputs, SiLU(gate)*up and its list inside the gate/up launch, down projection from "
+                             "the list") + "; the dense side adds the element-wise step as a kernel of its own"}
+        extra["chain_stacked_fused"] = chain_fused(False)
+        extra["chain_stacked_separate_step"] = chain_fused("kernel")
+        extra["chain_stacked_swiglu_in_down"] = chain_fused(True)
     print(json.dumps({"sweep": args.sweep, "protocol": "rotation over device copies of the layer (> 2x L2) captured in one "
                       "CUDA graph, CUDA events around the replays", "peak_GBps": peak, "points": points, **extra}))
 
@@ -681,6 +704,61 @@ def dram_traffic_per_launch(name):
         return None
 
 
+def run_regsplit_study(args):
+    """Register / shared-memory accumulation split (the question of the paper's Figure 13, asked of the software
+    analogue celty_set_register_rows): microseconds per call against the number of local rows per lane that are
+    summed in registers, at 30 / 50 / 70 % of the weights pruned, on 5120 x 5120 and 28672 x 8192 (Bernoulli masks,
+    50 % of the activations kept).  Rows = 0 is the library's kernel; the line "0 (8 teams)" is that kernel held to
+    the eight teams the register builds can run, so that the split is compared at equal parallelism."""
+    import torch
+    from paper_2608_01536_b200 import build as lib_build, celty
+    lib_build.build()
+    celty.load()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    points = []
+    for (M, K) in ((5120, 5120), (28672, 8192)):
+        for s in (0.3, 0.5, 0.7):
+            seed = synth.point_seed(5, 700 + int(s * 100))
+            W = synth.weights_tiled(seed, M, K, K // 8) if M * K > (1 << 26) else synth.weights(seed, M, K)
+            mask = synth.mask_bernoulli(seed, M, K, 1.0 - s)
+            first = celty.Matrix(W, mask, device=dev)
+            copies = int(np.ceil(2.5 * l2 / first.device_bytes()[0])) + 1
+            mats = [first] + [first.clone(device=dev) for _ in range(copies - 1)]
+            xs, taus = [], []
+            for c in range(copies):
+                x = synth.activations(synth.point_seed(5, 750 + c), K, "laplace")
+                taus.append(synth.threshold_for_density(x, 0.5))
+                xs.append(torch.from_numpy(x).to(dev))
+            ys = [torch.empty(M, dtype=torch.float32, device=dev) for _ in range(copies)]
+            R = first.row_map()[1]
+            for label, rows, groups in (("0", 0, 0), ("0 (8 teams)", 0, 8), ("32", 32, 0), ("64", 64, 0), ("96", 96, 0),
+                                        ("128", 128, 0)):
+                for m in mats:
+                    m.set_register_rows(rows)
+                    m.set_launch(groups=groups)
+                calls = [(lambda c=c: mats[c].spmspv(xs[c], taus[c], ys[c])) for c in range(copies)]
+                for f in calls:
+                    f()
+                torch.cuda.synchronize()
+                assert all(m.last_status() == 0 for m in mats)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for f in calls:
+                        f()
+                g.replay()
+                reps = max(3, -(-args.sweep_calls // copies))
+                us = float(np.median(timed_regions(torch, g.replay, reps, min_total_s=0.05))) * 1e3 / (reps * copies)
+                plan = mats[0].launch_plan()
+                points.append({"M": M, "K": K, "weight_sparsity": s, "tile_rows": R, "register_rows": label,
+                               "share_of_rows_in_registers": min(1.0, rows / R), "us_per_call": us,
+                               "teams": plan["teams_per_slab"], "threads": plan["threads"]})
+                print(json.dumps(points[-1]), file=sys.stderr, flush=True)
+            del mats, first
+    print(json.dumps({"sweep": "regsplit", "points": points}))
+
+
 def run_celty(args):
     import torch
     import torch.distributed as dist
@@ -880,7 +958,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-secondary", action="store_true", help="skip the second, labelled workload")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
-    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS) + ["format", "knobs"],
+    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS) + ["format", "knobs", "regsplit"],
                     help="time every point of a configured sweep; format = compression study on the host; "
                          "knobs = launch-parameter study of --workload")
     ap.add_argument("--sweep-calls", type=int, default=600, help="calls timed per sweep point (at least)")
@@ -889,6 +967,8 @@ def main():
         run_format_study(args)
     elif args.sweep == "knobs":
         run_knob_study(args)
+    elif args.sweep == "regsplit":
+        run_regsplit_study(args)
     elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

@@ -264,6 +264,18 @@ int celty_spmspv_batch(celty_matrix *m, const void *x_dev, int64_t ldx, int32_t 
 int celty_shard_columns(int64_t K, int32_t world, int32_t rank, int64_t *k_begin, int64_t *k_end);
 
 /*
+ * celty_spmspv_swiglu -- the down projection of an MLP whose activations are made inside the call: the input is the
+ * FP32 result of the stacked [gate; up] product (gate_up_dev: 2K values, the K gate results first), and step a1
+ * works on  x_j = SiLU(gate_j) * up_j  evaluated in FP32 and rounded once to FP16 -- the same values
+ * CELTY_EPILOGUE_SWIGLU stores -- thresholding them with `tau` and listing the survivors as celty_spmspv does
+ * (celty_last_compaction then reports that list, ascending).  No launch and no pass over memory sits between the
+ * two products.  h_out_dev (may be NULL) receives the K FP16 values of x.  `ep` as in celty_spmspv_ex.
+ * Errors: as celty_spmspv_ex.
+ */
+int celty_spmspv_swiglu(celty_matrix *m, const float *gate_up_dev, float tau, void *y_dev, void *h_out_dev,
+                        const celty_epilogue *ep, celty_stream_t stream);
+
+/*
  * celty_spmspv_host -- the same call for HOST vectors: copies x_host (K FP16) to x_stage_dev,
  * runs celty_spmspv into y_stage_dev, copies it to y_host (M FP32) and synchronises `stream`
  * before returning.  Use page-locked host memory for the copies to be asynchronous.
@@ -376,6 +388,21 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  * Errors: CELTY_EINVAL.
  */
 int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth, int32_t cluster);
+
+/*
+ * celty_set_register_rows -- the register / shared-memory accumulation split (LANE_TILE, single-launch kernel).
+ * The paper moves accumulation into the register file with new hardware (Section 4.1) and studies how much of it
+ * to move (Section 6.4, "Register vs. SMEM accumulation tradeoff"); this is the software analogue on a stock SM.
+ * The first `rows` local rows of every lane's tile (0, 32, 64, 96 or 128; 0 = all sums in shared memory, the
+ * library's default) are summed in registers across all the columns a warp team works on: for such a row the
+ * kernel stores the product value * x_j into the row's shared-memory cell without loading the cell first, and
+ * after every column each lane adds its cells to statically indexed registers and clears them; the registers go
+ * to shared memory once, before the merge.  Those builds run 256 threads per block (at most eight teams).
+ * Measured slower than the default at every split (the per-column collection costs more shared-memory traffic
+ * than the loads it saves); kept as the measured answer to that question.
+ * Errors: CELTY_EINVAL.
+ */
+int celty_set_register_rows(celty_matrix *m, int32_t rows);
 
 /*
  * celty_launch_plan -- the shape the fused kernel would be launched with for this handle on the current

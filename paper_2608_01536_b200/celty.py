@@ -36,6 +36,7 @@ SIGNATURES = {
     "celty_compact": (ctypes.c_int, [_vp, _i64, _f32, _vp, _vp, _vp, _vp]),
     "celty_spmspv": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp]),
     "celty_spmspv_ex": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp]),
+    "celty_spmspv_swiglu": (ctypes.c_int, [_vp, _vp, _f32, _vp, _vp, _vp, _vp]),
     "celty_spmspv_list": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "celty_spmspv_batch": (ctypes.c_int, [_vp, _vp, _i64, _i32, _f32, _vp, _i64, _vp, _sz, _vp]),
     "celty_shard_columns": (ctypes.c_int, [_i64, _i32, _i32, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
@@ -50,6 +51,7 @@ SIGNATURES = {
     "celty_last_status": (ctypes.c_int, [_vp, _vp]),
     "celty_set_launch": (ctypes.c_int, [_vp, _i32, _i32, _i32, _i32, _i32]),
     "celty_launch_plan": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), _i32]),
+    "celty_set_register_rows": (ctypes.c_int, [_vp, _i32]),
     "celty_set_wait_limit": (ctypes.c_int, [_vp, ctypes.c_uint32]),
     "celty_last_cuda_error": (ctypes.c_int, []),
     "celty_strerror": (ctypes.c_char_p, [ctypes.c_int]),
@@ -232,6 +234,10 @@ class Matrix:
                 "slabs_per_block", "slot_bytes", "merge")
         return dict(zip(keys, [int(v) for v in out]))
 
+    def set_register_rows(self, rows: int = 0):
+        """Local rows per lane summed in registers instead of shared memory (0, 32, 64, 96 or 128)."""
+        _check(load().celty_set_register_rows(self._h, rows), "celty_set_register_rows")
+
     def set_wait_limit(self, polls: int = 0):
         """Polls a bounded wait inside the kernels makes before it gives up (0 = the library's limit)."""
         _check(load().celty_set_wait_limit(self._h, polls), "celty_set_wait_limit")
@@ -275,6 +281,21 @@ class Matrix:
             ep = _Epilogue(1, fp16_out.data_ptr(), 0.0, None, None, None)
         _check(load().celty_spmspv_ex(self._h, x.data_ptr(), tau, y.data_ptr(), ctypes.byref(ep) if ep else None,
                                       _stream_ptr(stream)), "celty_spmspv_ex")
+        return y
+
+    def spmspv_swiglu(self, gate_up, tau: float, y=None, h_out=None, fp16_out=None, stream=None):
+        """Down projection whose activations SiLU(gate) * up are made inside the call from the FP32 result of the
+        stacked [gate; up] product (gate_up: 2K float32); h_out (K float16, optional) receives them."""
+        import torch
+        if y is None:
+            y = torch.empty(self.M, dtype=torch.float32, device=gate_up.device)
+        assert gate_up.dtype == torch.float32 and gate_up.numel() == 2 * self.K and gate_up.is_contiguous()
+        ep = None
+        if fp16_out is not None:
+            ep = _Epilogue(1, fp16_out.data_ptr(), 0.0, None, None, None)
+        _check(load().celty_spmspv_swiglu(self._h, gate_up.data_ptr(), tau, y.data_ptr(),
+                                          h_out.data_ptr() if h_out is not None else None,
+                                          ctypes.byref(ep) if ep else None, _stream_ptr(stream)), "celty_spmspv_swiglu")
         return y
 
     def spmspv_list(self, idx, val, count, y=None, fp16_out=None, stream=None):

@@ -55,6 +55,11 @@ struct FusedParams {
     const int32_t *list_idx;
     const uint16_t *list_val;
     const int32_t *list_count;
+    // The activations are not given but made on the fly from the FP32 result of a stacked [gate; up] product
+    // (2K values, gate first): x_j = SiLU(g_j) * u_j rounded to FP16, for the down projection.  h_out (may be
+    // null) receives the K FP16 values.
+    const float *swiglu_in;
+    uint16_t *h_out;
     // Work on y after the merge (bulk reduce-add merge only): 0 none; 1 an FP16 copy of y; 2 y holds a stacked
     // [gate; up] product of 2I rows: h_i = SiLU(y_i) * y_{I+i} rounded to FP16, stored, and the (i, h_i) with
     // |h_i| > ep_tau appended to a list that the next product takes as its survivors
@@ -236,8 +241,12 @@ __device__ __forceinline__ void step_fetch(StepBuf &b, uint32_t gl, uint32_t q, 
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(b.w) : "r"(ra));
 }
 
+// kRegRows > 0 (the register-accumulation study): cells below `reg_lim` belong to the lane's first kRegRows local
+// rows, whose sums live in registers; for them the accumulator is not loaded (the product alone is stored, and
+// collected after the sub-block), which is what takes shared-memory loads out of the loop.
+template <int kRegRows>
 __device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t spare, uint32_t slab_begin,
-                                            uint32_t slab_end)
+                                            uint32_t slab_end, uint32_t reg_lim)
 {
     uint32_t even, odd, total;
     decode_group(b.w, even, odd, total);
@@ -263,7 +272,8 @@ __device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t
     (void)slab_begin; (void)slab_end;
     cell += (total + kGroup) * 128u;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) b.c[e] = lds_f32(b.a[e]);
+    for (int e = 0; e < 8; ++e) b.c[e] = (kRegRows > 0 && b.a[e] < reg_lim) ? 0.f : lds_f32(b.a[e]);
+    (void)reg_lim;
 }
 
 __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
@@ -304,6 +314,13 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
 
 // Work on the finished y (FusedParams::ep_kind), every block on an equal share of the rows.  A function of its own
 // (not inlined), so that what it needs in registers does not weigh on the streaming loop of the kernel.
+// SiLU(gate) * up evaluated in FP32 and rounded once to FP16 (bit pattern): the one formula behind the work after
+// a gate/up product and behind the down projection that makes its activations on the fly.
+__device__ __forceinline__ uint32_t swiglu_half_bits(float gate, float up)
+{
+    return (uint32_t)__half_as_ushort(__float2half_rn(gate / (1.f + expf(-gate)) * up));
+}
+
 struct EpilogueArgs {
     const float *y;
     uint32_t *tickets, *status;
@@ -384,8 +401,12 @@ __device__ __noinline__ void fused_epilogue(const EpilogueArgs p)
 
 // kExtras = false compiles the list input and the work after the merge out: the plain product keeps its
 // register budget (92 registers against 128 with them), which the streaming loop's scheduling depends on.
-template <bool kExtras>
-__global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
+// kRegRows > 0 is the software analogue of register-file accumulation (Section 4.1, the register / shared-memory
+// split of Section 6.4): the first kRegRows local rows of every lane are summed in registers across the team's
+// columns and written to the accumulator slab once, at the end.  Those builds run 256 threads per block (eight
+// teams at most), which is what leaves a thread room for up to 128 more registers.
+template <bool kExtras, int kRegRows>
+__global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(const FusedParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x, nwarps = nthreads >> 5;
@@ -490,7 +511,36 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 for (int c = 0; c < 4; ++c) {                          // four independent 128-bit loads per thread
                     const int q = 4 * w + c;
                     h[c][0] = h[c][1] = h[c][2] = h[c][3] = 0u;        // zero past the end of x: never kept (tau >= 0)
-                    if (8 * q + 8 <= p.K) {
+                    if (kExtras && p.swiglu_in) {                      // the activations are made here, from FP32 gate / up
+                        if (q < ngroups) {
+                            float gt[8], up[8];
+                            if (8 * q + 8 <= p.K && (p.K & 3) == 0) {  // 128-bit loads (the up half starts 16-byte aligned)
+                                const float4 a0 = __ldg(reinterpret_cast<const float4 *>(p.swiglu_in + 8 * q));
+                                const float4 a1 = __ldg(reinterpret_cast<const float4 *>(p.swiglu_in + 8 * q + 4));
+                                const float4 b0 = __ldg(reinterpret_cast<const float4 *>(p.swiglu_in + p.K + 8 * q));
+                                const float4 b1 = __ldg(reinterpret_cast<const float4 *>(p.swiglu_in + p.K + 8 * q + 4));
+                                gt[0] = a0.x; gt[1] = a0.y; gt[2] = a0.z; gt[3] = a0.w; gt[4] = a1.x; gt[5] = a1.y; gt[6] = a1.z; gt[7] = a1.w;
+                                up[0] = b0.x; up[1] = b0.y; up[2] = b0.z; up[3] = b0.w; up[4] = b1.x; up[5] = b1.y; up[6] = b1.z; up[7] = b1.w;
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int j = 8 * q + k;
+                                    gt[k] = j < p.K ? __ldg(p.swiglu_in + j) : 0.f;          // SiLU(0) * 0 = 0: never kept
+                                    up[k] = j < p.K ? __ldg(p.swiglu_in + p.K + j) : 0.f;
+                                }
+                            }
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint32_t lo = swiglu_half_bits(gt[2 * k], up[2 * k]), hi = swiglu_half_bits(gt[2 * k + 1], up[2 * k + 1]);
+                                h[c][k] = lo | (hi << 16);
+                                // every block makes all of h; the blocks share the writing of it
+                                if (p.h_out && (q % gridDim.x) == blockIdx.x) {
+                                    if (8 * q + 2 * k < p.K) p.h_out[8 * q + 2 * k] = (uint16_t)lo;
+                                    if (8 * q + 2 * k + 1 < p.K) p.h_out[8 * q + 2 * k + 1] = (uint16_t)hi;
+                                }
+                            }
+                        }
+                    } else if (8 * q + 8 <= p.K) {
                         const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p.x + 8 * q));
                         h[c][0] = v.x; h[c][1] = v.y; h[c][2] = v.z; h[c][3] = v.w;
                     } else if (q < ngroups) {
@@ -580,6 +630,10 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
         uint32_t slot = 0, parity = 0, islot = 0;                     // consumed % D, (consumed / D) & 1, issued % D
         StepBuf b0, b1;                                               // pipeline registers, live across items
         const uint32_t zeros = smem_u32(zero_group);
+        float racc[kRegRows > 0 ? kRegRows : 1];                      // register-held sums of local rows 0 .. kRegRows-1
+#pragma unroll
+        for (int i = 0; i < (kRegRows > 0 ? kRegRows : 1); ++i) racc[i] = 0.f;
+        const uint32_t reg_lim = cell0 + (uint32_t)min(kRegRows, p.R) * 128u;
 
         for (int rb = r_begin;; rb += p.cap) {                        // at least one trip: the teams meet at a barrier in it
             const int cnt = failed ? 0 : max(0, min(p.cap, r_end - rb));
@@ -613,7 +667,8 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 if (!CELTY_CHECK(((word >> pos) & 1u) != 0 && k == 0, 8, w)) pos = 0;
                 j = 32 * w + pos;
                 if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
-                xb = __ldg(p.x + j);                                 // x went through L1 in the thresholding pass
+                if (kExtras && p.swiglu_in) xb = (uint16_t)swiglu_half_bits(__ldg(p.swiglu_in + j), __ldg(p.swiglu_in + p.K + j));
+                else xb = __ldg(p.x + j);                            // x went through L1 in the thresholding pass
                 }
                 items[i] = make_int2(j, (int)xb);
                 if (!from_list && part == 0 && sl == 0 && CELTY_CHECK(r >= 0 && r < p.K, 10, r)) {
@@ -686,24 +741,33 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
                 const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
                 step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                step_decode(b0, cell, spare, slab0, slab_end);                                    // step 0
+                step_decode<kRegRows>(b0, cell, spare, slab0, slab_end, reg_lim);                                    // step 0
                 step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 uint32_t q = 1;
 #pragma unroll 2
                 for (; q + 1 < steps; q += 2) {                                            // two real steps per pass
-                    step_decode(b1, cell, spare, slab0, slab_end);                                // step q
+                    step_decode<kRegRows>(b1, cell, spare, slab0, slab_end, reg_lim);                                // step q
                     step_finish(b0, xj);                                                   // step q-1
                     step_fetch(b1, gl, q + 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                    step_decode(b0, cell, spare, slab0, slab_end);                                // step q+1
+                    step_decode<kRegRows>(b0, cell, spare, slab0, slab_end, reg_lim);                                // step q+1
                     step_finish(b1, xj);                                                   // step q
                     step_fetch(b0, gl, q + 3, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
                 }
                 if (q < steps) {                                                           // one real step left
-                    step_decode(b1, cell, spare, slab0, slab_end);
+                    step_decode<kRegRows>(b1, cell, spare, slab0, slab_end, reg_lim);
                     step_finish(b0, xj);
                     step_finish(b1, xj);
                 } else {                                                                   // only the last one to finish
                     step_finish(b0, xj);
+                }
+                if (kRegRows > 0) {
+                    // collect this column's products of the register rows and leave their cells empty for the next
+#pragma unroll
+                    for (int i = 0; i < kRegRows; ++i)
+                        if (i < p.R) {
+                            racc[i] += lds_f32(cell0 + (uint32_t)i * 128u);
+                            sts_f32(cell0 + (uint32_t)i * 128u, 0.f);
+                        }
                 }
                 // The slot's contents were consumed by loads whose values have been used, and the barrier orders
                 // every lane's reads before this point: the copy may overwrite it.
@@ -714,6 +778,11 @@ __global__ void __launch_bounds__(512, 1) k_spmspv_fused(const FusedParams p)
             }
             __syncwarp();                                         // items / imeta are rewritten by the next batch
             if (failed || rb + p.cap >= r_end) break;
+        }
+        if (kRegRows > 0 && zeroed) {                                 // the register rows go to the slab for the merge
+#pragma unroll
+            for (int i = 0; i < kRegRows; ++i)
+                if (i < p.R) sts_f32(cell0 + (uint32_t)i * 128u, racc[i]);
         }
         if (!zeroed && s < p.S) {                                     // a team without columns still owns a slab
             float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);

@@ -488,6 +488,13 @@ extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, 
     return CELTY_OK;
 }
 
+extern "C" int celty_set_register_rows(celty_matrix *m, int32_t rows)
+{
+    if (!m || !(rows == 0 || rows == 32 || rows == 64 || rows == 96 || rows == 128)) return CELTY_EINVAL;
+    m->reg_rows = rows;
+    return CELTY_OK;
+}
+
 extern "C" int celty_set_wait_limit(celty_matrix *m, uint32_t polls)
 {
     if (!m) return CELTY_EINVAL;

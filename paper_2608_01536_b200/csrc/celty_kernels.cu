@@ -488,7 +488,7 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
 // asked for), so that steady-state calls make no attribute calls.  The attribute belongs to the kernel,
 // so every entry point that launches a kernel shares that kernel's cache (g_granted_*): two caches for
 // one kernel could disagree about what the runtime currently allows.
-int g_granted_fused[64], g_granted_fused_extras[64], g_granted_column[64], g_granted_lane[64];
+int g_granted_fused[64], g_granted_fused_extras[64], g_granted_column[64], g_granted_lane[64], g_granted_reg[4][64];
 
 template <typename Kernel>
 int ensure_smem(Kernel kernel, size_t bytes, int *granted /* [64], per device */)
@@ -525,7 +525,8 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     const size_t budget = (size_t)di.max_smem_optin;
     // Teams first (each needs its own accumulator), then as many ring slots as still fit (at least two, to
     // keep a copy in flight).
-    const int g_cap = std::max(1, 16 / pl.Sc);
+    const int reg_rows = m->reg_rows;          // register-accumulation study: 256 threads, eight teams at most
+    const int g_cap = std::max(1, (reg_rows > 0 ? 8 : 16) / pl.Sc);
     const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
     const int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 4;
     pl.G = 0;
@@ -541,7 +542,7 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
         pl.D = 1;
     }
     if (pl.G == 0) return CELTY_EINVAL;
-    pl.threads = 512;
+    pl.threads = reg_rows > 0 ? 256 : 512;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
     pl.merge = (m->merge >= 0 ? m->merge : 1);
     int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
@@ -585,7 +586,7 @@ int max_active_clusters(int cl, size_t smem, int threads, int *out)
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    CELTY_CUDA(cudaOccupancyMaxActiveClusters(&n, k_spmspv_fused<false>, &cfg));
+    CELTY_CUDA(cudaOccupancyMaxActiveClusters(&n, k_spmspv_fused<false, 0>, &cfg));
     if (used < 64) cache[used++] = Entry{dev, cl, kb, n};
     *out = n;
     return CELTY_OK;
@@ -619,7 +620,7 @@ extern "C" int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n)
     FusedPlan plan;
     rc = plan_fused(m, di, &plan);
     if (rc) return rc;
-    rc = ensure_smem(k_spmspv_fused<false>, plan.smem, g_granted_fused);
+    rc = ensure_smem(k_spmspv_fused<false, 0>, plan.smem, g_granted_fused);
     if (rc) return rc;
     rc = fit_clusters(&plan);
     if (rc) return rc;
@@ -664,6 +665,7 @@ extern "C" int celty_compact(const void *x_dev, int64_t K, float tau, int32_t *i
 namespace {
 
 struct ListInput { const int32_t *idx; const uint16_t *val; const int32_t *count; };
+struct SwigluInput { const float *gate_up; uint16_t *h_out; };
 
 int check_epilogue(const celty_matrix *m, const celty_epilogue *ep)
 {
@@ -678,16 +680,17 @@ int check_epilogue(const celty_matrix *m, const celty_epilogue *ep)
 // The product for every entry point: x thresholded by the kernel (list == nullptr) or the survivors given as a
 // list; optional work on y after the merge.
 int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *list, void *y_dev,
-                const celty_epilogue *ep, celty_stream_t stream)
+                const celty_epilogue *ep, celty_stream_t stream, const SwigluInput *sw = nullptr)
 {
-    if (!m || !y_dev || (!x_dev && !list)) return CELTY_EINVAL;
+    if (!m || !y_dev || (!x_dev && !list && !sw)) return CELTY_EINVAL;
+    if (sw && (!sw->gate_up || ((uintptr_t)sw->gate_up & 15))) return CELTY_EINVAL;
     if (list && (!list->idx || !list->val || !list->count)) return CELTY_EINVAL;
     if (!list && (!(tau >= 0.f) || !std::isfinite(tau))) return CELTY_EINVAL;
     if (((uintptr_t)x_dev | (uintptr_t)y_dev) & 15) return CELTY_EINVAL;
     if (!m->d_image || !m->d_ws) return CELTY_ESTATE;
     int rc = check_epilogue(m, ep);
     if (rc) return rc;
-    const bool extras = list || (ep && ep->kind != CELTY_EPILOGUE_NONE);
+    const bool extras = list || sw || (ep && ep->kind != CELTY_EPILOGUE_NONE);
     // lists and work after the merge exist in the single-launch kernel with the bulk reduce-add merge only
     if (extras && !(m->layout == CELTY_LAYOUT_LANE_TILE && m->variant == 0 && m->merge != 0)) return CELTY_EINVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -704,8 +707,13 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         FusedPlan plan;
         rc = plan_fused(m, di, &plan);
         if (rc) return rc;
-        rc = extras ? ensure_smem(k_spmspv_fused<true>, plan.smem, g_granted_fused_extras)
-                    : ensure_smem(k_spmspv_fused<false>, plan.smem, g_granted_fused);
+        if (extras && m->reg_rows) return CELTY_EINVAL;
+        rc = extras ? ensure_smem(k_spmspv_fused<true, 0>, plan.smem, g_granted_fused_extras)
+             : m->reg_rows == 32 ? ensure_smem(k_spmspv_fused<false, 32>, plan.smem, g_granted_reg[0])
+             : m->reg_rows == 64 ? ensure_smem(k_spmspv_fused<false, 64>, plan.smem, g_granted_reg[1])
+             : m->reg_rows == 96 ? ensure_smem(k_spmspv_fused<false, 96>, plan.smem, g_granted_reg[2])
+             : m->reg_rows == 128 ? ensure_smem(k_spmspv_fused<false, 128>, plan.smem, g_granted_reg[3])
+                                  : ensure_smem(k_spmspv_fused<false, 0>, plan.smem, g_granted_fused);
         if (rc) return rc;
         rc = fit_clusters(&plan);
         if (rc) return rc;
@@ -714,6 +722,10 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
             fp.list_idx = list->idx;
             fp.list_val = list->val;
             fp.list_count = list->count;
+        }
+        if (sw) {
+            fp.swiglu_in = sw->gate_up;
+            fp.h_out = sw->h_out;
         }
         if (ep && ep->kind != CELTY_EPILOGUE_NONE) {
             fp.ep_kind = ep->kind;
@@ -776,8 +788,12 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         }
         cfg.attrs = attr;
         cfg.numAttrs = na;
-        if (extras) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true>, fp));
-        else CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false>, fp));
+        if (extras) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true, 0>, fp));
+        else if (m->reg_rows == 32) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 32>, fp));
+        else if (m->reg_rows == 64) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 64>, fp));
+        else if (m->reg_rows == 96) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 96>, fp));
+        else if (m->reg_rows == 128) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 128>, fp));
+        else CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 0>, fp));
         return CELTY_OK;
     }
     // two launches: compaction (which also clears y), then the product.  Sizes are checked and the
@@ -825,6 +841,13 @@ extern "C" int celty_spmspv_ex(celty_matrix *m, const void *x_dev, float tau, vo
 {
     if (!x_dev) return CELTY_EINVAL;
     return run_product(m, x_dev, tau, nullptr, y_dev, ep, stream);
+}
+
+extern "C" int celty_spmspv_swiglu(celty_matrix *m, const float *gate_up_dev, float tau, void *y_dev, void *h_out_dev,
+                                   const celty_epilogue *ep, celty_stream_t stream)
+{
+    const SwigluInput sw{gate_up_dev, static_cast<uint16_t *>(h_out_dev)};
+    return run_product(m, nullptr, tau, nullptr, y_dev, ep, stream, &sw);
 }
 
 extern "C" int celty_spmspv_list(celty_matrix *m, const int32_t *idx_dev, const uint16_t *val_dev,

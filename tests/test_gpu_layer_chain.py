@@ -135,6 +135,36 @@ def test_swiglu_step_list_and_down_projection(I, K, d_a, d_h):
         assert np.all(err <= ref["tol_yd"]), (call, worst, err[worst], ref["tol_yd"][worst])
 
 
+@pytest.mark.parametrize("I,K,d_a,d_h", [(1536, 1024, 0.4, 0.4), (701, 333, 0.9, 0.1), (13824, 5120, 0.4, 0.4)])
+def test_swiglu_made_inside_the_down_projection(I, K, d_a, d_h):
+    """The other way to fuse the step: the gate/up product is a plain call, and the down projection makes
+    SiLU(gate) * up itself while it thresholds (no launch, no pass over memory in between)."""
+    Wgu, mgu, Wd, md = _layer(I + K + 1, I, K)
+    x = synth.activations(I + K + 1, K, "laplace")
+    tau = synth.threshold_for_density(x, d_a)
+    ref = _reference_chain(Wgu, mgu, Wd, md, x, tau, d_h)
+    mg = celty.Matrix(Wgu, mgu, device="cuda")
+    mdn = celty.Matrix(Wd, md, device="cuda")
+    h = torch.zeros(I, dtype=torch.float16, device="cuda")
+    for call in range(2):
+        y = mg.spmspv(_dev(x), tau)
+        yd = mdn.spmspv_swiglu(y, ref["tau2"], h_out=h)
+        torch.cuda.synchronize()
+        assert mg.last_status() == 0 and mdn.last_status() == 0
+        h_gpu = h.cpu().numpy()
+        assert np.all(np.abs(h_gpu.astype(np.float64) - ref["hv"]) <= ref["tol_h"]), call
+        li, lv = mdn.last_compaction()
+        li, lv = li.cpu().numpy(), lv.cpu().numpy().view(np.uint16)
+        with np.errstate(invalid="ignore"):
+            own = np.flatnonzero(~(np.abs(h_gpu.astype(np.float32)) <= np.float32(ref["tau2"])))
+        assert np.array_equal(li, own)                               # ascending, exactly the kernel's own h thresholded
+        assert np.array_equal(lv, h_gpu.view(np.uint16)[li])
+        sym = np.setxor1d(li, ref["idx"])
+        assert np.all(ref["near"][sym]) and sym.size <= max(2, I // 200)
+        err = np.abs(yd.cpu().numpy().astype(np.float64) - ref["yd"])
+        assert np.all(err <= ref["tol_yd"]), (call, float((err - ref["tol_yd"]).max()))
+
+
 def test_list_input_matches_thresholded_input():
     """A list made by the oracle's compaction (shuffled: any order is allowed) gives the product that thresholding x
     inside the call gives."""

@@ -459,6 +459,37 @@ def test_back_to_back_calls_do_not_interfere():
         _check_y(y.cpu().numpy(), W, mask, xs[i], taus[i])
 
 
+@pytest.mark.parametrize("rows", [32, 64, 96, 128])
+@pytest.mark.parametrize("M,K,d_w,tile_rows", [(4096, 512, 0.5, 0), (11008, 160, 0.3, 0), (3000, 200, 0.7, 40),
+                                               (28672, 64, 0.5, 0), (777, 129, 0.2, 5)])
+def test_register_accumulation_variants(rows, M, K, d_w, tile_rows):
+    """The software analogue of register-file accumulation (Section 4.1; the split of Section 6.4): the first
+    `rows` local rows of every lane summed in registers.  Bit-exact on integer data, within the bound on random
+    data, the list unchanged -- for every split, including splits beyond the tile's own rows."""
+    Wi = synth.integer_weights(M + K + rows, M, K)
+    mask = synth.mask_bernoulli(M + K + rows, M, K, d_w)
+    xi = synth.integer_activations(M + K, K)
+    m = celty.Matrix(Wi, mask, tile_rows=tile_rows, device="cuda")
+    m.set_register_rows(rows)
+    assert m.launch_plan()["threads"] == 256
+    for grid, groups in ((0, 0), (5, 3), (148, 8)):
+        m.set_launch(grid=grid, groups=groups)
+        _check_y(_run(m, xi, 1.0), Wi, mask, xi, 1.0, exact=True)
+    W = synth.weights(M + K, M, K)
+    x = synth.activations(M + K, K, "laplace")
+    tau = synth.threshold_for_density(x, 0.5)
+    m2 = celty.Matrix(W, mask, tile_rows=tile_rows, device="cuda")
+    m2.set_register_rows(rows)
+    for _ in range(2):
+        _check_y(_run(m2, x, tau), W, mask, x, tau)
+    idx, val = m2.last_compaction()
+    oi, ov, _ = orc.compact(x, tau)
+    assert np.array_equal(idx.cpu().numpy(), oi) and np.array_equal(val.cpu().numpy().view(np.uint16), ov)
+    m2.set_register_rows(0)
+    assert m2.launch_plan()["threads"] == 512
+    _check_y(_run(m2, x, tau), W, mask, x, tau)
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
     """Every wait inside the fused kernel has a poll limit.  Here one is made to run out without faulting or
     hanging anything: the limit is set low and the ticket counter that tells a block when every other block has
