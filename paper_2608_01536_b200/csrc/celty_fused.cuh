@@ -14,15 +14,18 @@
 //   a3  each lane decodes its own tile's runs on packed bytes and keeps a running row;
 //   a4  value * x_j is accumulated (FP16 x FP16 + FP32 fused multiply-add) into the lane's private bank of
 //       the team's accumulator;
-//   a5  the thread blocks of a cluster add their accumulators through distributed shared memory, each
-//       block the row segments it owns; the row map makes a slab's accumulator a sequence of 32*C-row
+//   a5  the block adds its G accumulators; the row map makes a slab's accumulator a sequence of 32*C-row
 //       segments of y, and each goes out as one bulk reduce-add copy (FP32 add in L2) once the tickets show
-//       that every block has cleared its share of y.  Option: per-block partial vectors, a bounded
-//       grid-wide ticket barrier and a sum in a fixed order (bit-reproducible, no clearing of y).
+//       that every block has cleared its share of y.  Options: clusters of 2 or 4 thread blocks that first add
+//       their sums through distributed shared memory, each block then sending only the segments it owns
+//       (measured: no faster, so off by default); per-block partial vectors, a bounded grid-wide ticket
+//       barrier and a sum in a fixed order (bit-reproducible, no clearing of y).
+//   then, on request: an FP16 copy of y, or SiLU(gate) * up of a stacked [gate; up] product with its
+//       thresholded list (fused_epilogue), once a second ticket shows that every block's adds are done.
 //
 // Rows are split over P parts of Sc slabs each, columns over the blocks of a part and, inside a block, over
-// G teams per slab; a team = one warp with its own accumulator slab.  Every block must be resident at once (grid <= SM count)
-// because of the tickets.  All waits are bounded: when one runs out the kernel sets kStatusTimeout in the
+// G teams per slab; a team = one warp with its own accumulator slab.  Every block must be resident at once
+// (grid <= SM count) because of the tickets.  All waits are bounded: when one runs out the kernel sets kStatusTimeout in the
 // status word and carries on to a clean exit.
 
 struct FusedParams {
@@ -35,12 +38,11 @@ struct FusedParams {
     uint16_t *val;
     int32_t *count;
     uint32_t *status;
-    uint32_t *tickets;         // [0] y cleared / partial stored, [1] departed
+    uint32_t *tickets;         // [0] y cleared / partial stored, [1] adds done (work after the merge) / departed
     float *partials;           // gridDim.x vectors of Sc * R * 32 floats (accumulator layout)
     int M, K, R, S, C;         // rows, columns, local rows per tile, slabs, chunk of the row map (tile_row)
     int G, Sc, P, D;           // teams per slab, slabs per block, row parts, ring depth
     int cl;                    // thread blocks per cluster (1, 2 or 4); blocks of a cluster share a row part
-    long long stream_bytes;    // size of the entry stream (used by the self-checks of development builds)
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // columns a team looks up per batch
     int win_cols;              // columns of the offset table a block copies into shared memory at its start
@@ -72,32 +74,6 @@ struct FusedParams {
 };
 
 constexpr uint32_t kSpinLimit = 1u << 21;   // default for FusedParams::spin_limit
-
-// Development builds only (compiled out of the product):
-//   -DCELTY_TRACE  thread 0 of every block stores clock64() at phase k into trace[blockIdx.x * 16 + k];
-//   -DCELTY_GUARD  every index is range-checked; a failed check records (value, count) at
-//                  trace[192 * 16 + 2 * code] and the access is skipped or redirected, so that a wrong
-//                  index shows up as data instead of as a fault.
-#if defined(CELTY_TRACE) || defined(CELTY_GUARD)
-__constant__ long long *g_celty_trace = nullptr;
-#endif
-#ifdef CELTY_TRACE
-#define CELTY_MARK(k)                                                        \
-    do {                                                                     \
-        if (threadIdx.x == 0 && g_celty_trace) g_celty_trace[blockIdx.x * 16 + (k)] = clock64(); \
-    } while (0)
-#else
-#define CELTY_MARK(k)
-#endif
-#ifdef CELTY_GUARD
-#define CELTY_CHECK(ok, code, value)                                                                   \
-    ((ok) ? true                                                                                       \
-          : (g_celty_trace ? (g_celty_trace[192 * 16 + 2 * (code)] = (long long)(value),               \
-                              g_celty_trace[192 * 16 + 2 * (code) + 1] += 1, false)                    \
-                           : false))
-#else
-#define CELTY_CHECK(ok, code, value) true
-#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -226,15 +202,12 @@ __device__ __forceinline__ void fma_pair(uint32_t pair, uint16_t x, float c0, fl
 }
 
 __device__ __forceinline__ void step_fetch(StepBuf &b, uint32_t gl, uint32_t q, uint32_t q_end, uint32_t &cum,
-                                           uint32_t lt_mask, uint32_t vbase, uint32_t rbase, uint32_t slot_end,
-                                           uint32_t zeros)
+                                           uint32_t lt_mask, uint32_t vbase, uint32_t rbase, uint32_t zeros)
 {
     bool act = gl > q && q < q_end;
     const uint32_t bal = __ballot_sync(kFull, act);
     const uint32_t k = cum + __popc(bal & lt_mask);
     cum += __popc(bal);
-    if (!CELTY_CHECK(!act || (vbase + 16 * k + 16 <= slot_end && rbase + 4 * k + 4 <= slot_end), 1, k)) act = false;
-    (void)slot_end;
     b.act = act;
     const uint32_t va = act ? vbase + 16 * k : zeros, ra = act ? rbase + 4 * k : zeros;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(b.v.x), "=r"(b.v.y), "=r"(b.v.z), "=r"(b.v.w) : "r"(va));
@@ -245,8 +218,7 @@ __device__ __forceinline__ void step_fetch(StepBuf &b, uint32_t gl, uint32_t q, 
 // rows, whose sums live in registers; for them the accumulator is not loaded (the product alone is stored, and
 // collected after the sub-block), which is what takes shared-memory loads out of the loop.
 template <int kRegRows>
-__device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t spare, uint32_t slab_begin,
-                                            uint32_t slab_end, uint32_t reg_lim)
+__device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t spare, uint32_t reg_lim)
 {
     uint32_t even, odd, total;
     decode_group(b.w, even, odd, total);
@@ -262,14 +234,6 @@ __device__ __forceinline__ void step_decode(StepBuf &b, uint32_t &cell, uint32_t
     b.a[6] = __dp4a(even, 0x80000000u, cell);
     b.a[7] = __dp4a(odd, 0x80000000u, cell);
     b.h = b.v;
-#ifdef CELTY_GUARD
-    for (int e = 0; e < 8; ++e)
-        if (!CELTY_CHECK(b.a[e] >= slab_begin && b.a[e] + 4 <= slab_end, 2, b.a[e])) {
-            b.a[e] = slab_begin + (b.a[e] & 124u);                 // a cell of this lane's bank; add nothing
-            b.h = make_uint4(0, 0, 0, 0);
-        }
-#endif
-    (void)slab_begin; (void)slab_end;
     cell += (total + kGroup) * 128u;
 #pragma unroll
     for (int e = 0; e < 8; ++e) b.c[e] = (kRegRows > 0 && b.a[e] < reg_lim) ? 0.f : lds_f32(b.a[e]);
@@ -442,7 +406,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const int g = team / p.Sc, sl = team - g * p.Sc;
     const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
 
-    CELTY_MARK(0);
     // Programmatic dependent launch: let the next kernel of the stream be scheduled as this one's blocks retire,
     // and do everything that touches neither the caller's vectors nor the workspace (warming L2 with the offset
     // table, setting up shared memory) before waiting for the previous kernel of the stream to be complete.
@@ -576,9 +539,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             if (lane == 31 && (w >> 5) < nblk) const_cast<int *>(blk)[w >> 5] = incl;
         }
     }
-    CELTY_MARK(10);
     __syncthreads();
-    CELTY_MARK(1);
     bool failed = false;
     // the window has had the whole thresholding pass to arrive; nobody may clear an accumulator before it has
     if (p.win_cols > 0 && !mbar_wait_bounded(win_bar, 0, p.spin_limit)) {
@@ -609,7 +570,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         n_surv = carry;
         if (blockIdx.x == 0 && warp == 0 && lane == 0) *p.count = carry;
     }
-    CELTY_MARK(2);
 
     if (streams) {
         // team u of nK * G owns n / units ranks, the first n mod units teams one more.  n / units without a
@@ -620,7 +580,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         const int u = kslice * p.G + g;
         const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
-        const uint32_t cell0 = slab0 + 4u * lane, slab_end = slab0 + (uint32_t)slab_words * 4u;
+        const uint32_t cell0 = slab0 + 4u * lane;
         const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
         const uint32_t bar0 = smem_u32(&bars[team * p.D]);
         bool zeroed = false;
@@ -664,14 +624,12 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                     const int c = __popc((word >> pos) & ((1u << sh) - 1u));
                     if (k >= c) { k -= c; pos += sh; }
                 }
-                if (!CELTY_CHECK(((word >> pos) & 1u) != 0 && k == 0, 8, w)) pos = 0;
                 j = 32 * w + pos;
-                if (!CELTY_CHECK(j >= 0 && j < p.K, 3, j)) j = 0;
                 if (kExtras && p.swiglu_in) xb = (uint16_t)swiglu_half_bits(__ldg(p.swiglu_in + j), __ldg(p.swiglu_in + p.K + j));
                 else xb = __ldg(p.x + j);                            // x went through L1 in the thresholding pass
                 }
                 items[i] = make_int2(j, (int)xb);
-                if (!from_list && part == 0 && sl == 0 && CELTY_CHECK(r >= 0 && r < p.K, 10, r)) {
+                if (!from_list && part == 0 && sl == 0) {
                     p.idx[r] = j;
                     p.val[r] = xb;
                 }
@@ -687,9 +645,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                         o1 = p.meta[(size_t)j * p.S + s + 1];
                     }
                     imeta[i] = make_uint2(o0, (o1 - o0) * 16u);
-                    if (!CELTY_CHECK(o1 > o0 && (o1 - o0) * 16u <= (uint32_t)p.slot_bytes &&
-                                         (long long)o1 * 16 <= p.stream_bytes, 4, o1 - o0))
-                        imeta[i] = make_uint2(0u, (uint32_t)kSubHeader);
                 }
             }
             // The accumulators take the place of the window: every team has to be through with its look-ups
@@ -711,7 +666,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 if (++islot == (uint32_t)p.D) islot = 0;
             };
             for (int i = 0; i < min(cnt, p.D); ++i) issue_im(imeta[i]);
-            CELTY_MARK(3);
             if (!zeroed) {                                          // clear the slab while the first copies fly
                 float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
                 for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -724,7 +678,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 if (!mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
                 failed = __any_sync(kFull, failed);
                 if (failed) break;                                    // the copies still in flight are awaited below
-                if (i == 0) CELTY_MARK(4);
                 const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
                 // what the refill at the end of this sub-block will need, read now so that it does not wait then
                 const bool refill = i + p.D < cnt;
@@ -736,25 +689,24 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 asm volatile("ld.shared.u32 %0, [%1];" : "=r"(hw) : "r"(sub + 32));       // vectors | steps << 16
                 const uint32_t steps = hw >> 16, Gs = hw & 0xFFFFu;
                 const uint32_t vbase = sub + kSubHeader, rbase = vbase + 16 * Gs;
-                const uint32_t slot_end = sub + (uint32_t)p.slot_bytes;
                 uint32_t cum = 0, cell = cell0;
                 const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
-                step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                step_decode<kRegRows>(b0, cell, spare, slab0, slab_end, reg_lim);                                    // step 0
-                step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, zeros);
+                step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, zeros);
+                step_decode<kRegRows>(b0, cell, spare, reg_lim);                                    // step 0
+                step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, zeros);
                 uint32_t q = 1;
 #pragma unroll 2
                 for (; q + 1 < steps; q += 2) {                                            // two real steps per pass
-                    step_decode<kRegRows>(b1, cell, spare, slab0, slab_end, reg_lim);                                // step q
+                    step_decode<kRegRows>(b1, cell, spare, reg_lim);                                // step q
                     step_finish(b0, xj);                                                   // step q-1
-                    step_fetch(b1, gl, q + 2, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
-                    step_decode<kRegRows>(b0, cell, spare, slab0, slab_end, reg_lim);                                // step q+1
+                    step_fetch(b1, gl, q + 2, steps, cum, lt_mask, vbase, rbase, zeros);
+                    step_decode<kRegRows>(b0, cell, spare, reg_lim);                                // step q+1
                     step_finish(b1, xj);                                                   // step q
-                    step_fetch(b0, gl, q + 3, steps, cum, lt_mask, vbase, rbase, slot_end, zeros);
+                    step_fetch(b0, gl, q + 3, steps, cum, lt_mask, vbase, rbase, zeros);
                 }
                 if (q < steps) {                                                           // one real step left
-                    step_decode<kRegRows>(b1, cell, spare, slab0, slab_end, reg_lim);
+                    step_decode<kRegRows>(b1, cell, spare, reg_lim);
                     step_finish(b0, xj);
                     step_finish(b1, xj);
                 } else {                                                                   // only the last one to finish
@@ -798,7 +750,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         }
     }
     __syncthreads();
-    CELTY_MARK(5);
 
     if (p.merge == 1) {
         // ---- a5 by bulk reduce-add.  The block adds its G accumulators; the row segments of its slabs (32*C rows
@@ -855,7 +806,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
-        CELTY_MARK(6);
         // The row map makes local rows [kC, kC + C) of a slab 32*C consecutive rows of y, in accumulator
         // order (with one slab the whole accumulator is y itself): each such segment is one bulk reduce-add.
         {
@@ -879,7 +829,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may go once it has been read
         }
-        CELTY_MARK(7);
         if (p.cl > 1) cluster_sync();                               // no block leaves while a peer may still read it
         if (!kExtras || p.ep_kind == 0) return;
         fused_epilogue(EpilogueArgs{p.y, p.tickets, p.status, p.spin_limit, p.M, p.ep_kind, p.ep_out, p.ep_tau, p.ep_idx,
@@ -905,7 +854,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 }
         }
         __syncthreads();
-        CELTY_MARK(6);
         if (tid == 0) {
             __threadfence();                                          // the block's stores, ordered by the barrier above
             atomicAdd(&p.tickets[0], 1u);
@@ -917,7 +865,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             if (!ok) atomicOr(p.status, kStatusTimeout);
         }
         __syncthreads();
-        CELTY_MARK(7);
 
         // ---- a5, stage 2: the nK blocks of a part share its words; partial b of this part = block b*P + part.
         // The block's words are cut into chunks of 32; the warps split (chunk, range of partials) pairs so that
@@ -943,9 +890,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                             float t[16];
     #pragma unroll
                             for (int k = 0; k < 16; ++k)
-                                t[k] = (b0 + k < b_hi && CELTY_CHECK((size_t)(b0 + k) * stride + (size_t)part * part_words + word <
-                                                                         (size_t)gridDim.x * part_words, 13, b0 + k))
-                                           ? __ldcg(src + (size_t)(b0 + k) * stride) : 0.f;
+                                t[k] = b0 + k < b_hi ? __ldcg(src + (size_t)(b0 + k) * stride) : 0.f;
     #pragma unroll
                             for (int k = 0; k < 16; ++k) sum += t[k];
                         }
@@ -968,7 +913,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             }
         }
     }
-    CELTY_MARK(8);
     __syncthreads();
     if (tid == 0) {
         const uint32_t t = atomicAdd(&p.tickets[1], 1u);
@@ -977,7 +921,6 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             atomicExch(&p.tickets[1], 0u);
         }
     }
-    CELTY_MARK(9);
 }
 
 struct FusedPlan {

@@ -97,7 +97,6 @@ struct celty_matrix {
     celty::WorkspaceLayout ws{};
     int32_t grid = 0, variant = 0, groups = 0, depth = 0, cluster = 0;
     int32_t reg_rows = 0;                     // register-accumulation study: local rows per lane summed in registers
-    int32_t exp_flags = 0;                    // experiments: 1 = no offset window
     uint32_t spin_limit = 0;                  // bounded waits inside the kernels: 0 = the library's limit
     int32_t last_grid = 0, last_merge = -1;   // what the tickets in the workspace were last used with
     int32_t no_overlap = 0; // fused kernel: 1 = plain launch (no programmatic dependent launch)

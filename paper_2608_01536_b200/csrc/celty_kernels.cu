@@ -630,14 +630,6 @@ extern "C" int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n)
     return CELTY_OK;
 }
 
-#if defined(CELTY_TRACE) || defined(CELTY_GUARD)
-// Development builds only: where the fused kernel stores its phase timestamps (device pointer, 16 per block).
-extern "C" int celty_debug_set_trace(long long *trace_dev)
-{
-    CELTY_CUDA(cudaMemcpyToSymbol(g_celty_trace, &trace_dev, sizeof(trace_dev)));
-    return CELTY_OK;
-}
-#endif
 
 extern "C" int celty_bind_device(celty_matrix *m, void *image_dev, size_t image_bytes, void *workspace_dev,
                                  size_t workspace_bytes, celty_stream_t stream)
@@ -751,8 +743,6 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
             const size_t words = std::min<size_t>(std::min<size_t>(acc_bytes, 32768) / 4, (size_t)m->K * m->S + 4);
             fp.win_cols = (int)std::min<int64_t>(m->K, words >= 8 ? (int64_t)((words - 8) / m->S) : 0);
         }
-        if (m->exp_flags & 1) fp.win_cols = 0;
-        fp.stream_bytes = (long long)m->stream_bytes;
         fp.merge = plan.merge;
         fp.spin_limit = m->spin_limit ? m->spin_limit : kSpinLimit;
         auto inverse = [](uint64_t units) { return units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / units); };
