@@ -629,6 +629,7 @@ class Workload:
         # x read, the list written, y written -- no alignment padding, no per-block headers
         self.bare_bytes = 2.5 * float(np.mean(entries)) + 8 * n + 2 * K + 6 * n + 4 * M
         self.info = self.mats[0].info()
+        self.layout_stats = self.mats[0].layout_stats() if layout == celty.LAYOUT_LANE_TILE else None
         self.graph = None
         self.unit = None
 
@@ -897,7 +898,12 @@ def run_celty(args):
         },
         "bytes_per_call": {"entry_stream": wl.stream_bytes, "total": wl.total_bytes, "bare_format": wl.bare_bytes,
                            "total_over_bare": wl.total_bytes / wl.bare_bytes, "dense_fp16": 2.0 * M * K,
-                           "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad},
+                           "stored_entries": info.nnz + info.n_pad, "pads": info.n_pad,
+                           "layout": None if not wl.layout_stats else {
+                               "sub_blocks": wl.layout_stats[0],
+                               "steps_per_sub_block": wl.layout_stats[1] / max(1, wl.layout_stats[0]),
+                               "mean_groups_per_lane": wl.layout_stats[2] / 32.0 / max(1, wl.layout_stats[0]),
+                               "step_slots_per_group": 32.0 * wl.layout_stats[1] / max(1, wl.layout_stats[2])}},
         "roofline": {"bound": "hbm", "achieved": wl.total_bytes / sec_per_call / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": wl.total_bytes / sec_per_call / 1e9 / peak, "traffic": dram_traffic_per_launch(name),
                      "frac_on_bare_format_bytes": wl.bare_bytes / sec_per_call / 1e9 / peak,

@@ -352,6 +352,14 @@ int celty_fetched_bytes(const celty_matrix *m, const int32_t *idx_host, int64_t 
 int celty_stored_entries(const celty_matrix *m, const int32_t *idx_host, int64_t n, int64_t *entries);
 
 /*
+ * celty_layout_stats -- how evenly the LANE_TILE image loads the 32 lanes of a warp: the number of sub-blocks
+ * (column, slab), the steps they take in total (a sub-block takes as many steps as its fullest lane has groups of 8
+ * entries) and the groups they hold in total.  32 * steps / groups is how many step slots the kernel runs per
+ * group that exists: 1 would be perfectly even lanes.  Host-only.  Errors: CELTY_EINVAL (COLUMN handle).
+ */
+int celty_layout_stats(const celty_matrix *m, int64_t *sub_blocks, int64_t *steps, int64_t *groups);
+
+/*
  * celty_count_entries -- how many entries the format of Section 3.2 would store for a mask if its
  * runs were `run_bits` wide (1..8), whole columns, without building anything: the kept positions
  * (nnz) and the padding entries the rule inserts (a gap of g dropped rows costs floor(g / 2^run_bits)

@@ -46,6 +46,7 @@ SIGNATURES = {
     "celty_decode_device": (ctypes.c_int, [_vp, _i64, _vp, _vp, _i64, _vp, _vp]),
     "celty_fetched_bytes": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
     "celty_stored_entries": (ctypes.c_int, [_vp, _vp, _i64, ctypes.POINTER(_i64)]),
+    "celty_layout_stats": (ctypes.c_int, [_vp] + [ctypes.POINTER(_i64)] * 3),
     "celty_count_entries": (ctypes.c_int, [_vp, _i64, _i64, _i64, ctypes.c_int, ctypes.POINTER(_i64),
                                            ctypes.POINTER(_i64)]),
     "celty_last_status": (ctypes.c_int, [_vp, _vp]),
@@ -215,6 +216,12 @@ class Matrix:
         _check(load().celty_fetched_bytes(self._h, _np_ptr(idx), idx.size, ctypes.byref(s), ctypes.byref(t)),
                "celty_fetched_bytes")
         return s.value, t.value
+
+    def layout_stats(self):
+        """(sub-blocks, steps in total, groups of 8 entries in total) of the LANE_TILE image."""
+        v = [_i64() for _ in range(3)]
+        _check(load().celty_layout_stats(self._h, *[ctypes.byref(a) for a in v]), "celty_layout_stats")
+        return tuple(a.value for a in v)
 
     def stored_entries(self, idx) -> int:
         """Stored entries (kept weights + padding entries) of the listed columns."""

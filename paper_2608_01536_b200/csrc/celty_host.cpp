@@ -36,8 +36,9 @@ struct Logical {                 // one run per byte, block-major (column, tile)
 // the configured shapes, S = ceil(M / 4096) was the best or within 6% of the best slab count everywhere.
 // On very tall layers (6 slabs or more) the streaming loop dominates, and what counts there is that eight warp
 // teams fit one SM's 227 KB of shared memory (accumulator slab + two ring slots each): when the density of the
-// kept weights makes the sub-blocks too large for that at 128 local rows, one or two more slabs of fewer rows are
-// taken (measured on 28672 x 8192: 6.5% / 2.8% faster at 70% / 50% of the weights kept, no change at 30%).
+// kept weights makes the sub-blocks too large for that at 128 local rows, fewer rows per tile (in steps of 8, down
+// to 96) and correspondingly more slabs are taken: 104 rows at 70% of the weights kept, 120 at 50%, 128 at 30% on
+// 28672 x 8192 (measured: 44.4 us against 53.0 at 128 rows and 47.0 at 96; 37.1 against 37.7; no change).
 void choose_shape(int64_t M, int64_t K, double density, int tile_rows, int64_t *S_out, int32_t *R_out, int32_t *C_out)
 {
     const int64_t Q = (M + 31) / 32;                                  // groups of 32 rows
@@ -49,16 +50,16 @@ void choose_shape(int64_t M, int64_t K, double density, int tile_rows, int64_t *
         S = std::max<int64_t>(1, (M + 4095) / 4096);
         auto rows_for = [&](int64_t slabs) { return std::max<int64_t>(16, ((Q + slabs - 1) / slabs + 15) / 16 * 16); };
         auto teams_that_fit = [&](int64_t rows) {
-            const double entries = 32.0 * rows * density;             // of one sub-block, mean; + 4 sigma for the largest
-            const double largest = entries + 4.0 * std::sqrt(entries * (1.0 - density)) + 32 * 4;   // + group filling
+            const double entries = 32.0 * rows * density;             // of one sub-block, mean; + 3.5 sigma for the largest
+            const double largest = entries + 3.5 * std::sqrt(entries * (1.0 - density)) + 32 * 3.5;  // + group filling
             const double slot = std::ceil((kSubHeader + 2.5 * largest) / 128.0) * 128.0;
             const double misc = 2.0 * ((K + 31) / 32) * 4 + 17.0 * ((K + 255) / 256) * 4 + 1024;
             return (int64_t)((232448.0 - misc) / ((rows + kTileSlack) * 128.0 + 2.0 * slot + 1024.0));
         };
         R = rows_for(S);
         if (S >= 6)
-            for (int fewer = 1; fewer <= 2 && teams_that_fit(R) < 8 && R > 32; ++fewer) {
-                R -= 16;
+            for (int fewer = 1; fewer <= 4 && teams_that_fit(R) < 8 && R > 32; ++fewer) {
+                R -= 8;                                                // in steps of 8 rows: the chunk of the row map halves
                 S = (Q + R - 1) / R;
             }
     }
@@ -426,6 +427,26 @@ extern "C" int celty_stored_entries(const celty_matrix *m, const int32_t *idx, i
         e += (int64_t)m->block_ptr[(j + 1) * m->T] - (int64_t)m->block_ptr[j * m->T];
     }
     *entries = e;
+    return CELTY_OK;
+}
+
+extern "C" int celty_layout_stats(const celty_matrix *m, int64_t *sub_blocks, int64_t *steps, int64_t *groups)
+{
+    if (!m) return CELTY_EINVAL;
+    if (m->layout != CELTY_LAYOUT_LANE_TILE) return CELTY_EINVAL;
+    const uint32_t *meta = reinterpret_cast<const uint32_t *>(m->image.data());
+    const uint8_t *stream = m->image.data() + m->meta_bytes;
+    int64_t nb = 0, st = 0, gr = 0;
+    for (int64_t b = 0; b < m->K * m->S; ++b) {
+        uint32_t hw;
+        std::memcpy(&hw, stream + (size_t)meta[b] * 16 + 32, 4);      // vectors | steps << 16 (see kSubHeader)
+        ++nb;
+        st += hw >> 16;
+        gr += hw & 0xFFFFu;
+    }
+    if (sub_blocks) *sub_blocks = nb;
+    if (steps) *steps = st;
+    if (groups) *groups = gr;
     return CELTY_OK;
 }
 
