@@ -386,7 +386,10 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            2 = merge the blocks' results through per-block partial vectors summed in a fixed
  *            order (bit-reproducible) instead of adding them into y with bulk reduce-add copies,
  *            4 = force the bulk reduce-add merge, 8 = plain launch instead of a programmatic dependent
- *            launch (with which the kernel's set-up overlaps the tail of the previous kernel of the stream)
+ *            launch (with which the kernel's set-up overlaps the tail of the previous kernel of the stream),
+ *            16 = always / 32 = never run warp pairs: two warps per team that take turns at the team's
+ *            accumulator, one waiting for its next sub-block and reading its header while the other runs its
+ *            steps (by default the library pairs warps where a team has a dozen or more columns to stream)
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   cluster  fused kernel, bulk reduce-add merge: thread blocks per cluster (1, 2 or 4); the blocks of a
@@ -417,7 +420,8 @@ int celty_set_register_rows(celty_matrix *m, int32_t rows);
  * device, with the knobs of celty_set_launch applied (LANE_TILE handles; needs a CUDA device):
  *   out[0..9] = thread blocks, threads per block, dynamic shared memory (bytes), warp teams per slab,
  *   ring slots per team, thread blocks per cluster, row parts, slabs per block, ring slot size (bytes),
- *   merge (0 ordered two-stage sum, 1 bulk reduce-add).   n = capacity of out (at least 10).
+ *   merge (0 ordered two-stage sum, 1 bulk reduce-add) + 16 if warp pairs are in use.   n = capacity of out
+ *   (at least 10).
  * Errors: CELTY_EINVAL, CELTY_ECUDA.
  */
 int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n);

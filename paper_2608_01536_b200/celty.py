@@ -239,7 +239,9 @@ class Matrix:
         _check(load().celty_launch_plan(self._h, out, 10), "celty_launch_plan")
         keys = ("grid", "threads", "smem_bytes", "teams_per_slab", "ring_depth", "cluster", "row_parts",
                 "slabs_per_block", "slot_bytes", "merge")
-        return dict(zip(keys, [int(v) for v in out]))
+        plan = dict(zip(keys, [int(v) for v in out]))
+        plan["warp_pairs"], plan["merge"] = plan["merge"] >> 4, plan["merge"] & 15
+        return plan
 
     def set_register_rows(self, rows: int = 0):
         """Local rows per lane summed in registers instead of shared memory (0, 32, 64, 96 or 128)."""

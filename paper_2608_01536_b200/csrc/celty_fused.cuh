@@ -43,6 +43,7 @@ struct FusedParams {
     int M, K, R, S, C;         // rows, columns, local rows per tile, slabs, chunk of the row map (tile_row)
     int G, Sc, P, D;           // teams per slab, slabs per block, row parts, ring depth
     int cl;                    // thread blocks per cluster (1, 2 or 4); blocks of a cluster share a row part
+    int pp;                    // 1: two warps per team that take turns at the team's accumulator (see the kernel)
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // columns a team looks up per batch
     int win_cols;              // columns of the offset table a block copies into shared memory at its start
@@ -254,7 +255,7 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
 // Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
 // (which sizes the launch with .total), so that the two can never disagree.
 struct FusedSmem {
-    size_t acc, ring, bars, items, imeta, zero, keep, wrel, blk, blkw, total;
+    size_t acc, ring, bars, flag, items, imeta, zero, keep, wrel, blk, blkw, total;
 };
 
 __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
@@ -264,6 +265,7 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, 
     l.acc = off;       off += (size_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
     l.ring = off;      off += (size_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
     l.bars = off;      off += (size_t)teams * D * 8 + 8;                   // one "full" mbarrier per slot, one for the offset window
+    l.flag = off;      off += (size_t)teams * 4;                           // per team: a wait of one of its warps ran out
     off = (off + 15) / 16 * 16;
     l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
     l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
@@ -380,9 +382,17 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const int slab_words = (p.R + kTileSlack) * 32;
     // Warps [0, teams) stream columns, one warp per team; the others only help with the phases that
     // are plain data-parallel work (thresholding, clearing, storing and summing partial vectors).
+    // With pp two warps share a team: warp `team` and warp `teams + team`.  Each streams every other column of the
+    // team's share into ring slots of its own, and the two take turns at the team's accumulator: while one runs
+    // its step loop, the other waits for its next sub-block, reads the header and fetches the first groups, so the
+    // accumulator never sits idle through those latencies.  A named barrier per team hands the accumulator over.
     const int teams = p.G * p.Sc;
-    const bool streams = warp < teams;
-    const int team = streams ? warp : 0;
+    // (The partner of warp t is warp t + 8: the two sit on the same warp scheduler, which suits them, since only
+    // one of them is in its step loop at any time.)
+    const bool streams = p.pp ? (warp & 7) < teams : warp < teams;
+    const int team = streams ? (p.pp ? (warp & 7) : warp) : 0;
+    const int half = streams && p.pp ? warp >> 3 : 0;               // which of the team's two warps (0 without pp)
+    const int stride = 1 + p.pp, Dw = p.D / stride;                 // columns between a warp's own, ring slots per warp
     const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.D, p.slot_bytes, p.cap);
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
@@ -434,8 +444,9 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         }
     }
     if (tid < 4) zero_group[tid] = 0;
+    if (tid < teams) reinterpret_cast<int *>(smem + lay.flag)[tid] = 0;
     if (streams && lane == 0) {
-        for (int d = 0; d < p.D; ++d) mbar_init(smem_u32(&bars[team * p.D + d]), 1);
+        for (int d = 0; d < Dw; ++d) mbar_init(smem_u32(&bars[team * p.D + half * Dw + d]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -542,10 +553,9 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     __syncthreads();
     bool failed = false;
     // the window has had the whole thresholding pass to arrive; nobody may clear an accumulator before it has
-    if (p.win_cols > 0 && !mbar_wait_bounded(win_bar, 0, p.spin_limit)) {
-        failed = true;
-        win_n = 0;
-    }
+    if (p.win_cols > 0 && !mbar_wait_bounded(win_bar, 0, p.spin_limit)) failed = true;
+    if (p.pp) failed = __syncthreads_or(failed);                  // the two warps of a team must agree on what follows
+    if (failed) win_n = 0;
     // ---- ranks: every streaming warp turns the block counts into survivors before each block for itself, 32
     // blocks at a time (a copy per warp costs a few hundred bytes and saves a block-wide barrier behind a single
     // warp); the list is then cut into equal shares for the groups that work on different columns.
@@ -581,13 +591,19 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
         const uint32_t cell0 = slab0 + 4u * lane;
-        const uint32_t ring0 = smem_u32(ring + (size_t)team * p.D * p.slot_bytes);
-        const uint32_t bar0 = smem_u32(&bars[team * p.D]);
+        const uint32_t ring0 = smem_u32(ring + ((size_t)team * p.D + (size_t)half * Dw) * p.slot_bytes);
+        const uint32_t bar0 = smem_u32(&bars[team * p.D + half * Dw]);
+        volatile int *team_flag = reinterpret_cast<volatile int *>(smem + lay.flag) + team;
+        const int stream_threads = teams * stride * 32;
+        auto team_sync = [&]() {                                      // the warp alone, or the two warps of the team
+            if (p.pp) asm volatile("bar.sync %0, 64;" ::"r"(2 + team) : "memory");
+            else __syncwarp();
+        };
         bool zeroed = false;
         const uint32_t lt_mask = (1u << lane) - 1u;
         const uint32_t items0 = smem_u32(items);
         uint32_t issued = 0, consumed = 0;                            // copies asked for / used up by this team
-        uint32_t slot = 0, parity = 0, islot = 0;                     // consumed % D, (consumed / D) & 1, issued % D
+        uint32_t slot = 0, parity = 0, islot = 0;                     // of this warp's Dw slots: consumed % Dw, its phase, issued % Dw
         StepBuf b0, b1;                                               // pipeline registers, live across items
         const uint32_t zeros = smem_u32(zero_group);
         float racc[kRegRows > 0 ? kRegRows : 1];                      // register-held sums of local rows 0 .. kRegRows-1
@@ -598,7 +614,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         for (int rb = r_begin;; rb += p.cap) {                        // at least one trip: the teams meet at a barrier in it
             const int cnt = failed ? 0 : max(0, min(p.cap, r_end - rb));
             // ---- column of rank r: the block of keep words that holds it, then the word, then the bit
-            for (int i = lane; i < cnt; i += 32) {
+            for (int i = half * 32 + lane; i < cnt; i += 32 * stride) {
                 const int r = rb + i;
                 int j;
                 uint16_t xb;
@@ -650,8 +666,8 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             // The accumulators take the place of the window: every team has to be through with its look-ups
             // before any team clears its slab.  (Teams with more than `cap` columns come back here for their
             // later batches, and find the offsets in global memory then.)
-            if (rb == r_begin) asm volatile("bar.sync 1, %0;" ::"r"(teams * 32) : "memory");
-            else __syncwarp();
+            if (rb == r_begin) asm volatile("bar.sync 1, %0;" ::"r"(stream_threads) : "memory");
+            else team_sync();
             win_n = 0;
             if (rb + p.cap >= r_end && (cnt == 0 || s >= p.S)) break;
             if (cnt == 0 || s >= p.S) continue;
@@ -663,25 +679,33 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 bulk_load_elected(ring0 + islot * (uint32_t)p.slot_bytes, p.stream + (size_t)im.x * 16, im.y,
                                   bar0 + 8u * islot);
                 ++issued;
-                if (++islot == (uint32_t)p.D) islot = 0;
+                if (++islot == (uint32_t)Dw) islot = 0;
             };
-            for (int i = 0; i < min(cnt, p.D); ++i) issue_im(imeta[i]);
+            for (int k = 0, i = half; k < Dw && i < cnt; ++k, i += stride) issue_im(imeta[i]);
             if (!zeroed) {                                          // clear the slab while the first copies fly
                 float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
-                for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int i = half * 32 + lane; i < slab_words / 4; i += 32 * stride) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                 zeroed = true;
-                __syncwarp();
+                team_sync();
             }
-            for (int i = 0; i < cnt; ++i) {
+            for (int i = half; i < cnt; i += stride) {
                 uint32_t xbits;                                       // the column's activation: asked for before the wait
                 asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(items0 + 8u * (uint32_t)i + 4u));
-                if (!mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
+                if (!failed && !mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
                 failed = __any_sync(kFull, failed);
-                if (failed) break;                                    // the copies still in flight are awaited below
+                if (failed) {
+                    // The copies still in flight are awaited below.  A warp that gave up keeps meeting its partner at
+                    // the hand-overs of this batch, so that nobody waits for it in vain.
+                    if (!p.pp) break;
+                    if (lane == 0) *team_flag = 1;
+                    if (i > 0) team_sync();
+                    if (i + 1 < cnt) team_sync();
+                    continue;
+                }
                 const uint32_t sub = ring0 + slot * (uint32_t)p.slot_bytes;
                 // what the refill at the end of this sub-block will need, read now so that it does not wait then
-                const bool refill = i + p.D < cnt;
-                const uint2 next_im = refill ? imeta[i + p.D] : make_uint2(0u, 0u);
+                const bool refill = i + stride * Dw < cnt;
+                const uint2 next_im = refill ? imeta[i + stride * Dw] : make_uint2(0u, 0u);
                 const uint16_t xj = (uint16_t)xbits;
                 // ---- a3 + a4.  Header: groups per lane, vectors and steps (see kSubHeader).
                 uint32_t gl, hw;
@@ -693,6 +717,9 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 const uint32_t spare = cell0 + (uint32_t)p.R * 128u;
                 step_fetch(b0, gl, 0, steps, cum, lt_mask, vbase, rbase, zeros);
                 step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, zeros);
+                // nothing above touches the accumulator: here the partner hands it over (it has finished the
+                // column before this one)
+                if (p.pp && i > 0) team_sync();
                 step_decode<kRegRows>(b0, cell, spare, reg_lim);                                    // step 0
                 step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, zeros);
                 uint32_t q = 1;
@@ -725,10 +752,12 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 // every lane's reads before this point: the copy may overwrite it.
                 __syncwarp();
                 if (refill) issue_im(next_im);
+                if (p.pp && i + 1 < cnt) team_sync();                 // the accumulator goes to the partner
                 ++consumed;
-                if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
+                if (++slot == (uint32_t)Dw) { slot = 0; parity ^= 1u; }
             }
-            __syncwarp();                                         // items / imeta are rewritten by the next batch
+            team_sync();                                          // items / imeta are rewritten by the next batch
+            if (p.pp && *team_flag) failed = true;                // both warps of a team stop together
             if (failed || rb + p.cap >= r_end) break;
         }
         if (kRegRows > 0 && zeroed) {                                 // the register rows go to the slab for the merge
@@ -744,7 +773,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             // give the copies that are still in flight a last (bounded) chance to land before the block goes on
             for (; consumed < issued; ++consumed) {
                 mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit);
-                if (++slot == (uint32_t)p.D) { slot = 0; parity ^= 1u; }
+                if (++slot == (uint32_t)Dw) { slot = 0; parity ^= 1u; }
             }
             if (lane == 0) atomicOr(p.status, kStatusTimeout);
         }
@@ -924,7 +953,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
 }
 
 struct FusedPlan {
-    int G, Sc, P, D, cl, slot_bytes, cap, threads, grid, merge;
+    int G, Sc, P, D, cl, pp, slot_bytes, cap, threads, grid, merge;
     size_t smem;
 };
 

@@ -96,6 +96,8 @@ struct celty_matrix {
     uint8_t *d_ws = nullptr;
     celty::WorkspaceLayout ws{};
     int32_t grid = 0, variant = 0, groups = 0, depth = 0, cluster = 0;
+    int32_t pairs = -1;                       // fused kernel, two warps per team that take turns at its accumulator:
+                                              // -1 = library's choice, 0 = never, 1 = always
     int32_t reg_rows = 0;                     // register-accumulation study: local rows per lane summed in registers
     uint32_t spin_limit = 0;                  // bounded waits inside the kernels: 0 = the library's limit
     int32_t last_grid = 0, last_merge = -1;   // what the tickets in the workspace were last used with

@@ -522,35 +522,58 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     if (pl.Sc > 16) return CELTY_EINVAL;      // one warp per team, 16 warps per block
     pl.slot_bytes = (int)round_up((size_t)m->max_unit16 * 16, 128);
     pl.cap = 64;
-    const size_t budget = (size_t)di.max_smem_optin;
-    // Teams first (each needs its own accumulator), then as many ring slots as still fit (at least two, to
-    // keep a copy in flight).
     const int reg_rows = m->reg_rows;          // register-accumulation study: 256 threads, eight teams at most
-    const int g_cap = std::max(1, (reg_rows > 0 ? 8 : 16) / pl.Sc);
-    const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
-    const int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 4;
-    pl.G = 0;
-    for (int g = g_max; g >= 1 && pl.G == 0; --g)
-        for (int d = d_max; d >= d_min; --d)
-            if (fused_smem_bytes(m->R, (int)m->K, g, pl.Sc, d, pl.slot_bytes, pl.cap) <= budget) {
-                pl.G = g;
-                pl.D = d;
-                break;
-            }
+    const size_t budget = (size_t)di.max_smem_optin;
+    int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
+    if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
+    pl.grid = std::max(blocks, pl.P);           // any number of blocks >= P: parts may differ by one column slice
+    if (pl.grid > di.sms) return CELTY_EINVAL;
+    // Teams first (each needs its own accumulator), then as many ring slots as still fit (at least two, to
+    // keep a copy in flight).  With warp pairs (two warps take turns at a team's accumulator, each with ring slots
+    // of its own) there are eight teams at most and an even number of slots.
+    auto fit = [&](int pairs) {
+        pl.pp = pairs;
+        const int g_cap = std::max(1, ((reg_rows > 0 || pairs) ? 8 : 16) / pl.Sc);
+        const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
+        int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 4;
+        if (pairs) {
+            d_min = std::max(2, d_min + (d_min & 1));
+            d_max = std::max(d_min, d_max & ~1);
+        }
+        pl.G = 0;
+        for (int g = g_max; g >= 1 && pl.G == 0; --g)
+            for (int d = d_max; d >= d_min; --d)
+                if ((!pairs || (d & 1) == 0) &&
+                    fused_smem_bytes(m->R, (int)m->K, g, pl.Sc, d, pl.slot_bytes, pl.cap) <= budget) {
+                    pl.G = g;
+                    pl.D = d;
+                    break;
+                }
+    };
+    fit(0);
+    // Pairs pay where a team has many columns to stream (the hand-over hides the latencies at the head of every
+    // sub-block) and cost a little where it has few: measured +7-8 % at 28672 x 8192 and 8192 x 28672, +2 % at
+    // 11008 x 4096 and 13824 x 5120, -1 % at 5120 x 5120, -5 % at 4096 x 4096.  The number of survivors is not known
+    // here, so the rule goes by the columns: a dozen or more per team.
+    if (reg_rows == 0 && pl.Sc <= 8 && m->pairs != 0 && pl.G > 0) {
+        const int teams_per_part = std::max(1, pl.grid / pl.P) * std::min(pl.G, std::max(1, 8 / pl.Sc));
+        if (m->pairs > 0 || m->K / teams_per_part >= 12) {
+            const FusedPlan keep = pl;
+            fit(1);
+            if (pl.G == 0) pl = keep;
+        }
+    }
     if (pl.G == 0 && m->depth == 0 && fused_smem_bytes(m->R, (int)m->K, 1, pl.Sc, 1, pl.slot_bytes, pl.cap) <= budget) {
         pl.G = 1;
         pl.D = 1;
+        pl.pp = 0;
     }
     if (pl.G == 0) return CELTY_EINVAL;
     pl.threads = reg_rows > 0 ? 256 : 512;
     pl.smem = fused_smem_bytes(m->R, (int)m->K, pl.G, pl.Sc, pl.D, pl.slot_bytes, pl.cap);
     pl.merge = (m->merge >= 0 ? m->merge : 1);
-    int blocks = std::min(di.sms, kMaxBlocks);  // every block must be resident: they wait for one another's tickets
-    if (m->grid > 0) blocks = std::min(blocks, (int)m->grid);
-    pl.grid = std::max(blocks, pl.P);           // any number of blocks >= P: parts may differ by one column slice
-    if (pl.grid > di.sms) return CELTY_EINVAL;
-    // Clusters (bulk reduce-add merge only): pairs unless asked otherwise, as long as the grid is made of whole
-    // clusters, every row part gets at least one, and the device can hold them all at once.
+    // Clusters (bulk reduce-add merge only, on request): as long as the grid is made of whole clusters, every row
+    // part gets at least one, and the device can hold them all at once.
     pl.cl = pl.merge == 1 ? (m->cluster > 0 ? m->cluster : 1) : 1;
     while (pl.cl > 1 && (pl.grid % pl.cl != 0 || pl.grid / pl.cl < pl.P)) pl.cl >>= 1;
     *out = pl;
@@ -625,7 +648,7 @@ extern "C" int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n)
     rc = fit_clusters(&plan);
     if (rc) return rc;
     const int32_t v[10] = {plan.grid, plan.threads, (int32_t)plan.smem, plan.G, plan.D, plan.cl, plan.P, plan.Sc,
-                           plan.slot_bytes, plan.merge};
+                           plan.slot_bytes, plan.merge + 16 * plan.pp};
     for (int i = 0; i < 10; ++i) out[i] = v[i];
     return CELTY_OK;
 }
@@ -735,7 +758,7 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         fp.idx = idx; fp.val = val; fp.count = count; fp.status = status; fp.tickets = status + 2;
         fp.partials = reinterpret_cast<float *>(m->d_ws + m->ws.partial_off);
         fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.C = m->C;
-        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.cl = plan.cl;
+        fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.cl = plan.cl; fp.pp = plan.pp;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         {
             // offset window: as many columns as 32 KB (or the accumulator area, or the table) hold
