@@ -556,6 +556,8 @@ def run_knob_study(args):
         add("depth", depth, depth=depth)
     for cluster in (1, 2, 4):
         add("cluster", cluster, cluster=cluster)
+    for name_, bit in (("never", 32), ("always", 16)):              # two warps per team taking turns at its accumulator
+        add("pairs", name_, variant=bit)
     for m in mats:
         m.set_launch()
     print(json.dumps({"sweep": "knobs", "workload": name, "row_parts": int(S), "device_copies": copies,

@@ -553,11 +553,12 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     fit(0);
     // Pairs pay where a team has many columns to stream (the hand-over hides the latencies at the head of every
     // sub-block) and cost a little where it has few: measured +7-8 % at 28672 x 8192 and 8192 x 28672, +2 % at
-    // 11008 x 4096 and 13824 x 5120, -1 % at 5120 x 5120, -5 % at 4096 x 4096.  The number of survivors is not known
-    // here, so the rule goes by the columns: a dozen or more per team.
-    if (reg_rows == 0 && pl.Sc <= 8 && m->pairs != 0 && pl.G > 0) {
-        const int teams_per_part = std::max(1, pl.grid / pl.P) * std::min(pl.G, std::max(1, 8 / pl.Sc));
-        if (m->pairs > 0 || m->K / teams_per_part >= 12) {
+    // 11008 x 4096 and 13824 x 5120, -1 % at 5120 x 5120, -5 % at 4096 x 4096; and they must not cost teams (5120 x 13824
+    // runs 11 teams of one warp faster than 8 pairs).  The number of survivors is not known here, so the rule goes
+    // by the columns: a dozen or more per team, and no more than eight teams to begin with.
+    if (reg_rows == 0 && m->pairs != 0 && pl.G > 0) {
+        const int teams_per_part = std::max(1, pl.grid / pl.P) * pl.G;
+        if (m->pairs > 0 || (pl.G * pl.Sc <= 8 && m->K / teams_per_part >= 12)) {
             const FusedPlan keep = pl;
             fit(1);
             if (pl.G == 0) pl = keep;
