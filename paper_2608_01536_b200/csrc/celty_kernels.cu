@@ -556,7 +556,7 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
     // 11008 x 4096 and 13824 x 5120, -1 % at 5120 x 5120, -5 % at 4096 x 4096; and they must not cost teams (5120 x 13824
     // runs 11 teams of one warp faster than 8 pairs).  The number of survivors is not known here, so the rule goes
     // by the columns: a dozen or more per team, and no more than eight teams to begin with.
-    if (reg_rows == 0 && m->pairs != 0 && pl.G > 0) {
+    if (reg_rows == 0 && m->pairs != 0 && pl.G > 0 && pl.Sc <= 8) {             // a pair is warps t and t + 8
         const int teams_per_part = std::max(1, pl.grid / pl.P) * pl.G;
         if (m->pairs > 0 || (pl.G * pl.Sc <= 8 && m->K / teams_per_part >= 12)) {
             const FusedPlan keep = pl;
