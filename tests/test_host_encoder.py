@@ -179,3 +179,45 @@ def test_entry_count_rejects_bad_arguments():
     assert lib.celty_count_entries(p, 3, 4, 4, 4, ctypes.byref(n), None) == -1
     assert lib.celty_count_entries(p, 4, 0, 4, 4, ctypes.byref(n), None) == -1
     assert lib.celty_count_entries(p, 4, 4, 4, 4, ctypes.byref(n), None) == 0 and n.value == 16
+
+
+def test_clone_is_an_independent_copy():
+    M, K = 300, 40
+    W = synth.weights(3, M, K)
+    mask = synth.mask_bernoulli(3, M, K, 0.4)
+    a = celty.Matrix(W, mask)
+    b = a.clone()
+    ia, ib = a.info(), b.info()
+    assert (ia.nnz, ia.n_pad, ia.tile_rows, ia.layout) == (ib.nnz, ib.n_pad, ib.tile_rows, ib.layout)
+    ha, hb = a.host_image(), b.host_image()
+    assert ha[1] == hb[1] and np.array_equal(ha[0], hb[0])
+    del a                                                   # the copy owns its memory
+    for j in (0, 7, K - 1):
+        rows, vals, runs, pad = b.decode_host(j)
+        kept = np.flatnonzero(mask[:, j])
+        assert np.array_equal(np.sort(rows[pad == 0]), kept)
+
+
+def test_stored_entries_and_layout_statistics_against_the_oracle():
+    """Stored entries of a set of columns and the step / group totals of the lane-tile image, from the oracle's
+    encoder on the row-permuted matrix: a sub-block (column, slab) takes as many steps as its fullest lane has groups
+    of 8 entries."""
+    M, K = 2100, 37
+    W = synth.weights(8, M, K)
+    mask = synth.mask_bernoulli(8, M, K, 0.45)
+    m = celty.Matrix(W, mask)
+    S, R, C = m.row_map()
+    Wp, mp, _ = permute_for_lane_tiles(W, mask, S, R, C)
+    ptr = orc.rlc_count(mp, 4, R)                               # entries before (column, tile); 32 * S tiles per column
+    n = np.diff(ptr).reshape(K, 32 * S)
+    cols = np.array([0, 5, 6, 36], np.int32)
+    assert m.stored_entries(cols) == int(n[cols].sum())
+    groups = (n + 7) // 8
+    per_sub = groups.reshape(K, S, 32)
+    nb, steps, total_groups = m.layout_stats()
+    assert nb == K * S
+    assert steps == int(per_sub.max(axis=2).sum())
+    assert total_groups == int(groups.sum())
+    col = celty.Matrix(W, mask, layout=celty.LAYOUT_COLUMN)
+    with pytest.raises(celty.CeltyError):
+        col.layout_stats()
