@@ -762,6 +762,57 @@ def run_regsplit_study(args):
     print(json.dumps({"sweep": "regsplit", "points": points}))
 
 
+def run_batch_study(args):
+    """Small batches (Sections 2.2-2.3 place the method against SpMM kernels that need N >= 8): microseconds per
+    batch of N activation vectors through celty_spmspv_batch (union of the surviving columns, N accumulators per
+    row; the simple two-launch kernels), beside N calls of the single-vector kernel and the dense cuBLAS FP16 GEMM
+    on the same weights, under the same rotation."""
+    import torch
+    from paper_2608_01536_b200 import build as lib_build, celty
+    lib_build.build()
+    celty.load()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    points = []
+    for name in ("llama7b_attn_4096x4096_s50_a50", "llama7b_gateup_11008x4096_s50_a50"):
+        M, K, s, family, dist_name, d_a, cfg = WORKLOADS[name]
+        W, mask = make_layer(name, 0)
+        first = celty.Matrix(W, mask, device=dev)
+        copies = int(np.ceil(2.5 * l2 / first.device_bytes()[0])) + 1
+        mats = [first] + [first.clone(device=dev) for _ in range(copies - 1)]
+        Wd = [torch.from_numpy(np.where(mask != 0, W, np.float16(0))).to(dev) for _ in range(min(copies, int(np.ceil(2.5 * l2 / (2 * M * K))) + 1))]
+        for N in (1, 2, 4, 8):
+            X = np.stack([make_x(name, 10 * c + n)[0] for c in range(copies) for n in range(N)]).reshape(copies, N, K)
+            tau = make_x(name, 0)[1]
+            xs = [torch.from_numpy(X[c]).to(dev) for c in range(copies)]
+            ys = [torch.empty(N, M, dtype=torch.float32, device=dev) for _ in range(copies)]
+            yd = torch.empty(M, N, dtype=torch.float16, device=dev)
+
+            def timed(calls):
+                for f in calls:
+                    f()
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for f in calls:
+                        f()
+                g.replay()
+                reps = max(3, -(-args.sweep_calls // len(calls)))
+                return float(np.median(timed_regions(torch, g.replay, reps, min_total_s=0.05))) * 1e3 / (reps * len(calls))
+            us_batch = timed([(lambda c=c: mats[c].spmspv_batch(xs[c], tau, ys[c])) for c in range(copies)])
+            us_single = timed([(lambda c=c, n=n: mats[c].spmspv(xs[c][n], tau, ys[c][n])) for c in range(copies) for n in range(N)]) * N
+            us_gemm = timed([(lambda c=c: torch.mm(Wd[c % len(Wd)], xs[c].t(), out=yd)) for c in range(copies)])
+            keep = [np.abs(X[c].astype(np.float32)) > np.float32(tau) for c in range(copies)]
+            points.append({"workload": name, "N": N, "us_per_batch": us_batch, "us_N_single_calls": us_single,
+                           "us_cublas_gemm": us_gemm,
+                           "union_density": float(np.mean([k.any(axis=0).mean() for k in keep])),
+                           "activation_density": float(np.mean([k.mean() for k in keep]))})
+            print(json.dumps(points[-1]), file=sys.stderr, flush=True)
+        del mats, first, Wd
+    print(json.dumps({"sweep": "batch", "points": points}))
+
+
 def run_celty(args):
     import torch
     import torch.distributed as dist
@@ -966,7 +1017,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-secondary", action="store_true", help="skip the second, labelled workload")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
-    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS) + ["format", "knobs", "regsplit"],
+    ap.add_argument("--sweep", default="", choices=[""] + sorted(SWEEPS) + ["format", "knobs", "regsplit", "batch"],
                     help="time every point of a configured sweep; format = compression study on the host; "
                          "knobs = launch-parameter study of --workload")
     ap.add_argument("--sweep-calls", type=int, default=600, help="calls timed per sweep point (at least)")
@@ -977,6 +1028,8 @@ def main():
         run_knob_study(args)
     elif args.sweep == "regsplit":
         run_regsplit_study(args)
+    elif args.sweep == "batch":
+        run_batch_study(args)
     elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
