@@ -389,7 +389,11 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            launch (with which the kernel's set-up overlaps the tail of the previous kernel of the stream),
  *            16 = always / 32 = never run warp pairs: two warps per team that take turns at the team's
  *            accumulator, one waiting for its next sub-block and reading its header while the other runs its
- *            steps (by default the library pairs warps where a team has a dozen or more columns to stream)
+ *            steps (by default the library pairs warps where a team has a dozen or more columns to stream),
+ *            64 = never share a thread block between row parts.  (By default, with the bulk reduce-add merge and
+ *            no clusters: when the blocks do not divide by the row parts and the blocks left over can be shared
+ *            evenly, each of them serves several parts with correspondingly fewer teams per part, instead of
+ *            giving some parts one block more than others, which would leave those blocks idle at the end.)
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   cluster  fused kernel, bulk reduce-add merge: thread blocks per cluster (1, 2 or 4); the blocks of a
@@ -420,8 +424,8 @@ int celty_set_register_rows(celty_matrix *m, int32_t rows);
  * device, with the knobs of celty_set_launch applied (LANE_TILE handles; needs a CUDA device):
  *   out[0..9] = thread blocks, threads per block, dynamic shared memory (bytes), warp teams per slab,
  *   ring slots per team, thread blocks per cluster, row parts, slabs per block, ring slot size (bytes),
- *   merge (0 ordered two-stage sum, 1 bulk reduce-add) + 16 if warp pairs are in use.   n = capacity of out
- *   (at least 10).
+ *   merge (0 ordered two-stage sum, 1 bulk reduce-add) + 16 if warp pairs are in use + 256 x the number of row
+ *   parts a left-over block serves (1 = blocks are not shared between parts).   n = capacity of out (at least 10).
  * Errors: CELTY_EINVAL, CELTY_ECUDA.
  */
 int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n);

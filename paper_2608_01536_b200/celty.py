@@ -240,7 +240,8 @@ class Matrix:
         keys = ("grid", "threads", "smem_bytes", "teams_per_slab", "ring_depth", "cluster", "row_parts",
                 "slabs_per_block", "slot_bytes", "merge")
         plan = dict(zip(keys, [int(v) for v in out]))
-        plan["warp_pairs"], plan["merge"] = plan["merge"] >> 4, plan["merge"] & 15
+        plan["parts_per_spare_block"] = plan["merge"] >> 8
+        plan["warp_pairs"], plan["merge"] = (plan["merge"] >> 4) & 1, plan["merge"] & 15
         return plan
 
     def set_register_rows(self, rows: int = 0):

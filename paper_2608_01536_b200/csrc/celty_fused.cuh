@@ -44,6 +44,12 @@ struct FusedParams {
     int G, Sc, P, D;           // teams per slab, slabs per block, row parts, ring depth
     int cl;                    // thread blocks per cluster (1, 2 or 4); blocks of a cluster share a row part
     int pp;                    // 1: two warps per team that take turns at the team's accumulator (see the kernel)
+    // mix >= 2 (bulk reduce-add merge without clusters): the gridDim mod P blocks that are left when every row part
+    // has floor(gridDim / P) blocks are not given to the first parts (which would then finish early, one slice
+    // ahead of the others); each of them serves mix = P / (gridDim mod P) consecutive parts instead, with G / mix
+    // teams per slab, so that every part is shared by the same number of teams.  units_inv then holds
+    // floor(2^32 / (floor(gridDim / P) * G + G / mix)).
+    int mix;
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // columns a team looks up per batch
     int win_cols;              // columns of the offset table a block copies into shared memory at its start
@@ -409,12 +415,25 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     // their accumulators before anything goes to y).  The number of clusters need not be a multiple of P: the
     // first (clusters mod P) parts then have one cluster more than the others.
     const int crank = blockIdx.x % p.cl, cid = blockIdx.x / p.cl, nclusters = gridDim.x / p.cl;
-    const int part = cid % p.P;
-    const bool long_part = part < nclusters % p.P;
+    int part = cid % p.P;
+    const bool long_part = p.mix < 2 && part < nclusters % p.P;
     const int nK = p.cl * (nclusters / p.P + (long_part ? 1 : 0));
     const int kslice = (cid / p.P) * p.cl + crank;
-    const int g = team / p.Sc, sl = team - g * p.Sc;
-    const int s = part * p.Sc + sl;                               // this team's slab; may be >= S (idle)
+    // G teams per slab and Sc slabs in this block; unit0 = this block's first team among the `units` teams that
+    // share the survivor list of its part(s)
+    int G = p.G, Sc = p.Sc, unit0 = kslice * p.G, units = nK * p.G;
+    if (p.mix >= 2) {
+        const int nfull = (int)gridDim.x / p.P;
+        units = nfull * p.G + p.G / p.mix;
+        if ((int)blockIdx.x >= nfull * p.P) {                     // one of the blocks that serve several parts
+            G = p.G / p.mix;
+            Sc = p.Sc * p.mix;
+            part = (int)blockIdx.x - nfull * p.P;                 // counted in groups of mix parts
+            unit0 = nfull * p.G;
+        }
+    }
+    const int g = team / Sc, sl = team - g * Sc;
+    const int s = part * Sc + sl;                                 // this team's slab; may be >= S (idle)
 
     // Programmatic dependent launch: let the next kernel of the stream be scheduled as this one's blocks retire,
     // and do everything that touches neither the caller's vectors nor the workspace (warming L2 with the offset
@@ -428,7 +447,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const uint32_t *win = reinterpret_cast<const uint32_t *>(smem + lay.acc);
     int win_w0 = 0, win_n = 0;                                     // first table word in the window, words in it
     if (p.win_cols > 0) {
-        const int mid = (int)(((int64_t)(2 * kslice + 1) * p.K) / (2 * nK));
+        const int mid = (int)(((int64_t)(2 * unit0 + G) * p.K) / (2 * units));
         const int c0 = max(0, min(p.K - p.win_cols, mid - p.win_cols / 2));
         win_w0 = (c0 * p.S) & ~3;
         win_n = min(((c0 + p.win_cols) * p.S + 1 - win_w0 + 3) & ~3, ((p.K * p.S + 1 + 3) & ~3) - win_w0);
@@ -584,10 +603,10 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     if (streams) {
         // team u of nK * G owns n / units ranks, the first n mod units teams one more.  n / units without a
         // division: units_inv = floor(2^32 / units) gives a quotient that is at most one too small
-        const uint32_t units = (uint32_t)(nK * p.G), units_inv = long_part ? p.units_inv_long : p.units_inv;
-        uint32_t share = __umulhi((uint32_t)n_surv, units_inv), extra = (uint32_t)n_surv - share * units;
-        if (extra >= units) { ++share; extra -= units; }
-        const int u = kslice * p.G + g;
+        const uint32_t units_inv = long_part ? p.units_inv_long : p.units_inv;
+        uint32_t share = __umulhi((uint32_t)n_surv, units_inv), extra = (uint32_t)n_surv - share * (uint32_t)units;
+        if (extra >= (uint32_t)units) { ++share; extra -= (uint32_t)units; }
+        const int u = unit0 + g;
         const int r_begin = u * (int)share + min(u, (int)extra), r_end = r_begin + (int)share + (u < (int)extra ? 1 : 0);
         const uint32_t slab0 = smem_u32(acc + (size_t)team * slab_words);
         const uint32_t cell0 = slab0 + 4u * lane;
@@ -802,13 +821,13 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         }
         __syncwarp();
         // add the G accumulators of every slab into the first one
-        const int group_words = p.Sc * slab_words;
-        if (p.G > 1) {
+        const int group_words = Sc * slab_words;
+        if (G > 1) {
             float4 *acc4 = reinterpret_cast<float4 *>(acc);
             const int group4 = group_words / 4;
             for (int q4 = tid; q4 < group4; q4 += nthreads) {
                 float4 v = acc4[q4];
-                for (int gg = 1; gg < p.G; ++gg) {
+                for (int gg = 1; gg < G; ++gg) {
                     const float4 t = acc4[(size_t)gg * group4 + q4];
                     v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
                 }
@@ -816,7 +835,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             }
         }
         const int seg = p.S == 1 ? 16 : p.C, nseg = (p.R + seg - 1) / seg, seg4 = seg * 8;
-        const int owned = (p.Sc * nseg - crank + p.cl - 1) / p.cl;   // segments crank, crank + cl, ...
+        const int owned = (Sc * nseg - crank + p.cl - 1) / p.cl;   // segments crank, crank + cl, ...
         if (p.cl > 1) {
             cluster_sync();                                         // the peers' sums are complete
             for (int t = tid; t < owned * seg4; t += nthreads) {
@@ -840,7 +859,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         {
             for (int o = tid; o < owned; o += nthreads) {
                 const int sg = crank + p.cl * o;
-                const int fsl = sg / nseg, k = sg - fsl * nseg, sfull = part * p.Sc + fsl;
+                const int fsl = sg / nseg, k = sg - fsl * nseg, sfull = part * Sc + fsl;
                 if (sfull >= p.S) continue;
                 const int i0 = k * seg, i1 = min(p.R, i0 + seg);
                 const int64_t row0 = tile_row(p.S, p.C, sfull, 0, i0);
@@ -953,7 +972,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
 }
 
 struct FusedPlan {
-    int G, Sc, P, D, cl, pp, slot_bytes, cap, threads, grid, merge;
+    int G, Sc, P, D, cl, pp, mix, slot_bytes, cap, threads, grid, merge;
     size_t smem;
 };
 

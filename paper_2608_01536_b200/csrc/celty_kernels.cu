@@ -616,8 +616,7 @@ int max_active_clusters(int cl, size_t smem, int threads, int *out)
     return CELTY_OK;
 }
 
-// fall back to smaller clusters while the device cannot hold the whole grid of them at once
-int fit_clusters(FusedPlan *plan)
+int fit_clusters_only(FusedPlan *plan)
 {
     while (plan->cl > 1) {
         int fit = 0;
@@ -628,6 +627,21 @@ int fit_clusters(FusedPlan *plan)
         while (plan->cl > 1 && (plan->grid % plan->cl != 0 || plan->grid / plan->cl < plan->P)) plan->cl >>= 1;
     }
     return CELTY_OK;
+}
+
+// fall back to smaller clusters while the device cannot hold the whole grid of them at once; then, without
+// clusters, decide whether the blocks that are left over when the grid is dealt to the row parts serve several
+// parts each (FusedParams::mix): only where they can be shared evenly
+int fit_clusters(const celty_matrix *m, FusedPlan *plan)
+{
+    const int rc = fit_clusters_only(plan);
+    plan->mix = 1;
+    const int left = plan->grid % plan->P;
+    if (rc == CELTY_OK && plan->cl == 1 && plan->merge == 1 && m->mix != 0 && left > 0 && plan->P % left == 0) {
+        const int mix = plan->P / left;
+        if (plan->G % mix == 0 && plan->Sc * mix <= 16) plan->mix = mix;
+    }
+    return rc;
 }
 
 }  // namespace
@@ -646,10 +660,10 @@ extern "C" int celty_launch_plan(const celty_matrix *m, int32_t *out, int32_t n)
     if (rc) return rc;
     rc = ensure_smem(k_spmspv_fused<false, 0>, plan.smem, g_granted_fused);
     if (rc) return rc;
-    rc = fit_clusters(&plan);
+    rc = fit_clusters(m, &plan);
     if (rc) return rc;
     const int32_t v[10] = {plan.grid, plan.threads, (int32_t)plan.smem, plan.G, plan.D, plan.cl, plan.P, plan.Sc,
-                           plan.slot_bytes, plan.merge + 16 * plan.pp};
+                           plan.slot_bytes, plan.merge + 16 * plan.pp + 256 * plan.mix};
     for (int i = 0; i < 10; ++i) out[i] = v[i];
     return CELTY_OK;
 }
@@ -731,7 +745,7 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
              : m->reg_rows == 128 ? ensure_smem(k_spmspv_fused<false, 128>, plan.smem, g_granted_reg[3])
                                   : ensure_smem(k_spmspv_fused<false, 0>, plan.smem, g_granted_fused);
         if (rc) return rc;
-        rc = fit_clusters(&plan);
+        rc = fit_clusters(m, &plan);
         if (rc) return rc;
         FusedParams fp{};
         if (list) {
@@ -760,6 +774,7 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         fp.partials = reinterpret_cast<float *>(m->d_ws + m->ws.partial_off);
         fp.M = (int)m->M; fp.K = (int)m->K; fp.R = m->R; fp.S = (int)m->S; fp.C = m->C;
         fp.G = plan.G; fp.Sc = plan.Sc; fp.P = plan.P; fp.D = plan.D; fp.cl = plan.cl; fp.pp = plan.pp;
+        fp.mix = plan.mix;
         fp.slot_bytes = plan.slot_bytes; fp.cap = plan.cap;
         {
             // offset window: as many columns as 32 KB (or the accumulator area, or the table) hold
@@ -771,7 +786,8 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         fp.spin_limit = m->spin_limit ? m->spin_limit : kSpinLimit;
         auto inverse = [](uint64_t units) { return units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / units); };
         const int nclusters = plan.grid / plan.cl;
-        fp.units_inv = inverse((uint64_t)plan.cl * std::max(1, nclusters / plan.P) * plan.G);
+        fp.units_inv = plan.mix >= 2 ? inverse((uint64_t)(plan.grid / plan.P) * plan.G + plan.G / plan.mix)
+                                     : inverse((uint64_t)plan.cl * std::max(1, nclusters / plan.P) * plan.G);
         fp.units_inv_long = inverse((uint64_t)plan.cl * (nclusters / plan.P + 1) * plan.G);
         // the tickets count blocks of one launch shape: start them over when the shape changes
         if (m->last_grid != plan.grid || m->last_merge != plan.merge) {
