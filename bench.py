@@ -558,6 +558,7 @@ def run_knob_study(args):
         add("cluster", cluster, cluster=cluster)
     for name_, bit in (("never", 32), ("always", 16)):              # two warps per team taking turns at its accumulator
         add("pairs", name_, variant=bit)
+    add("spare_blocks", "not shared", variant=64)                  # left-over blocks given whole to the first row parts
     for m in mats:
         m.set_launch()
     print(json.dumps({"sweep": "knobs", "workload": name, "row_parts": int(S), "device_copies": copies,
