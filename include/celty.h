@@ -390,10 +390,11 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            16 = always / 32 = never run warp pairs: two warps per team that take turns at the team's
  *            accumulator, one waiting for its next sub-block and reading its header while the other runs its
  *            steps (by default the library pairs warps where a team has a dozen or more columns to stream),
- *            64 = never share a thread block between row parts.  (By default, with the bulk reduce-add merge and
- *            no clusters: when the blocks do not divide by the row parts and the blocks left over can be shared
- *            evenly, each of them serves several parts with correspondingly fewer teams per part, instead of
- *            giving some parts one block more than others, which would leave those blocks idle at the end.)
+ *            64 = never / 128 = wherever possible share a thread block between row parts.  (With the bulk
+ *            reduce-add merge and no clusters: when the blocks do not divide by the row parts and the blocks left
+ *            over can be shared evenly, each of them can serve several parts with correspondingly fewer teams per
+ *            part, instead of giving some parts one block more than others, which leaves those blocks idle at the
+ *            end.  By default the library does so where the parts have few enough blocks each for that to pay.)
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   cluster  fused kernel, bulk reduce-add merge: thread blocks per cluster (1, 2 or 4); the blocks of a

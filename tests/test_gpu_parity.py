@@ -228,18 +228,18 @@ def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows, spb
                                                       (14336, 257, 56, 148, 2), (11008, 96, 0, 0, 1)])
 def test_spare_blocks_shared_between_row_parts(M, K, tile_rows, grid, expect):
     """Where the blocks do not divide by the row parts, the blocks left over serve several parts each (with fewer
-    teams per part) when that can be done evenly; variant bit 64 switches it off.  Integer data: both must equal
-    the fp64 definition bit for bit, list included."""
+    teams per part) when that can be done evenly (variant bit 128: wherever it can, 64: never, neither: where it
+    pays).  Integer data: every setting must equal the fp64 definition bit for bit, list included."""
     W = synth.integer_weights(M + K, M, K)
     mask = synth.mask_bernoulli(M + K, M, K, 0.5)
     x = synth.integer_activations(M + K, K)
     tau = synth.threshold_for_density(x, 0.6)
     m = _matrix(W, mask, (celty.LAYOUT_LANE_TILE, 0), tile_rows, 0)
     oi, ov, _ = orc.compact(x, tau)
-    for variant in (0, 64, 16, 32):
+    for variant in (0, 128, 64, 16 + 128, 32 + 128):
         m.set_launch(grid=grid, variant=variant)
         plan = m.launch_plan()
-        if variant == 0 and plan["teams_per_slab"] % max(1, expect) == 0 and plan["cluster"] == 1:
+        if variant & 128 and plan["teams_per_slab"] % max(1, expect) == 0 and plan["cluster"] == 1:
             assert plan["parts_per_spare_block"] == expect, plan
         if variant == 64:
             assert plan["parts_per_spare_block"] == 1, plan
@@ -272,7 +272,7 @@ def test_random_shapes_and_options(case):
         return
     grid, groups, depth, cluster = (int(rng.choice([0, 0, 1, 5, 40, 148])), int(rng.choice([0, 0, 1, 3])),
                                     int(rng.choice([0, 0, 1, 3])), int(rng.choice([0, 1, 2, 4])))
-    variant = int(rng.choice([0, 0, 2, 8, 16, 24, 32, 64, 80]))
+    variant = int(rng.choice([0, 0, 2, 8, 16, 24, 32, 64, 128, 144]))
     m.set_launch(grid=grid, variant=variant, groups=groups, depth=depth, cluster=cluster)
     _check_y(_run(m, x, tau), W, mask, x, tau)
     idx, val = m.last_compaction()
