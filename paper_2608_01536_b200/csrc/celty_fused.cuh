@@ -24,9 +24,11 @@
 //       thresholded list (fused_epilogue), once a second ticket shows that every block's adds are done.
 //
 // Rows are split over P parts of Sc slabs each, columns over the blocks of a part and, inside a block, over
-// G teams per slab; a team = one warp with its own accumulator slab.  Every block must be resident at once
-// (grid <= SM count) because of the tickets.  All waits are bounded: when one runs out the kernel sets kStatusTimeout in the
-// status word and carries on to a clean exit.
+// G teams per slab; a team = one warp (or, with pp, two warps that take turns) with its own accumulator slab.
+// Blocks that are left over when the grid does not divide by P may serve several parts each with fewer teams per
+// part (FusedParams::mix).  Every block must be resident at once (grid <= SM count) because of the tickets.  All
+// waits are bounded: when one runs out the kernel sets kStatusTimeout in the status word and carries on to a clean
+// exit.
 
 struct FusedParams {
     const uint32_t *meta;      // [K*S + 1] offset/16 of sub-block (j, s) in the stream
