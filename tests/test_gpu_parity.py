@@ -255,7 +255,7 @@ def test_random_shapes_and_options(case):
     """Seeded draws (forty unless CELTY_RANDOM_CASES says otherwise) of shape, densities, tile rows, slabs per
     block and launch knobs on the fused path."""
     rng = np.random.default_rng(5000 + case)
-    M = int(rng.choice([1, 7, 31, 32, 33, 100, 255, 777, 2048, 5000, 9001]))
+    M = int(rng.choice([1, 7, 31, 32, 33, 100, 255, 777, 2048, 5000, 9001, 14000, 28672]))
     K = int(rng.choice([1, 5, 8, 31, 32, 33, 64, 200, 513, 1500]))
     d_w = float(rng.choice([0.02, 0.2, 0.5, 0.8, 1.0]))
     d_a = float(rng.choice([0.05, 0.3, 0.5, 0.9, 1.0]))
