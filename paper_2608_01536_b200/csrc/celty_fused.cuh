@@ -104,9 +104,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// a / b for 0 <= a < 2^16 and 0 < b < 2^7 through one approximate float division (exact for such operands: the
+// quotient of (a + 0.5) is at least 2^-8 away from every integer, far more than the division's error): the block
+// and team indices of the kernel are made of a dozen such quotients, and an integer division is 25 instructions
+// of code that a block runs once.
+__device__ __forceinline__ int idiv_small(int a, int b)
+{
+    return (int)__fdividef((float)a + 0.5f, (float)b);
+}
+
 // Wait for a phase of an mbarrier with an iteration limit; false = gave up.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit)
 {
+#pragma unroll 1
     for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 256) __nanosleep(128);
@@ -295,6 +305,20 @@ __device__ __forceinline__ uint32_t swiglu_half_bits(float gate, float up)
     return (uint32_t)__half_as_ushort(__float2half_rn(gate / (1.f + expf(-gate)) * up));
 }
 
+// The group of 8 activations that the end of x cuts short (K not a multiple of 8), zero-filled.  Out of line: one
+// thread of a block needs it, if any, and the thresholding pass is unrolled four times around the call.
+__device__ __noinline__ uint4 ragged_group(const uint16_t *x, int K, int q)
+{
+    uint32_t h[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t lo = (8 * q + 2 * k < K) ? x[8 * q + 2 * k] : 0u;
+        const uint32_t hi = (8 * q + 2 * k + 1 < K) ? x[8 * q + 2 * k + 1] : 0u;
+        h[k] = lo | (hi << 16);
+    }
+    return make_uint4(h[0], h[1], h[2], h[3]);
+}
+
 struct EpilogueArgs {
     const float *y;
     uint32_t *tickets, *status;
@@ -379,9 +403,18 @@ __device__ __noinline__ void fused_epilogue(const EpilogueArgs p)
 // split of Section 6.4): the first kRegRows local rows of every lane are summed in registers across the team's
 // columns and written to the accumulator slab once, at the end.  Those builds run 256 threads per block (eight
 // teams at most), which is what leaves a thread room for up to 128 more registers.
-template <bool kExtras, int kRegRows>
+// kLean > 0 are the builds for the library's default launch (bulk reduce-add merge, no clusters; 1: one warp per
+// team, 2: warp pairs): the code of the options they do not have is not merely skipped but absent.  A block runs
+// most of this kernel's code once per call, from an instruction cache that a call's worth of code overflows, so a
+// taken branch over code that is not run costs a trip to L2 (250 cycles and more, measured with stand-alone loops:
+// a cliff at about 24 KB of code touched per launch); what falls through in sequence is prefetched and costs
+// nothing.
+template <bool kExtras, int kRegRows, int kLean = 0>
 __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(const FusedParams p)
 {
+    const int pp = kLean ? (kLean == 2 ? 1 : 0) : p.pp;
+    const int merge = kLean ? 1 : p.merge;
+    const int cl = kLean ? 1 : p.cl;
     extern __shared__ __align__(128) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x, nwarps = nthreads >> 5;
     // the warp index through a shuffle: the compiler then knows that it (and every team, slab and loop bound
@@ -397,10 +430,10 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const int teams = p.G * p.Sc;
     // (The partner of warp t is warp t + 8: the two sit on the same warp scheduler, which suits them, since only
     // one of them is in its step loop at any time.)
-    const bool streams = p.pp ? (warp & 7) < teams : warp < teams;
-    const int team = streams ? (p.pp ? (warp & 7) : warp) : 0;
-    const int half = streams && p.pp ? warp >> 3 : 0;               // which of the team's two warps (0 without pp)
-    const int stride = 1 + p.pp, Dw = p.D / stride;                 // columns between a warp's own, ring slots per warp
+    const bool streams = pp ? (warp & 7) < teams : warp < teams;
+    const int team = streams ? (pp ? (warp & 7) : warp) : 0;
+    const int half = streams && pp ? warp >> 3 : 0;               // which of the team's two warps (0 without pp)
+    const int stride = 1 + pp, Dw = p.D / stride;                 // columns between a warp's own, ring slots per warp
     const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.D, p.slot_bytes, p.cap);
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
@@ -416,25 +449,27 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     // Row part and column slice of this block.  The blocks of a cluster work on the same row part (they add
     // their accumulators before anything goes to y).  The number of clusters need not be a multiple of P: the
     // first (clusters mod P) parts then have one cluster more than the others.
-    const int crank = blockIdx.x % p.cl, cid = blockIdx.x / p.cl, nclusters = gridDim.x / p.cl;
-    int part = cid % p.P;
-    const bool long_part = p.mix < 2 && part < nclusters % p.P;
-    const int nK = p.cl * (nclusters / p.P + (long_part ? 1 : 0));
-    const int kslice = (cid / p.P) * p.cl + crank;
+    const int cl_shift = cl >> 1;                                   // cl is 1, 2 or 4
+    const int crank = blockIdx.x & (cl - 1), cid = blockIdx.x >> cl_shift, nclusters = gridDim.x >> cl_shift;
+    const int cpart = idiv_small(cid, p.P), clusters_per_part = idiv_small(nclusters, p.P);
+    int part = cid - cpart * p.P;
+    const bool long_part = p.mix < 2 && part < nclusters - clusters_per_part * p.P;
+    const int nK = cl * (clusters_per_part + (long_part ? 1 : 0));
+    const int kslice = cpart * cl + crank;
     // G teams per slab and Sc slabs in this block; unit0 = this block's first team among the `units` teams that
     // share the survivor list of its part(s)
     int G = p.G, Sc = p.Sc, unit0 = kslice * p.G, units = nK * p.G;
     if (p.mix >= 2) {
-        const int nfull = (int)gridDim.x / p.P;
-        units = nfull * p.G + p.G / p.mix;
+        const int nfull = clusters_per_part;                      // (no clusters with mix)
+        units = nfull * p.G + idiv_small(p.G, p.mix);
         if ((int)blockIdx.x >= nfull * p.P) {                     // one of the blocks that serve several parts
-            G = p.G / p.mix;
+            G = idiv_small(p.G, p.mix);
             Sc = p.Sc * p.mix;
             part = (int)blockIdx.x - nfull * p.P;                 // counted in groups of mix parts
             unit0 = nfull * p.G;
         }
     }
-    const int g = team / Sc, sl = team - g * Sc;
+    const int g = idiv_small(team, Sc), sl = team - g * Sc;
     const int s = part * Sc + sl;                                 // this team's slab; may be >= S (idle)
 
     // Programmatic dependent launch: let the next kernel of the stream be scheduled as this one's blocks retire,
@@ -449,7 +484,8 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const uint32_t *win = reinterpret_cast<const uint32_t *>(smem + lay.acc);
     int win_w0 = 0, win_n = 0;                                     // first table word in the window, words in it
     if (p.win_cols > 0) {
-        const int mid = (int)(((int64_t)(2 * unit0 + G) * p.K) / (2 * units));
+        // the middle of the block's share of the columns, if the survivors were spread evenly (a float will do)
+        const int mid = (int)((float)(2 * unit0 + G) * (float)p.K / (float)(2 * units));
         const int c0 = max(0, min(p.K - p.win_cols, mid - p.win_cols / 2));
         win_w0 = (c0 * p.S) & ~3;
         win_n = min(((c0 + p.win_cols) * p.S + 1 - win_w0 + 3) & ~3, ((p.K * p.S + 1 + 3) & ~3) - win_w0);
@@ -467,6 +503,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     if (tid < 4) zero_group[tid] = 0;
     if (tid < teams) reinterpret_cast<int *>(smem + lay.flag)[tid] = 0;
     if (streams && lane == 0) {
+#pragma unroll 1
         for (int d = 0; d < Dw; ++d) mbar_init(smem_u32(&bars[team * p.D + half * Dw + d]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -475,8 +512,9 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     uint32_t y_ticket = 0;
     // Bulk reduce-add merge: the adds at the end need a cleared y.  The last warp clears this block's share
     // and announces it right away, so that the fence and the ticket overlap the loads of a1.
-    if (p.merge == 1 && warp == nwarps - 1) {
+    if (merge == 1 && warp == nwarps - 1) {
         const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
+#pragma unroll 1
         for (int i = r0 + lane; i < r1; i += 32) p.y[i] = 0.f;
         if (kExtras && p.ep_kind == 2 && blockIdx.x == 0 && lane == 0) *p.ep_count = 0;   // appended to after the merge
         __syncwarp();
@@ -497,6 +535,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const bool from_list = kExtras && p.list_count != nullptr;    // a1 was done by whoever produced the activations
     if (!from_list) {
         const __half2 tau2 = __half2half2(__float2half_rd(p.tau));
+#pragma unroll 1
         for (int w0 = 0; w0 < nwords; w0 += nthreads) {             // the same trip count for every thread
             const int w = w0 + tid;
             uint32_t word = 0;
@@ -539,12 +578,8 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                         const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p.x + 8 * q));
                         h[c][0] = v.x; h[c][1] = v.y; h[c][2] = v.z; h[c][3] = v.w;
                     } else if (q < ngroups) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const uint32_t lo = (8 * q + 2 * k < p.K) ? p.x[8 * q + 2 * k] : 0u;
-                            const uint32_t hi = (8 * q + 2 * k + 1 < p.K) ? p.x[8 * q + 2 * k + 1] : 0u;
-                            h[c][k] = lo | (hi << 16);
-                        }
+                        const uint4 v = ragged_group(p.x, p.K, q);     // the one group that K cuts short
+                        h[c][0] = v.x; h[c][1] = v.y; h[c][2] = v.z; h[c][3] = v.w;
                     }
                 }
 #pragma unroll
@@ -575,7 +610,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     bool failed = false;
     // the window has had the whole thresholding pass to arrive; nobody may clear an accumulator before it has
     if (p.win_cols > 0 && !mbar_wait_bounded(win_bar, 0, p.spin_limit)) failed = true;
-    if (p.pp) failed = __syncthreads_or(failed);                  // the two warps of a team must agree on what follows
+    if (pp) failed = __syncthreads_or(failed);                  // the two warps of a team must agree on what follows
     if (failed) win_n = 0;
     // ---- ranks: every streaming warp turns the block counts into survivors before each block for itself, 32
     // blocks at a time (a copy per warp costs a few hundred bytes and saves a block-wide barrier behind a single
@@ -586,6 +621,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         if (blockIdx.x == 0 && tid == 0) *p.count = n_surv;
     } else if (streams) {
         int carry = 0;
+#pragma unroll 1
         for (int e0 = 0; e0 < nblk; e0 += 32) {
             const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
             int incl = cnt;
@@ -617,7 +653,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         volatile int *team_flag = reinterpret_cast<volatile int *>(smem + lay.flag) + team;
         const int stream_threads = teams * stride * 32;
         auto team_sync = [&]() {                                      // the warp alone, or the two warps of the team
-            if (p.pp) asm volatile("bar.sync %0, 64;" ::"r"(2 + team) : "memory");
+            if (pp) asm volatile("bar.sync %0, 64;" ::"r"(2 + team) : "memory");
             else __syncwarp();
         };
         bool zeroed = false;
@@ -635,6 +671,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         for (int rb = r_begin;; rb += p.cap) {                        // at least one trip: the teams meet at a barrier in it
             const int cnt = failed ? 0 : max(0, min(p.cap, r_end - rb));
             // ---- column of rank r: the block of keep words that holds it, then the word, then the bit
+#pragma unroll 1
             for (int i = half * 32 + lane; i < cnt; i += 32 * stride) {
                 const int r = rb + i;
                 int j;
@@ -646,6 +683,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 // the block of 32 keep words that holds rank r (the last one with blk[e] <= r), the word in it
                 // (the last one with wrel[w] <= what is left) ...
                 int e = 0;
+#pragma unroll 1
                 for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
                     if (e + step < nblk && myblk[e + step] <= r) e += step;
                 int k = r - myblk[e], w = 32 * e;
@@ -702,9 +740,11 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 ++issued;
                 if (++islot == (uint32_t)Dw) islot = 0;
             };
+#pragma unroll 1
             for (int k = 0, i = half; k < Dw && i < cnt; ++k, i += stride) issue_im(imeta[i]);
             if (!zeroed) {                                          // clear the slab while the first copies fly
                 float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
+#pragma unroll 1
                 for (int i = half * 32 + lane; i < slab_words / 4; i += 32 * stride) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                 zeroed = true;
                 team_sync();
@@ -717,7 +757,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 if (failed) {
                     // The copies still in flight are awaited below.  A warp that gave up keeps meeting its partner at
                     // the hand-overs of this batch, so that nobody waits for it in vain.
-                    if (!p.pp) break;
+                    if (!pp) break;
                     if (lane == 0) *team_flag = 1;
                     if (i > 0) team_sync();
                     if (i + 1 < cnt) team_sync();
@@ -740,7 +780,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 step_fetch(b1, gl, 1, steps, cum, lt_mask, vbase, rbase, zeros);
                 // nothing above touches the accumulator: here the partner hands it over (it has finished the
                 // column before this one)
-                if (p.pp && i > 0) team_sync();
+                if (pp && i > 0) team_sync();
                 step_decode<kRegRows>(b0, cell, spare, reg_lim);                                    // step 0
                 step_fetch(b0, gl, 2, steps, cum, lt_mask, vbase, rbase, zeros);
                 uint32_t q = 1;
@@ -773,12 +813,12 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 // every lane's reads before this point: the copy may overwrite it.
                 __syncwarp();
                 if (refill) issue_im(next_im);
-                if (p.pp && i + 1 < cnt) team_sync();                 // the accumulator goes to the partner
+                if (pp && i + 1 < cnt) team_sync();                 // the accumulator goes to the partner
                 ++consumed;
                 if (++slot == (uint32_t)Dw) { slot = 0; parity ^= 1u; }
             }
             team_sync();                                          // items / imeta are rewritten by the next batch
-            if (p.pp && *team_flag) failed = true;                // both warps of a team stop together
+            if (pp && *team_flag) failed = true;                // both warps of a team stop together
             if (failed || rb + p.cap >= r_end) break;
         }
         if (kRegRows > 0 && zeroed) {                                 // the register rows go to the slab for the merge
@@ -788,10 +828,12 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         }
         if (!zeroed && s < p.S) {                                     // a team without columns still owns a slab
             float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
+#pragma unroll 1
             for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (failed) {
             // give the copies that are still in flight a last (bounded) chance to land before the block goes on
+#pragma unroll 1
             for (; consumed < issued; ++consumed) {
                 mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit);
                 if (++slot == (uint32_t)Dw) { slot = 0; parity ^= 1u; }
@@ -801,7 +843,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     }
     __syncthreads();
 
-    if (p.merge == 1) {
+    if (merge == 1) {
         // ---- a5 by bulk reduce-add.  The block adds its G accumulators; the row segments of its slabs (32*C rows
         // of y each, see the row map) are then dealt to the blocks of the cluster, a block adds its peers' sums
         // for its segments (through distributed shared memory), and the copy engine adds the result into y
@@ -827,6 +869,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         if (G > 1) {
             float4 *acc4 = reinterpret_cast<float4 *>(acc);
             const int group4 = group_words / 4;
+#pragma unroll 1
             for (int q4 = tid; q4 < group4; q4 += nthreads) {
                 float4 v = acc4[q4];
                 for (int gg = 1; gg < G; ++gg) {
@@ -836,18 +879,18 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 acc4[q4] = v;
             }
         }
-        const int seg = p.S == 1 ? 16 : p.C, nseg = (p.R + seg - 1) / seg, seg4 = seg * 8;
-        const int owned = (Sc * nseg - crank + p.cl - 1) / p.cl;   // segments crank, crank + cl, ...
-        if (p.cl > 1) {
+        const int seg = p.S == 1 ? 16 : p.C, nseg = idiv_small(p.R + seg - 1, seg), seg4 = seg * 8;
+        const int owned = (Sc * nseg - crank + cl - 1) / cl;   // segments crank, crank + cl, ...
+        if (cl > 1) {
             cluster_sync();                                         // the peers' sums are complete
             for (int t = tid; t < owned * seg4; t += nthreads) {
-                const int sg = crank + p.cl * (t / seg4), q4 = t % seg4;
+                const int sg = crank + cl * (t / seg4), q4 = t % seg4;
                 const int fsl = sg / nseg, i0 = (sg - fsl * nseg) * seg;
                 if (i0 * 32 + q4 * 4 >= p.R * 32) continue;         // a slab's last segment may be short
                 float4 *cellp = reinterpret_cast<float4 *>(acc + (size_t)fsl * slab_words + (size_t)i0 * 32 + (size_t)q4 * 4);
                 float4 v = *cellp;
-                for (int b = 1; b < p.cl; ++b) {
-                    const float4 u = ld_cluster_f4(smem_u32(cellp), (uint32_t)((crank + b) % p.cl));
+                for (int b = 1; b < cl; ++b) {
+                    const float4 u = ld_cluster_f4(smem_u32(cellp), (uint32_t)((crank + b) % cl));
                     v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
                 }
                 // no other block reads this place: a block reads only the segments it owns, from everybody
@@ -859,12 +902,15 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         // The row map makes local rows [kC, kC + C) of a slab 32*C consecutive rows of y, in accumulator
         // order (with one slab the whole accumulator is y itself): each such segment is one bulk reduce-add.
         {
+#pragma unroll 1
             for (int o = tid; o < owned; o += nthreads) {
-                const int sg = crank + p.cl * o;
-                const int fsl = sg / nseg, k = sg - fsl * nseg, sfull = part * Sc + fsl;
+                const int sg = crank + cl * o;
+                const int fsl = idiv_small(sg, nseg), k = sg - fsl * nseg, sfull = part * Sc + fsl;
                 if (sfull >= p.S) continue;
                 const int i0 = k * seg, i1 = min(p.R, i0 + seg);
-                const int64_t row0 = tile_row(p.S, p.C, sfull, 0, i0);
+                // tile_row(S, C, sfull, 0, i0) for a segment's first local row i0 = k * seg, without its divisions:
+                // seg is C (one chunk of the row map) unless there is one slab, whose rows are y in order
+                const int64_t row0 = p.S == 1 ? (int64_t)i0 * 32 : ((int64_t)(k * p.S + sfull) * p.C) * 32;
                 if (row0 >= p.M) continue;
                 const int nrows = min((i1 - i0) * 32, p.M - (int)row0);
                 const uint32_t bytes = ((uint32_t)nrows * 4u) & ~15u;
@@ -873,13 +919,14 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                     asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(p.y + row0),
                                  "r"(smem_u32(src)), "r"(bytes)
                                  : "memory");
+#pragma unroll 1
                 for (int i = (int)(bytes >> 2); i < nrows; ++i)
                     if (src[i] != 0.f) atomicAdd(p.y + row0 + i, src[i]);
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may go once it has been read
         }
-        if (p.cl > 1) cluster_sync();                               // no block leaves while a peer may still read it
+        if (cl > 1) cluster_sync();                               // no block leaves while a peer may still read it
         if (!kExtras || p.ep_kind == 0) return;
         fused_epilogue(EpilogueArgs{p.y, p.tickets, p.status, p.spin_limit, p.M, p.ep_kind, p.ep_out, p.ep_tau, p.ep_idx,
                                     p.ep_val, p.ep_count});

@@ -494,7 +494,7 @@ extern "C" int celty_count_entries(const uint8_t *mask, int64_t ldm, int64_t M, 
 extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, int32_t groups, int32_t depth,
                                 int32_t cluster)
 {
-    if (!m || grid < 0 || variant < 0 || variant > 253 || groups < 0 || groups > 16 || depth < 0 || depth > 16 ||
+    if (!m || grid < 0 || variant < 0 || variant > 509 || groups < 0 || groups > 16 || depth < 0 || depth > 16 ||
         !(cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4))
         return CELTY_EINVAL;
     m->grid = grid;
@@ -504,6 +504,7 @@ extern "C" int celty_set_launch(celty_matrix *m, int32_t grid, int32_t variant, 
     m->variant = variant & 1;
     m->pairs = (variant & 16) ? 1 : (variant & 32) ? 0 : -1;
     m->mix = (variant & 64) ? 0 : (variant & 128) ? 1 : -1;
+    m->lean = (variant & 256) ? 0 : -1;
     m->groups = groups;
     m->depth = depth;
     m->cluster = cluster;

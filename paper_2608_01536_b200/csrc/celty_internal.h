@@ -102,6 +102,7 @@ struct celty_matrix {
     uint32_t spin_limit = 0;                  // bounded waits inside the kernels: 0 = the library's limit
     int32_t last_grid = 0, last_merge = -1;   // what the tickets in the workspace were last used with
     int32_t mix = -1;       // fused kernel, left-over blocks shared between row parts: 0 never, 1 wherever it is even, -1 where it pays
+    int32_t lean = -1;      // fused kernel: 0 = always the build with every option compiled in
     int32_t no_overlap = 0; // fused kernel: 1 = plain launch (no programmatic dependent launch)
     int32_t merge = -1;     // fused kernel: -1 = library's choice, 0 = ordered two-stage sum, 1 = bulk reduce-add
 };
