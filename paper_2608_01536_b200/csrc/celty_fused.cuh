@@ -55,6 +55,7 @@ struct FusedParams {
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // columns a team looks up per batch
     int win_cols;              // columns of the offset table a block copies into shared memory at its start
+    int clear_rows, clear_extra;   // M / gridDim.x and M mod gridDim.x: block b clears clear_rows (+ 1 if b < clear_extra) rows of y
     // teams that share the survivor list of a row part: units = (column slices of the part) * G;
     // units_inv = floor(2^32 / units) for parts with gridDim / cl / P clusters, units_inv_long for those with
     // one cluster more
@@ -513,7 +514,8 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     // Bulk reduce-add merge: the adds at the end need a cleared y.  The last warp clears this block's share
     // and announces it right away, so that the fence and the ticket overlap the loads of a1.
     if (merge == 1 && warp == nwarps - 1) {
-        const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
+        const int b = (int)blockIdx.x;
+        const int r0 = b * p.clear_rows + min(b, p.clear_extra), r1 = r0 + p.clear_rows + (b < p.clear_extra ? 1 : 0);
 #pragma unroll 1
         for (int i = r0 + lane; i < r1; i += 32) p.y[i] = 0.f;
         if (kExtras && p.ep_kind == 2 && blockIdx.x == 0 && lane == 0) *p.ep_count = 0;   // appended to after the merge
@@ -872,6 +874,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
 #pragma unroll 1
             for (int q4 = tid; q4 < group4; q4 += nthreads) {
                 float4 v = acc4[q4];
+#pragma unroll 2
                 for (int gg = 1; gg < G; ++gg) {
                     const float4 t = acc4[(size_t)gg * group4 + q4];
                     v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;

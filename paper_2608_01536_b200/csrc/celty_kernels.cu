@@ -794,6 +794,8 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
             fp.win_cols = (int)std::min<int64_t>(m->K, words >= 8 ? (int64_t)((words - 8) / m->S) : 0);
         }
         fp.merge = plan.merge;
+        fp.clear_rows = (int)(m->M / plan.grid);
+        fp.clear_extra = (int)(m->M % plan.grid);
         fp.spin_limit = m->spin_limit ? m->spin_limit : kSpinLimit;
         auto inverse = [](uint64_t units) { return units == 1 ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / units); };
         const int nclusters = plan.grid / plan.cl;
