@@ -30,6 +30,32 @@
 // waits are bounded: when one runs out the kernel sets kStatusTimeout in the status word and carries on to a clean
 // exit.
 
+// Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
+// (which sizes the launch with .total), so that the two can never disagree.
+struct FusedSmem {
+    size_t acc, ring, bars, flag, items, imeta, zero, keep, wrel, blk, blkw, total;
+};
+
+__host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
+{
+    FusedSmem l;
+    uint32_t off = 0;
+    l.acc = off;       off += (uint32_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
+    l.ring = off;      off += (uint32_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
+    l.bars = off;      off += (uint32_t)teams * D * 8 + 8;                   // one "full" mbarrier per slot, one for the offset window
+    l.flag = off;      off += (uint32_t)teams * 4;                           // per team: a wait of one of its warps ran out
+    off = (off + 15) / 16 * 16;
+    l.items = off;     off += (uint32_t)teams * cap * 8;                     // {column, x bits} per looked-up item
+    l.imeta = off;     off += (uint32_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
+    l.zero = off;      off += 16;                                          // the all-zero group that idle lanes fetch
+    l.keep = off;      off += ((uint32_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
+    l.wrel = off;      off += ((uint32_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 32
+    l.blk = off;       off += ((uint32_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16; // survivors in each block of 32 keep words
+    l.blkw = off;      off += 16 * (((uint32_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
+    l.total = off;
+    return l;
+}
+
 struct FusedParams {
     const uint32_t *meta;      // [K*S + 1] offset/16 of sub-block (j, s) in the stream
     const uint8_t *stream;
@@ -55,6 +81,7 @@ struct FusedParams {
     int slot_bytes;            // ring slot size, multiple of 128
     int cap;                   // columns a team looks up per batch
     int win_cols;              // columns of the offset table a block copies into shared memory at its start
+    FusedSmem lay;             // the block's shared memory, worked out once on the host (fused_smem_layout)
     int clear_rows, clear_extra;   // M / gridDim.x and M mod gridDim.x: block b clears clear_rows (+ 1 if b < clear_extra) rows of y
     // teams that share the survivor list of a row part: units = (column slices of the part) * G;
     // units_inv = floor(2^32 / units) for parts with gridDim / cl / P clusters, units_inv_long for those with
@@ -271,32 +298,6 @@ __device__ __forceinline__ void step_finish(const StepBuf &b, uint16_t xj)
     for (int e = 0; e < 8; ++e) sts_f32(b.a[e], d[e]);
 }
 
-// Shared-memory carve-up of the fused kernel, computed by ONE function for the kernel and for the host
-// (which sizes the launch with .total), so that the two can never disagree.
-struct FusedSmem {
-    size_t acc, ring, bars, flag, items, imeta, zero, keep, wrel, blk, blkw, total;
-};
-
-__host__ __device__ inline FusedSmem fused_smem_layout(int R, int K, int teams, int D, int slot_bytes, int cap)
-{
-    FusedSmem l;
-    size_t off = 0;
-    l.acc = off;       off += (size_t)teams * (R + kTileSlack) * 32 * 4;   // FP32 accumulators, one slab per team
-    l.ring = off;      off += (size_t)teams * D * slot_bytes;              // bulk-copy ring slots (multiples of 128 bytes)
-    l.bars = off;      off += (size_t)teams * D * 8 + 8;                   // one "full" mbarrier per slot, one for the offset window
-    l.flag = off;      off += (size_t)teams * 4;                           // per team: a wait of one of its warps ran out
-    off = (off + 15) / 16 * 16;
-    l.items = off;     off += (size_t)teams * cap * 8;                     // {column, x bits} per looked-up item
-    l.imeta = off;     off += (size_t)teams * cap * 8;                     // {offset/16, bytes} of its sub-block
-    l.zero = off;      off += 16;                                          // the all-zero group that idle lanes fetch
-    l.keep = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // one keep bit per activation
-    l.wrel = off;      off += ((size_t)((K + 31) / 32) * 4 + 15) / 16 * 16;   // survivors before each keep word, in its block of 32
-    l.blk = off;       off += ((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16; // survivors in each block of 32 keep words
-    l.blkw = off;      off += 16 * (((size_t)((K + 1023) / 1024) * 4 + 15) / 16 * 16);   // per warp: survivors before each block
-    l.total = off;
-    return l;
-}
-
 // Work on the finished y (FusedParams::ep_kind), every block on an equal share of the rows.  A function of its own
 // (not inlined), so that what it needs in registers does not weigh on the streaming loop of the kernel.
 // SiLU(gate) * up evaluated in FP32 and rounded once to FP16 (bit pattern): the one formula behind the work after
@@ -435,7 +436,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
     const int team = streams ? (pp ? (warp & 7) : warp) : 0;
     const int half = streams && pp ? warp >> 3 : 0;               // which of the team's two warps (0 without pp)
     const int stride = 1 + pp, Dw = p.D / stride;                 // columns between a warp's own, ring slots per warp
-    const FusedSmem lay = fused_smem_layout(p.R, p.K, teams, p.D, p.slot_bytes, p.cap);
+    const FusedSmem &lay = p.lay;
     float *acc = reinterpret_cast<float *>(smem + lay.acc);
     uint8_t *ring = smem + lay.ring;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
@@ -579,7 +580,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                     } else if (8 * q + 8 <= p.K) {
                         const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p.x + 8 * q));
                         h[c][0] = v.x; h[c][1] = v.y; h[c][2] = v.z; h[c][3] = v.w;
-                    } else if (q < ngroups) {
+                    } else if (__builtin_expect(q < ngroups, 0)) {
                         const uint4 v = ragged_group(p.x, p.K, q);     // the one group that K cuts short
                         h[c][0] = v.x; h[c][1] = v.y; h[c][2] = v.z; h[c][3] = v.w;
                     }
@@ -627,13 +628,15 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         for (int e0 = 0; e0 < nblk; e0 += 32) {
             const int e = e0 + lane, cnt = e < nblk ? blk[e] : 0;
             int incl = cnt;
+            const int nscan = min(32, nblk - e0);                     // no more steps than there are blocks
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
+                if (d >= nscan) break;
                 const int up = __shfl_up_sync(kFull, incl, d);
                 if (lane >= d) incl += up;
             }
             if (e < nblk) myblk[e] = carry + incl - cnt;
-            carry += __shfl_sync(kFull, incl, 31);
+            carry += __shfl_sync(kFull, incl, min(31, nblk - e0 - 1));   // the last block's inclusive sum
         }
         __syncwarp();
         n_surv = carry;
@@ -714,7 +717,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                     // the two offsets of sub-block (j, s): from the block's window of the table if they are in it
                     const int wq = j * p.S + s - win_w0;
                     uint32_t o0, o1;
-                    if (wq >= 0 && wq + 1 < win_n) {
+                    if (__builtin_expect(wq >= 0 && wq + 1 < win_n, 1)) {
                         o0 = win[wq];
                         o1 = win[wq + 1];
                     } else {
@@ -756,7 +759,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 asm volatile("ld.shared.u32 %0, [%1];" : "=r"(xbits) : "r"(items0 + 8u * (uint32_t)i + 4u));
                 if (!failed && !mbar_wait_bounded(bar0 + 8u * slot, parity, p.spin_limit)) failed = true;
                 failed = __any_sync(kFull, failed);
-                if (failed) {
+                if (__builtin_expect(failed, 0)) {
                     // The copies still in flight are awaited below.  A warp that gave up keeps meeting its partner at
                     // the hand-overs of this batch, so that nobody waits for it in vain.
                     if (!pp) break;
@@ -828,12 +831,12 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             for (int i = 0; i < kRegRows; ++i)
                 if (i < p.R) sts_f32(cell0 + (uint32_t)i * 128u, racc[i]);
         }
-        if (!zeroed && s < p.S) {                                     // a team without columns still owns a slab
+        if (__builtin_expect(!zeroed && s < p.S, 0)) {                // a team without columns still owns a slab
             float4 *slab4 = reinterpret_cast<float4 *>(acc + (size_t)team * slab_words);
 #pragma unroll 1
             for (int i = lane; i < slab_words / 4; i += 32) slab4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (failed) {
+        if (__builtin_expect(failed, 0)) {
             // give the copies that are still in flight a last (bounded) chance to land before the block goes on
 #pragma unroll 1
             for (; consumed < issued; ++consumed) {
@@ -863,7 +866,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
             // the clearing stores of the other blocks (generic proxy) come before this block's reduce-adds
             // (asynchronous proxy) to the same addresses
             asm volatile("fence.proxy.async.global;" ::: "memory");
-            if (!ok) atomicOr(p.status, kStatusTimeout);
+            if (__builtin_expect(!ok, 0)) atomicOr(p.status, kStatusTimeout);
         }
         __syncwarp();
         // add the G accumulators of every slab into the first one
@@ -962,7 +965,7 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 if (ld_acquire_u32(&p.tickets[0]) >= gridDim.x) { ok = true; break; }
                 __nanosleep(32);
             }
-            if (!ok) atomicOr(p.status, kStatusTimeout);
+            if (__builtin_expect(!ok, 0)) atomicOr(p.status, kStatusTimeout);
         }
         __syncthreads();
 

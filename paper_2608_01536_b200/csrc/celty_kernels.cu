@@ -794,6 +794,7 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
             fp.win_cols = (int)std::min<int64_t>(m->K, words >= 8 ? (int64_t)((words - 8) / m->S) : 0);
         }
         fp.merge = plan.merge;
+        fp.lay = fused_smem_layout(m->R, (int)m->K, plan.G * plan.Sc, plan.D, plan.slot_bytes, plan.cap);
         fp.clear_rows = (int)(m->M / plan.grid);
         fp.clear_extra = (int)(m->M % plan.grid);
         fp.spin_limit = m->spin_limit ? m->spin_limit : kSpinLimit;
