@@ -491,7 +491,9 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
         const int c0 = max(0, min(p.K - p.win_cols, mid - p.win_cols / 2));
         win_w0 = (c0 * p.S) & ~3;
         win_n = min(((c0 + p.win_cols) * p.S + 1 - win_w0 + 3) & ~3, ((p.K * p.S + 1 + 3) & ~3) - win_w0);
-        if (tid == 0) {
+        // (by the first lane of the last warp, which is not a streaming warp unless all are: the first lanes of the
+        // streaming warps have their ring barriers to set up at the same time)
+        if (tid == nthreads - 32) {
             mbar_init(win_bar, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
