@@ -358,12 +358,15 @@ __device__ __noinline__ void fused_epilogue(const EpilogueArgs p)
     __syncthreads();
     // every block takes an equal share of the rows; y is read past L1 (it was written by adds in L2)
     if (p.ep_kind == 1) {
-        const int r0 = (int)((int64_t)blockIdx.x * p.M / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * p.M / gridDim.x);
+        // (shares without a 64-bit division: n / blocks rows each, the first n mod blocks one more)
+        const int per = p.M / (int)gridDim.x, extra = p.M - per * (int)gridDim.x, b = (int)blockIdx.x;
+        const int r0 = b * per + min(b, extra), r1 = r0 + per + (b < extra ? 1 : 0);
         for (int i = r0 + tid; i < r1; i += nthreads) p.ep_out[i] = __half_as_ushort(__float2half_rn(__ldcg(p.y + i)));
         return;
     }
     const int half_rows = p.M / 2;
-    const int r0 = (int)((int64_t)blockIdx.x * half_rows / gridDim.x), r1 = (int)((int64_t)(blockIdx.x + 1) * half_rows / gridDim.x);
+    const int per = half_rows / (int)gridDim.x, extra = half_rows - per * (int)gridDim.x, b = (int)blockIdx.x;
+    const int r0 = b * per + min(b, extra), r1 = r0 + per + (b < extra ? 1 : 0);
     for (int base = r0; base < r1; base += nthreads) {          // the same trip count for every thread
         const int i = base + tid;
         bool keep = false;
