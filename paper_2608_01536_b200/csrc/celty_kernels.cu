@@ -488,7 +488,7 @@ __global__ void k_decode_lane(const uint32_t *__restrict__ meta, const uint8_t *
 // asked for), so that steady-state calls make no attribute calls.  The attribute belongs to the kernel,
 // so every entry point that launches a kernel shares that kernel's cache (g_granted_*): two caches for
 // one kernel could disagree about what the runtime currently allows.
-int g_granted_fused[64], g_granted_lean[2][64], g_granted_fused_extras[64], g_granted_column[64], g_granted_lane[64], g_granted_reg[4][64];
+int g_granted_fused[64], g_granted_lean[2][64], g_granted_fused_extras[64], g_granted_lean_extras[2][64], g_granted_column[64], g_granted_lane[64], g_granted_reg[4][64];
 
 template <typename Kernel>
 int ensure_smem(Kernel kernel, size_t bytes, int *granted /* [64], per device */)
@@ -752,10 +752,12 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         rc = fit_clusters(m, &plan);
         if (rc) return rc;
         // the library's default launch has builds of its own (k_spmspv_fused, kLean)
-        const int lean = (!extras && m->reg_rows == 0 && plan.merge == 1 && plan.cl == 1 && m->lean != 0) ? 1 + plan.pp : 0;
+        const int lean = (m->reg_rows == 0 && plan.merge == 1 && plan.cl == 1 && m->lean != 0) ? 1 + plan.pp : 0;
         if (lean) {
-            rc = lean == 2 ? ensure_smem(k_spmspv_fused<false, 0, 2>, plan.smem, g_granted_lean[1])
-                           : ensure_smem(k_spmspv_fused<false, 0, 1>, plan.smem, g_granted_lean[0]);
+            rc = extras ? (lean == 2 ? ensure_smem(k_spmspv_fused<true, 0, 2>, plan.smem, g_granted_lean_extras[1])
+                                     : ensure_smem(k_spmspv_fused<true, 0, 1>, plan.smem, g_granted_lean_extras[0]))
+                        : (lean == 2 ? ensure_smem(k_spmspv_fused<false, 0, 2>, plan.smem, g_granted_lean[1])
+                                     : ensure_smem(k_spmspv_fused<false, 0, 1>, plan.smem, g_granted_lean[0]));
             if (rc) return rc;
         }
         FusedParams fp{};
@@ -832,7 +834,9 @@ int run_product(celty_matrix *m, const void *x_dev, float tau, const ListInput *
         }
         cfg.attrs = attr;
         cfg.numAttrs = na;
-        if (extras) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true, 0>, fp));
+        if (extras && lean == 2) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true, 0, 2>, fp));
+        else if (extras && lean == 1) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true, 0, 1>, fp));
+        else if (extras) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<true, 0>, fp));
         else if (m->reg_rows == 32) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 32>, fp));
         else if (m->reg_rows == 64) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 64>, fp));
         else if (m->reg_rows == 96) CELTY_CUDA(cudaLaunchKernelEx(&cfg, k_spmspv_fused<false, 96>, fp));
