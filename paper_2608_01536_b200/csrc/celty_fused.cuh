@@ -132,10 +132,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// a / b for 0 <= a < 2^16 and 0 < b < 2^7 through one approximate float division (exact for such operands: the
-// quotient of (a + 0.5) is at least 2^-8 away from every integer, far more than the division's error): the block
-// and team indices of the kernel are made of a dozen such quotients, and an integer division is 25 instructions
-// of code that a block runs once.
+// a / b for 0 <= a < 2^20 and b > 0 through one approximate float division.  Exact for such operands: (a + 0.5) / b
+// is at least 0.5 / b away from every integer, and the division's error (2 units in the last place of a value of
+// at most a / b) stays below 2^-22 a / b, which is less than that for a < 2^21.  The block and team indices of the
+// kernel are made of a dozen such quotients, and an integer division is 25 instructions of code that a block runs
+// once.
 __device__ __forceinline__ int idiv_small(int a, int b)
 {
     return (int)__fdividef((float)a + 0.5f, (float)b);
