@@ -395,6 +395,9 @@ int celty_last_status(celty_matrix *m, celty_stream_t stream);
  *            over can be shared evenly, each of them can serve several parts with correspondingly fewer teams per
  *            part, instead of giving some parts one block more than others, which leaves those blocks idle at the
  *            end.  By default the library does so where the parts have few enough blocks each for that to pay.)
+ *            256 = run the build of the fused kernel that has every option compiled in even where the launch is
+ *            the default one (bulk reduce-add merge, no clusters), for which the library otherwise uses smaller
+ *            builds without the other options' code (same results; the smaller builds are faster).
  *   groups   fused kernel: warp teams per slab working on different columns (each has an accumulator)
  *   depth    fused kernel: bulk copies each team keeps in flight (ring slots)
  *   cluster  fused kernel, bulk reduce-add merge: thread blocks per cluster (1, 2 or 4); the blocks of a

@@ -217,7 +217,8 @@ def test_spmspv_integer_data_is_bit_exact(layout, M, K, d_w, d_a, tile_rows, spb
     m = _matrix(W, mask, layout, tile_rows, spb)
     for grid, groups, depth, cluster in ((0, 0, 0, 0), (1, 0, 0, 1), (3, 1, 1, 4), (36, 3, 2, 2), (148, 2, 4, 1),
                                         (148, 0, 0, 4), (7, 16, 0, 2)):
-        for pairs in ((0, 16, 32) if layout == (celty.LAYOUT_LANE_TILE, 0) else (0,)):     # warp pairs: auto, always, never
+        # warp pairs: auto, always, never; 256: the build with every option compiled in instead of the lean ones
+        for pairs in ((0, 16, 32, 256, 256 + 16) if layout == (celty.LAYOUT_LANE_TILE, 0) else (0,)):
             m.set_launch(grid=grid, variant=m.variant + pairs, groups=groups, depth=depth, cluster=cluster)
             y = _run(m, x, tau)
             _check_y(y, W, mask, x, tau, exact=True)
@@ -272,7 +273,7 @@ def test_random_shapes_and_options(case):
         return
     grid, groups, depth, cluster = (int(rng.choice([0, 0, 1, 5, 40, 148])), int(rng.choice([0, 0, 1, 3])),
                                     int(rng.choice([0, 0, 1, 3])), int(rng.choice([0, 1, 2, 4])))
-    variant = int(rng.choice([0, 0, 2, 8, 16, 24, 32, 64, 128, 144]))
+    variant = int(rng.choice([0, 0, 2, 8, 16, 24, 32, 64, 128, 144, 256, 272, 288]))
     m.set_launch(grid=grid, variant=variant, groups=groups, depth=depth, cluster=cluster)
     _check_y(_run(m, x, tau), W, mask, x, tau)
     idx, val = m.last_compaction()
