@@ -48,6 +48,11 @@ void choose_shape(int64_t M, int64_t K, double density, int tile_rows, int64_t *
         S = (Q + R - 1) / R;
     } else {
         S = std::max<int64_t>(1, (M + 4095) / 4096);
+        // A layer of one slab and few columns streams for so short a time that the merge dominates: two slabs
+        // halve what every block adds up and adds into y (and the contributors per row), for twice as many
+        // sub-blocks of half the size.  Measured at 4096 x 4096: 8.3 us against 8.8; at 4096 x 11008, where a team
+        // has five sub-blocks to stream, no gain, so the rule stops short of it.
+        if (S == 1 && Q >= 32 && K <= 6144) S = 2;
         auto rows_for = [&](int64_t slabs) { return std::max<int64_t>(16, ((Q + slabs - 1) / slabs + 15) / 16 * 16); };
         auto teams_that_fit = [&](int64_t rows) {
             const double entries = 32.0 * rows * density;             // of one sub-block, mean; + 3.5 sigma for the largest

@@ -536,9 +536,15 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
         // no more teams than a block can have columns (a tiny layer then leaves half the shared memory free, and
         // the next call's block can set itself up beside this one: 5.25 -> 4.95 us at 1024 x 1024)
         const int64_t cols_per_block = (m->K + std::max(1, pl.grid / pl.P) - 1) / std::max(1, pl.grid / pl.P);
-        const int g_cap = (int)std::max<int64_t>(1, std::min<int64_t>(((reg_rows > 0 || pairs) ? 8 : 16) / pl.Sc, cols_per_block));
+        // Eight teams saturate the shared-memory data path; more of them only pay where a team has a long list of
+        // columns to stream (5120 x 13824: 11 teams 4 % faster than 8), and otherwise cost what the block has to
+        // add up at the end (4096 x 4096 at 64 rows per tile: 9.1 us with 13 teams, 8.3-8.5 with 7 to 10).
+        const int most = (reg_rows > 0 || pairs || cols_per_block < 96) ? 8 : 16;
+        const int g_cap = (int)std::max<int64_t>(1, std::min<int64_t>(most / pl.Sc, cols_per_block));
         const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
-        int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 4;
+        // two ring slots per team unless asked otherwise: deeper rings measured no faster anywhere, and slower where
+        // they only add set-up (4096 x 4096 at 64 rows per tile, eight teams: 8.5 us with two slots, 8.7 with four)
+        int d_min = m->depth > 0 ? m->depth : 2, d_max = m->depth > 0 ? m->depth : 2;
         if (pairs) {
             d_min = std::max(2, d_min + (d_min & 1));
             d_max = std::max(d_min, d_max & ~1);
