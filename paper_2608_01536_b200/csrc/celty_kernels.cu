@@ -625,6 +625,7 @@ int max_active_clusters(int cl, size_t smem, int threads, int *out)
     return CELTY_OK;
 }
 
+// fall back to smaller clusters while the device cannot hold the whole grid of them at once
 int fit_clusters_only(FusedPlan *plan)
 {
     while (plan->cl > 1) {
@@ -638,9 +639,8 @@ int fit_clusters_only(FusedPlan *plan)
     return CELTY_OK;
 }
 
-// fall back to smaller clusters while the device cannot hold the whole grid of them at once; then, without
-// clusters, decide whether the blocks that are left over when the grid is dealt to the row parts serve several
-// parts each (FusedParams::mix): only where they can be shared evenly
+// the cluster size the device can hold; then, without clusters, whether the blocks that are left over when the grid
+// is dealt to the row parts serve several parts each (FusedParams::mix): only where they can be shared evenly
 int fit_clusters(const celty_matrix *m, FusedPlan *plan)
 {
     const int rc = fit_clusters_only(plan);
