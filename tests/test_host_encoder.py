@@ -221,3 +221,19 @@ def test_stored_entries_and_layout_statistics_against_the_oracle():
     col = celty.Matrix(W, mask, layout=celty.LAYOUT_COLUMN)
     with pytest.raises(celty.CeltyError):
         col.layout_stats()
+
+
+@pytest.mark.parametrize("M,K,slabs,rows", [(4096, 4096, 2, 64), (4096, 6144, 2, 64), (4096, 6145, 1, 128), (4096, 11008, 1, 128),
+                                            (1024, 1024, 2, 16), (512, 512, 1, 16), (5120, 5120, 2, 80), (11008, 4096, 3, 128),
+                                            (28672, 64, 8, 120)])
+def test_default_tile_shape(M, K, slabs, rows):
+    """The library's own choice of slabs and rows per tile: one slab per 4096 rows, two for a layer of one slab and
+    few columns (it streams for so short a time that halving what a block adds into y at the end is worth more than
+    large sub-blocks), fewer rows per tile on very tall layers so that eight teams fit shared memory.  Every row has
+    exactly one place whatever the shape."""
+    W = synth.weights(77, M, K) if M * K <= 1 << 22 else np.zeros((M, K), np.float16)
+    mask = synth.mask_bernoulli(78, M, K, 0.5)
+    m = celty.Matrix(W, mask)
+    S, R, C = m.row_map()
+    assert (S, R) == (slabs, rows)
+    assert 32 * S * R >= M and R % C == 0
