@@ -538,8 +538,9 @@ int plan_fused(const celty_matrix *m, const DeviceInfo &di, FusedPlan *out)
         const int64_t cols_per_block = (m->K + std::max(1, pl.grid / pl.P) - 1) / std::max(1, pl.grid / pl.P);
         // Eight teams saturate the shared-memory data path; more of them only pay where a team has a long list of
         // columns to stream (5120 x 13824: 11 teams 4 % faster than 8), and otherwise cost what the block has to
-        // add up at the end (4096 x 4096 at 64 rows per tile: 9.1 us with 13 teams, 8.3-8.5 with 7 to 10).
-        const int most = (reg_rows > 0 || pairs || cols_per_block < 96) ? 8 : 16;
+        // add up at the end (4096 x 4096 at 64 rows per tile: 9.1 us with 13 teams, 8.3-8.5 with 7 to 10; 11008 x 4096
+        // at 88 rows per tile, 110 columns to a block: 12.7 us with 10 teams, 12.3 with 8 pairs).
+        const int most = (reg_rows > 0 || pairs || cols_per_block < 128) ? 8 : 16;
         const int g_cap = (int)std::max<int64_t>(1, std::min<int64_t>(most / pl.Sc, cols_per_block));
         const int g_max = std::max(1, std::min(g_cap, m->groups > 0 ? m->groups : g_cap));
         // two ring slots per team unless asked otherwise: deeper rings measured no faster anywhere, and slower where
