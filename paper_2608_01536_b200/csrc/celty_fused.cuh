@@ -693,14 +693,29 @@ __global__ void __launch_bounds__(kRegRows > 0 ? 256 : 512, 1) k_spmspv_fused(co
                 } else {
                 // the block of 32 keep words that holds rank r (the last one with blk[e] <= r), the word in it
                 // (the last one with wrel[w] <= what is left) ...
+                // (both tables are nondecreasing, so "the last entry <= r" is a count of such entries, and counting
+                // takes independent loads where a binary search takes dependent ones: up to eight blocks in one
+                // round, the 32 words of a block in two -- quarters, then the eight words of the quarter)
                 int e = 0;
-#pragma unroll 1
-                for (int step = 1 << (31 - __clz(max(1, nblk - 1))); step; step >>= 1)
-                    if (e + step < nblk && myblk[e + step] <= r) e += step;
-                int k = r - myblk[e], w = 32 * e;
+                if (nblk <= 8) {
 #pragma unroll
-                for (int step = 16; step; step >>= 1)
-                    if (w + step < nwords && wrel[w + step] <= k) w += step;
+                    for (int u = 1; u < 8; ++u) e += (u < nblk && myblk[u] <= r) ? 1 : 0;
+                } else {
+#pragma unroll 1
+                    for (int step = 1 << (31 - __clz(nblk - 1)); step; step >>= 1)
+                        if (e + step < nblk && myblk[e + step] <= r) e += step;
+                }
+                int k = r - myblk[e], w = 32 * e;
+                {
+                    int quarter = 0;
+#pragma unroll
+                    for (int u = 8; u < 32; u += 8) quarter += (w + u < nwords && wrel[w + u] <= k) ? 1 : 0;
+                    w += 8 * quarter;
+                    int in_quarter = 0;
+#pragma unroll
+                    for (int u = 1; u < 8; ++u) in_quarter += (w + u < nwords && wrel[w + u] <= k) ? 1 : 0;
+                    w += in_quarter;
+                }
                 k -= wrel[w];
                 // ... and the bit in it: halve the word, keep the half that holds the wanted set bit
                 const uint32_t word = kbw[w];
