@@ -765,8 +765,8 @@ def run_regsplit_study(args):
 
 def run_batch_study(args):
     """Small batches (Sections 2.2-2.3 place the method against SpMM kernels that need N >= 8): microseconds per
-    batch of N activation vectors through celty_spmspv_batch (union of the surviving columns, N accumulators per
-    row; the simple two-launch kernels), beside N calls of the single-vector kernel and the dense cuBLAS FP16 GEMM
+    batch of N activation vectors through celty_spmspv_batch with the widened kernels (union of the surviving columns,
+    N accumulators per row; two launches) and as the library runs it by default, beside N calls of the single-vector kernel and the dense cuBLAS FP16 GEMM
     on the same weights, under the same rotation."""
     import torch
     from paper_2608_01536_b200 import build as lib_build, celty
@@ -801,11 +801,17 @@ def run_batch_study(args):
                 g.replay()
                 reps = max(3, -(-args.sweep_calls // len(calls)))
                 return float(np.median(timed_regions(torch, g.replay, reps, min_total_s=0.05))) * 1e3 / (reps * len(calls))
+            for mt in mats:
+                mt.set_launch(variant=1)                              # the widened two-launch kernels
             us_batch = timed([(lambda c=c: mats[c].spmspv_batch(xs[c], tau, ys[c])) for c in range(copies)])
+            for mt in mats:
+                mt.set_launch()
+            us_default = timed([(lambda c=c: mats[c].spmspv_batch(xs[c], tau, ys[c])) for c in range(copies)])
             us_single = timed([(lambda c=c, n=n: mats[c].spmspv(xs[c][n], tau, ys[c][n])) for c in range(copies) for n in range(N)]) * N
             us_gemm = timed([(lambda c=c: torch.mm(Wd[c % len(Wd)], xs[c].t(), out=yd)) for c in range(copies)])
             keep = [np.abs(X[c].astype(np.float32)) > np.float32(tau) for c in range(copies)]
-            points.append({"workload": name, "N": N, "us_per_batch": us_batch, "us_N_single_calls": us_single,
+            points.append({"workload": name, "N": N, "us_per_batch": us_batch, "us_per_batch_default": us_default,
+                           "us_N_single_calls": us_single,
                            "us_cublas_gemm": us_gemm,
                            "union_density": float(np.mean([k.any(axis=0).mean() for k in keep])),
                            "activation_density": float(np.mean([k.mean() for k in keep]))})

@@ -241,9 +241,13 @@ int celty_spmspv_list(celty_matrix *m, const int32_t *idx_dev, const uint16_t *v
 /*
  * celty_spmspv_batch -- the product for a small batch of N = 1 .. 8 activation vectors against the same matrix
  * (LANE_TILE handles):  y[n] = W . threshold(x[n], tau)  for every n.  Sections 2.2-2.3 place the method against
- * SpMM kernels that need N >= 8; this call keeps the batch-1 scheme and widens it: a column is fetched once when any
- * of the N activations in it survives (the union of the surviving columns), and every stored entry is multiplied
- * into N accumulators.  Two launches (union compaction, product with plain loads and an atomic merge).
+ * SpMM kernels that need N >= 8.  Two ways are built.  The widened scheme: a column is fetched once when any of the
+ * N activations in it survives (the union of the surviving columns), and every stored entry is multiplied into N
+ * accumulators; two launches (union compaction, product with plain loads and an atomic merge); taken when the
+ * handle runs the two-launch variant (celty_set_launch, variant 1), has no workspace bound, or a row of x or y
+ * does not start on a 16-byte boundary.  Otherwise N launches of the single-vector kernel, which measured faster at
+ * every N (the widened kernels have room for fewer warps, and the union is nearly every column from N = 4 on);
+ * celty_last_compaction then reports the last vector's list.
  *   x_dev  N rows of K FP16 values, row n at x_dev + n * ldx (elements), not modified
  *   y_dev  N rows of M FP32 values, row n at y_dev + n * ldy, overwritten
  *   list_scratch_dev  device scratch, 256-byte aligned, at least 256 + round_up(4 K, 256) + 16 K bytes (union list

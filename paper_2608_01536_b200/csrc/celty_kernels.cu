@@ -999,6 +999,18 @@ extern "C" int celty_spmspv_batch(celty_matrix *m, const void *x_dev, int64_t ld
     const size_t need = 256 + round_up((size_t)m->K * 4, 256) + (size_t)8 * m->K * 2;
     if (scratch_bytes < need || ((uintptr_t)list_scratch_dev & 255)) return CELTY_ENOMEM;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Measured, the widened kernels below lose to the single-vector kernel called N times at every N (N accumulators
+    // per warp leave room for fewer warps, and the union of N activation patterns is nearly every column from N = 4
+    // on): unless the two-launch variant is asked for, the batch is N launches of the single-launch kernel, where the
+    // handle has its workspace and every row of x and y starts on a 16-byte boundary.
+    if (m->variant == 0 && m->d_ws && !(((uintptr_t)x_dev | (uintptr_t)(ldx * 2) | (uintptr_t)y_dev | (uintptr_t)(ldy * 4)) & 15)) {
+        for (int32_t n = 0; n < N; ++n) {
+            const int rc1 = celty_spmspv(m, static_cast<const uint16_t *>(x_dev) + (size_t)n * ldx, tau,
+                                         static_cast<float *>(y_dev) + (size_t)n * ldy, stream);
+            if (rc1) return rc1;
+        }
+        return CELTY_OK;
+    }
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc) return rc;

@@ -21,15 +21,17 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
+@pytest.mark.parametrize("variant", [0, 1])          # N launches of the single-vector kernel / the widened kernels
 @pytest.mark.parametrize("N", [1, 2, 3, 4, 5, 8])
 @pytest.mark.parametrize("M,K,d_w,d_a", [(1000, 520, 0.5, 0.5), (4096, 1024, 0.3, 0.2), (11008, 300, 0.5, 0.9),
                                          (28672, 96, 0.5, 0.5)])
-def test_batch_matches_independent_products(N, M, K, d_w, d_a):
+def test_batch_matches_independent_products(N, M, K, d_w, d_a, variant):
     W = synth.weights(M + K, M, K)
     mask = synth.mask_bernoulli(M + K, M, K, d_w)
     X = np.stack([synth.activations(100 * n + K, K, "laplace") for n in range(N)])
     tau = synth.threshold_for_density(X[0], d_a)
     m = celty.Matrix(W, mask, device="cuda")
+    m.set_launch(variant=variant)
     Y = m.spmspv_batch(_dev(X), tau, y=torch.full((N, M), 4.0, device="cuda"))
     torch.cuda.synchronize()
     got = Y.cpu().numpy().astype(np.float64)
